@@ -1,0 +1,175 @@
+"""CPU oracle: the speculative-decoding block loop around a multimodal target.
+
+TEST INFRASTRUCTURE ONLY -- see oracle/llama.py.  Shares no code with the CUDA path.
+
+Follows Sec. 2.1 and Sec. 3 of the paper, step by step (letters: p = target, q = draft):
+
+1. prefill: the target reads [V_1..V_m ; embed(X_1..X_n)] (Eq. 1) and its last row gives
+   the first generated token; the draft reads embed(X_1..X_n) only (Sec. 3), or, for the
+   draft with an image adapter (Sec. 4 "Draft Model Candidates", Appendix A.1), the rows
+   [H W_a^T ; embed(X)];
+2. draft: gamma tokens, auto-regressively, x_j ~ q_j(. | text so far) (Sec. 2.1);
+3. verify: ONE target call on [pending, x_1..x_gamma] gives p_1..p_{gamma+1}; the
+   rejection rule of oracle/sampling.py decides the accepted count a and the next token;
+4. commit: x_1..x_a and the next token are emitted; both caches are cut back to the rows
+   of emitted tokens (the paper is silent on caches; rows of rejected tokens are simply
+   overwritten by the next block).
+
+The last emitted token ("pending") has not been fed to either model yet.  `seq` holds the
+prompt followed by every emitted token; position of pending in the target = m + len(seq)-1.
+
+Pinned by tests/test_oracle_spd.py: greedy speculative output == the target's own greedy
+continuation (Sec. 4 "Decoding"), block efficiency <= gamma + 1, cache state after a
+rejection == a fresh model fed only the emitted tokens.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from .llama import Model, F32
+from . import sampling as S
+
+
+class SpdOracle:
+    def __init__(self, target: Model, draft: Model, temperature: float = 1.0,
+                 greedy: bool = False, adapter_w: np.ndarray | None = None):
+        self.t, self.d = target, draft
+        self.temperature, self.greedy = float(temperature), bool(greedy)
+        self.adapter_w = adapter_w  # fp32 [d_draft, adapter_in] or None
+        self.tc = self.dc = None
+        self.last_logits = None
+        self.last_draft_logits = None
+
+    # ---- helpers
+    def _pick(self, logits_row: np.ndarray, u):
+        if self.greedy:
+            return S.argmax_lowest(logits_row), None
+        prob = S.softmax_t(logits_row, self.temperature)
+        return S.sample_fixed_point(prob, u), prob
+
+    @property
+    def pending(self) -> int:
+        return self.seq[-1]
+
+    # ---- step 1
+    def prefill(self, image_embeds, prompt_ids, u0=None, draft_image_feats=None):
+        prompt_ids = [int(x) for x in prompt_ids]
+        self.m = 0 if image_embeds is None else int(image_embeds.shape[0])
+        self.tc, self.dc = self.t.new_cache(), self.d.new_cache()
+        rows = self.t.embed(prompt_ids)
+        if self.m:
+            rows = np.concatenate([np.asarray(image_embeds, dtype=F32), rows], axis=0)
+        logits = self.t.forward(self.tc, rows, 0)
+        self.prefill_logits = logits[-1]
+        x0, _ = self._pick(logits[-1], u0)
+
+        drows = self.d.embed(prompt_ids)
+        self.off = 0
+        if self.adapter_w is not None:
+            adapted = np.asarray(draft_image_feats, dtype=F32) @ self.adapter_w.T
+            drows = np.concatenate([adapted, drows], axis=0)
+            self.off = adapted.shape[0]
+        self.d.forward(self.dc, drows, 0)
+        self.seq = prompt_ids + [x0]
+        self.d_fed = len(prompt_ids)      # tokens of seq whose rows the draft cache holds
+        self.n_prompt = len(prompt_ids)
+        return x0
+
+    def set_state(self, seq):
+        """Replace the committed sequence (prompt + emitted tokens) by one that shares a
+        prefix with the current one; caches keep the rows of the shared prefix."""
+        seq = [int(x) for x in seq]
+        common = 0
+        for a, b in zip(seq, self.seq):
+            if a != b:
+                break
+            common += 1
+        self.d_fed = min(self.d_fed, common, len(seq) - 1)
+        self.seq = seq
+        self.tc.length = self.m + len(seq) - 1
+
+    # ---- step 2
+    def draft(self, gamma: int, u_draft):
+        ids, probs, raw = [], [], []
+        feed = self.seq[self.d_fed:]                    # pending, plus an unseen accepted token
+        pos0 = self.off + self.d_fed
+        for j in range(gamma):
+            logits = self.d.forward(self.dc, self.d.embed(feed), pos0)
+            raw.append(logits[-1])
+            x, prob = self._pick(logits[-1], None if self.greedy else u_draft[j])
+            ids.append(x)
+            probs.append(prob)
+            pos0 += len(feed)
+            feed = [x]
+        self.last_draft_logits = np.stack(raw) if raw else None
+        q = None if (self.greedy or gamma == 0) else np.stack(probs).astype(F32)
+        return np.asarray(ids, dtype=np.int32), q
+
+    # ---- steps 3 and 4
+    def verify(self, ids, q, u):
+        ids = [int(x) for x in ids]
+        gamma = len(ids)
+        pos0 = self.m + len(self.seq) - 1
+        logits = self.t.forward(self.tc, self.t.embed([self.pending] + ids), pos0)
+        self.last_logits = logits
+        if self.greedy:
+            a, nxt = S.reject_sample(logits, None, ids, None, greedy=True)
+        else:
+            p = S.softmax_t(logits, self.temperature)
+            self.last_p = p
+            a, nxt = S.reject_sample(p, q, ids, u, greedy=False)
+        old_len = len(self.seq)
+        self.seq += ids[:a] + [nxt]
+        self.tc.length = self.m + len(self.seq) - 1
+        if gamma > 0:   # the draft holds rows for the old sequence and x_1..x_{gamma-1}
+            self.d_fed = old_len + min(a, gamma - 1)
+        self.dc.length = self.off + self.d_fed
+        return a, nxt
+
+    def target_decode(self, u=None) -> int:
+        """Plain auto-regressive step of the target alone: a block with gamma = 0."""
+        _, nxt = self.verify([], None, None if self.greedy else [u])
+        return nxt
+
+    # ---- loops
+    def generate(self, n_new: int, gamma: int, uniforms):
+        """Emit until n_new tokens after the prompt exist (the prefill's token counts as
+        the first).  uniforms [n_blocks_max, 2*gamma+1]: gamma for the draft's draws, then
+        gamma+1 for the verification.  Returns (tokens [n_new], stats)."""
+        start = self.n_prompt
+        blocks = accepted = 0
+        while len(self.seq) - start < n_new:
+            ub = None if uniforms is None else uniforms[blocks]
+            ids, q = self.draft(gamma, None if ub is None else ub[:gamma])
+            a, _ = self.verify(ids, q, None if ub is None else ub[gamma:])
+            blocks += 1
+            accepted += a
+        emitted = len(self.seq) - start - 1   # tokens produced by the blocks themselves
+        out = np.asarray(self.seq[start:start + n_new], dtype=np.int32)
+        return out, {"blocks": blocks, "accepted": accepted,
+                     "tau": emitted / max(blocks, 1)}
+
+    def generate_target_only(self, n_new: int, uniforms=None):
+        start = self.n_prompt
+        step = 0
+        while len(self.seq) - start < n_new:
+            self.target_decode(None if uniforms is None else uniforms[step])
+            step += 1
+        return np.asarray(self.seq[start:start + n_new], dtype=np.int32)
+
+
+def block_efficiency_closed_form(alpha: float, gamma: int) -> float:
+    """Expected tokens per target call when each draft token is accepted independently
+    with probability alpha: 1 + alpha + ... + alpha^gamma (bounded by gamma + 1, the
+    maximum of block efficiency stated in Sec. 4 "Metrics")."""
+    if abs(1.0 - alpha) < 1e-12:
+        return float(gamma + 1)
+    return (1.0 - alpha ** (gamma + 1)) / (1.0 - alpha)
+
+
+def mbsu(tau: float, c: float, gamma: int) -> float:
+    """Memory-bound speed-up (Sec. 4 "Metrics") with c = draft/target parameter ratio.
+    The printed formula c*tau/(c*gamma+1) cannot produce the paper's 2.37x for c ~ 0.017;
+    it is read as tau / (c*gamma + 1): a block costs gamma draft steps of relative cost c
+    plus one target step, and yields tau tokens."""
+    return tau / (c * gamma + 1.0)

@@ -1,0 +1,96 @@
+"""Pins for the CPU oracle's block loop (oracle/spd.py) on the tiny workload.  CPU only.
+
+The paper fixes one exact behaviour: with greedy decoding the speculative output is
+identical to the target's own auto-regressive output (Sec. 4 "Decoding"), for any draft
+and any block size.  Beyond that: block efficiency <= gamma + 1 (Sec. 4 "Metrics"), the
+caches after a rejection hold exactly the emitted tokens, and with the draft equal to the
+target every token is accepted.
+"""
+import numpy as np
+import pytest
+
+import synth
+from oracle import llama
+from oracle.spd import SpdOracle
+
+F32 = np.float32
+
+
+def build(wl, temperature=1.0, greedy=False, same_draft=False, std=0.02):
+    tw = synth.Weights(wl.target, wl.seeds["weights"], "target", std=std)
+    dw = tw if same_draft else synth.Weights(wl.draft, wl.seeds["weights"], "draft",
+                                             adapter_in=wl.adapter_in, std=std)
+    t = llama.Model(wl.target, tw, 128)
+    d = llama.Model(wl.target if same_draft else wl.draft, dw, 128)
+    ad = dw.f32("adapter") if wl.adapter_in and not same_draft else None
+    return SpdOracle(t, d, temperature, greedy, adapter_w=ad)
+
+
+@pytest.mark.parametrize("gamma", [1, 3, 4])
+def test_greedy_speculative_equals_target_only(gamma):
+    # std 0.2 so that logits are well separated and the draft agrees with the target now
+    # and then (both accept and reject paths run)
+    wl = synth.tiny_workload(gamma)
+    img, ids = synth.image_embeds(wl), synth.prompt_ids(wl)
+    a = build(wl, greedy=True, std=0.2)
+    a.prefill(img, ids)
+    spd, st = a.generate(wl.n_new, gamma, None)
+    b = build(wl, greedy=True, std=0.2)
+    b.prefill(img, ids)
+    ar = b.generate_target_only(wl.n_new)
+    assert np.array_equal(spd, ar)
+    assert 1.0 <= st["tau"] <= gamma + 1
+    assert st["blocks"] <= wl.n_new
+
+
+def test_identical_draft_accepts_all_and_tau_is_gamma_plus_one():
+    wl = synth.Workload("same", synth.TINY_TARGET, synth.TINY_TARGET, 0, 16, 3, 24)
+    ids = synth.prompt_ids(wl)
+    for greedy in (True, False):
+        o = build(wl, greedy=greedy, same_draft=True, std=0.2)
+        o.prefill(None, ids, u0=0.3)
+        u = synth.uniforms(3, "same.spd", (wl.n_new, 2 * 3 + 1))
+        out, st = o.generate(wl.n_new, 3, None if greedy else u)
+        assert st["accepted"] == 3 * st["blocks"]
+        assert st["tau"] == 4.0
+
+
+def test_sampling_loop_caches_hold_exactly_the_emitted_tokens():
+    wl = synth.tiny_workload(4)
+    img, ids = synth.image_embeds(wl), synth.prompt_ids(wl)
+    o = build(wl, temperature=1.0, std=0.1)
+    o.prefill(img, ids, u0=0.5)
+    u = synth.uniforms(3, "loop", (wl.n_new, 9))
+    out, st = o.generate(20, 4, u)
+    assert st["tau"] <= 5 and len(out) == 20
+    assert st["accepted"] > 0                      # accept path exercised
+    assert st["accepted"] < 4 * st["blocks"]       # reject path exercised
+    # the target's next logits equal those of a fresh model fed only the emitted tokens
+    seq = list(o.seq)
+    nxt_logits = o.t.forward(o.tc, o.t.embed([seq[-1]]), o.m + len(seq) - 1)[0]
+    fresh = build(wl, std=0.1)
+    rows = np.concatenate([img, fresh.t.embed(seq)], 0)
+    want = fresh.t.forward(fresh.t.new_cache(), rows, 0)[-1]
+    assert np.abs(nxt_logits - want).max() < 2e-5
+    # same for the draft (text rows only)
+    dl = o.d.forward(o.dc, o.d.embed(seq[o.d_fed:]), o.off + o.d_fed)[-1]
+    dwant = fresh.d.forward(fresh.d.new_cache(), fresh.d.embed(seq), 0)[-1]
+    assert np.abs(dl - dwant).max() < 2e-5
+
+
+def test_draft_with_image_adapter_sees_projected_features():
+    wl = synth.tiny_workload(4, adapter=True)
+    img, ids, feats = synth.image_embeds(wl), synth.prompt_ids(wl), synth.image_features(wl)
+    o = build(wl, greedy=True, std=0.2)
+    o.prefill(img, ids, draft_image_feats=feats)
+    assert o.off == wl.n_image and o.dc.length == wl.n_image + wl.n_prompt
+    d_ids, _ = o.draft(4, None)
+    # the draft's first logits equal a cache-free pass over [H W_a^T ; embed(text)]
+    rows = np.concatenate([feats @ o.adapter_w.T, o.d.embed(o.seq)], 0)
+    want = o.d.forward_full(rows)[-1]
+    assert np.abs(o.last_draft_logits[0] - want).max() < 2e-5
+    # and differ from a text-only draft's (the image rows matter)
+    t = build(synth.tiny_workload(4), greedy=True, std=0.2)
+    t.prefill(img, ids)
+    t.draft(4, None)
+    assert np.abs(t.last_draft_logits[0] - want).max() > 1e-3
