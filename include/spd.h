@@ -1,0 +1,195 @@
+/*
+ * spd.h -- C ABI of the speculative-decoding verification path for a multimodal target.
+ *
+ * The operations follow the paper's statement of the problem (letters: p = target,
+ * q = draft; the paper uses the opposite letters):
+ *   - the target generates conditioned on m projected image embeddings followed by the
+ *     text, X_{n+1} ~ p(. | V_1..V_m, X_1..X_n)                      (Sec. 2.2, Eq. 1);
+ *   - a small draft of the same architecture proposes gamma tokens auto-regressively from
+ *     the text alone, x_j ~ q(. | X, x_1..x_{j-1})                    (Sec. 2.1, Sec. 3);
+ *   - ONE target call scores all of them; token j is accepted with probability
+ *     min{1, p_j(x_j)/q_j(x_j)}, the first rejected one is replaced by a draw from the
+ *     normalised residual max(0, p_j - q_j), and if none is rejected one more token is
+ *     drawn from the target's next row                                (Sec. 2.1, Sec. 3,
+ *     Sec. 4 "Metrics": at most gamma + 1 tokens per target call);
+ *   - with greedy decoding the output equals the target's own greedy continuation
+ *                                                                     (Sec. 4 "Decoding").
+ *
+ * Conventions
+ *   - Every function returns spd_status; none throws, aborts or traps the device.
+ *     spd_last_error() gives a message for the last non-OK status of a context.
+ *   - "device" pointers are CUDA device memory of the context's device; "host or device"
+ *     pointers are classified with cudaPointerGetAttributes.  All work is enqueued on
+ *     cfg.stream; a call that returns results into HOST memory synchronises that stream
+ *     before returning, a call with only device outputs does not.
+ *   - The caller owns every buffer it passes.  spd_create makes its own (repacked) device
+ *     copy of the weights, so the caller may free them afterwards.
+ *   - Matrices are row-major [out, in], in the model's dtype (0 = fp32, 1 = bfloat16);
+ *     norm gains are fp32 [d_model]; there are no biases.
+ *   - One sequence per context (batch 1).
+ *   - Call order: create -> prefill -> (draft -> verify)* ; anything else is SPD_ESTATE.
+ */
+#ifndef SPD_H_
+#define SPD_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct spd_ctx spd_ctx;
+
+typedef enum {
+  SPD_OK = 0,
+  SPD_EINVAL = 1,    /* bad argument or unsupported shape */
+  SPD_ESTATE = 2,    /* call out of order */
+  SPD_ENOMEM = 3,    /* device or host allocation failed */
+  SPD_EOVERFLOW = 4, /* KV cache (max_seq) or gamma_max would be exceeded */
+  SPD_ECUDA = 5,     /* a CUDA call failed */
+  SPD_ETIMEOUT = 6,  /* a bounded device-side wait ran out; the context stays usable */
+  SPD_ENOTIMPL = 7
+} spd_status;
+
+/* LLaMA-style decoder (Table 1: layers, heads, intermediate dim, hidden dim, SiLU). */
+typedef struct {
+  int n_layers, d_model, n_heads, d_ffn, vocab;
+  int tied_embeddings; /* 1: LM head = token embedding table */
+  float rms_eps;       /* RMSNorm epsilon (1e-5) */
+  float rope_theta;    /* rotary base (10000); pairs are (i, i + d_head/2) */
+  int dtype;           /* storage of matrices and KV cache: 0 = fp32, 1 = bf16 */
+} spd_model_cfg;
+
+typedef struct {
+  spd_model_cfg target, draft;
+  int max_seq;          /* KV rows per model (image rows + text + gamma_max + 1) */
+  int gamma_max;        /* largest block size that will be used, 0..7 */
+  float temperature;    /* both models' logits are divided by it before softmax */
+  int greedy;           /* 1: argmax rule, probabilities and uniforms unused */
+  int draft_adapter_in; /* 0: text-only draft (Sec. 3); else width of the image features
+                           its linear adapter projects (Sec. 4 "Draft Model Candidates") */
+  void* stream;         /* cudaStream_t, may be NULL (legacy default stream) */
+} spd_cfg;
+
+/* Host or device pointers; per-layer entries are HOST arrays of n_layers pointers. */
+typedef struct {
+  const void* tok_embed;   /* [vocab, d_model] */
+  const void* lm_head;     /* [vocab, d_model]; ignored when tied_embeddings */
+  const float* final_norm; /* [d_model] */
+  const void* adapter;     /* draft only: [d_model, draft_adapter_in], or NULL */
+  const float* const* attn_norm;
+  const void* const* wq;
+  const void* const* wk;
+  const void* const* wv;
+  const void* const* wo;   /* each [d_model, d_model] */
+  const float* const* ffn_norm;
+  const void* const* w_gate;
+  const void* const* w_up; /* each [d_ffn, d_model] */
+  const void* const* w_down; /* [d_model, d_ffn] */
+} spd_weights;
+
+typedef struct {
+  int blocks;          /* target calls made */
+  int accepted;        /* draft tokens accepted in total */
+  int tokens;          /* tokens written to out_ids */
+  float tau;           /* block efficiency: tokens emitted per target call (Sec. 4) */
+  float ms_total, ms_draft, ms_verify; /* device time (CUDA events) */
+} spd_stats;
+
+/* Validates cfg, copies and repacks the weights, allocates KV caches and workspaces,
+ * builds the rotary table.  Shapes must satisfy: d_model <= 4096 and a multiple of 8 per
+ * head pair (d_head even), d_ffn and d_model multiples of 8, gamma_max <= 7, equal vocab
+ * for both models.  *out is NULL on failure. */
+spd_status spd_create(const spd_weights* target_w, const spd_weights* draft_w,
+                      const spd_cfg* cfg, spd_ctx** out);
+void spd_destroy(spd_ctx* ctx);
+const char* spd_last_error(const spd_ctx* ctx);
+
+/* Prefill (Eq. 1): the target reads [image_embeds ; embed(prompt_ids)] at positions
+ * 0..m+n-1 and fills its KV cache; its last row gives the first generated token (argmax,
+ * or a draw with *u0).  The draft reads embed(prompt_ids) only, or, with an adapter,
+ * [draft_image_feats W_a^T ; embed(prompt_ids)].
+ *   image_embeds       fp32 [m, d_target], host or device; NULL iff m == 0
+ *   draft_image_feats  fp32 [m, draft_adapter_in], host or device; NULL without adapter
+ *   prompt_ids         int32 [n], host or device, n >= 1, each < vocab
+ *   u0                 host, one uniform in [0,1); may be NULL when greedy
+ *   first_token        host, out, may be NULL
+ * Resets any earlier sequence. SPD_EOVERFLOW if m + n + gamma_max + 1 > max_seq. */
+spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m,
+                       const float* draft_image_feats, const int32_t* prompt_ids, int n,
+                       const float* u0, int32_t* first_token);
+
+/* Draft step (Sec. 2.1): gamma tokens, one after the other, each drawn from the draft's
+ * softmax(logits / T) with uniforms[j] (or argmax when greedy).
+ *   uniforms     fp32 [gamma], host or device; may be NULL when greedy
+ *   draft_ids    int32 [gamma], out, host or device; may be NULL (kept internally)
+ *   draft_probs  fp32 [gamma, vocab], out, DEVICE; may be NULL (kept internally);
+ *                not written when greedy */
+spd_status spd_draft(spd_ctx* ctx, int gamma, const float* uniforms, int32_t* draft_ids,
+                     float* draft_probs);
+
+/* Verification (Sec. 2.1, Sec. 3): one target call on [pending, x_1..x_gamma] against
+ * the KV cache, then the rejection rule; commits the accepted tokens and the next token
+ * and rolls both KV caches back to the accepted length.
+ *   draft_ids    int32 [gamma], host or device; NULL = the ids of the last spd_draft.
+ *                They must be the tokens the draft was fed, or the draft's cache no
+ *                longer matches the sequence (timing experiments may accept that).
+ *   draft_probs  fp32 [gamma, vocab], DEVICE; NULL = those of the last spd_draft; unused
+ *                when greedy
+ *   uniforms     fp32 [gamma+1], host or device: gamma accept tests, then the one
+ *                replacement / bonus draw; may be NULL when greedy
+ *   n_accepted, next_token  int32, out, host or device (may be NULL)
+ * gamma == 0 is a plain auto-regressive step of the target. */
+spd_status spd_verify(spd_ctx* ctx, int gamma, const int32_t* draft_ids,
+                      const float* draft_probs, const float* uniforms,
+                      int32_t* n_accepted, int32_t* next_token);
+
+/* Block loop (Fig. 1): repeats draft + verify until n_new tokens exist after the prompt;
+ * the token produced by spd_prefill is the first of them.
+ *   uniforms  fp32 [n_new, 2*gamma+1], host or device: per block gamma draft draws, then
+ *             gamma+1 verification uniforms; may be NULL when greedy
+ *   out_ids   int32 [n_new], HOST
+ *   stats     host, may be NULL
+ * gamma == 0 runs the target alone (the auto-regressive baseline). */
+spd_status spd_generate(spd_ctx* ctx, int n_new, int gamma, const float* uniforms,
+                        int32_t* out_ids, spd_stats* stats);
+
+/* ---- test and benchmark support ---- */
+
+/* Logits of the last spd_verify (rows <= gamma+1) / of the last spd_draft (rows <= gamma):
+ * fp32 [rows, vocab] into host or device memory.  Prefill's last row: spd_get_logits with
+ * rows = 1 directly after spd_prefill. */
+spd_status spd_get_logits(spd_ctx* ctx, float* logits, int rows);
+spd_status spd_get_draft_logits(spd_ctx* ctx, float* logits, int rows);
+
+/* Rollback / resynchronisation: declares that the committed text is n_text tokens long
+ * (prompt included, pending token excluded), that prev_token is its last token and
+ * pending_token the token to feed next.  KV rows of positions >= the new length are
+ * treated as stale; rows below it must belong to the same sequence.  O(1). */
+spd_status spd_rollback(spd_ctx* ctx, int n_text, int32_t prev_token, int32_t pending_token);
+spd_status spd_get_state(spd_ctx* ctx, int32_t* n_text, int32_t* pending_token);
+
+/* The rejection rule alone (Sec. 2.1) on given probabilities, B independent sequences:
+ *   p [B, gamma+1, V], q [B, gamma, V] fp32 DEVICE (q may be NULL when greedy)
+ *   ids int32 [B, gamma], u fp32 [B, gamma+1] DEVICE (u may be NULL when greedy)
+ *   n_acc, next int32 [B] DEVICE, out
+ * Integer inverse-CDF sampling (weights truncated to 32 fractional bits, summed as
+ * integers) makes the result independent of summation order. Asynchronous on stream. */
+spd_status spd_reject_sample(const float* p, const float* q, const int32_t* ids,
+                             const float* u, int B, int gamma, int V, int greedy,
+                             int32_t* n_acc, int32_t* next, void* stream);
+
+/* Y[M,N] = X[M,K] W[N,K]^T with the weight-streaming kernel of the verify projections
+ * (Eq. 1's linear maps at M = gamma+1 rows).  x, y fp32 DEVICE, w DEVICE in `dtype`;
+ * 1 <= M <= 8, K a multiple of 8.  Asynchronous on stream. */
+spd_status spd_skinny_gemm(const float* x, const void* w, int dtype, int M, int N, int K,
+                           float* y, void* stream);
+
+/* Bytes that one verify step must move (weights + KV read + KV written) at the current
+ * sequence length, the figure the roofline is computed from. */
+spd_status spd_verify_bytes(spd_ctx* ctx, int gamma, double* bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPD_H_ */

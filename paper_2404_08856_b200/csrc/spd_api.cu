@@ -1,0 +1,761 @@
+// Host side of the C ABI declared in include/spd.h: context, weight repacking, launches.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/spd.h"
+#include "spd_kernel.cuh"
+
+using namespace spd;
+
+// ------------------------------------------------------------------------------ helpers
+
+namespace {
+
+struct ModelHost {
+  spd_model_cfg cfg{};
+  ModelDev md{};            // host copy of the device descriptor
+  ModelDev* md_dev = nullptr;
+  LayerDev* layers_dev = nullptr;
+  int pos_base = 0;         // rows in front of the text (image rows / adapter rows)
+  float* logits = nullptr;  // [8][V]
+  void* adapter = nullptr;  // draft only [d][adapter_in]
+  size_t wbytes = 0;        // bytes of matrices streamed per forward (layers + LM head)
+  size_t esz = 2;
+};
+
+}  // namespace
+
+struct spd_ctx {
+  spd_cfg cfg{};
+  cudaStream_t stream = nullptr;
+  int device = 0, n_sm = 0, smem_optin = 0;
+  ModelHost target, draft;
+  DevState* st = nullptr;
+  unsigned* bars = nullptr;     // pool of grid-barrier counters
+  int bar_next = 0;
+  float* ubuf = nullptr;        // [16] uniforms of direct calls: [0..7] draft, [8..15] verify
+  float* qbuf = nullptr;        // [gamma_max][V] draft distributions
+  float* rows = nullptr;        // prefill rows staging [max_seq][d_max]
+  int* ids_dev = nullptr;       // prompt ids [max_seq]
+  float* upool = nullptr; size_t upool_cap = 0;
+  int* out_dev = nullptr; int out_cap = 0;
+  DevState* st_host = nullptr;  // pinned
+  std::vector<void*> allocs;
+  std::string err;
+  bool prefilled = false;
+  int drafted_gamma = -1;       // gamma of the last spd_draft not yet verified
+  int len_ub = 0;               // upper bound of n_text known to the host
+  int n_prompt = 0, m_image = 0;
+  int last_verify_rows = 0, last_draft_rows = 0;
+  cudaEvent_t ev[4]{};
+};
+
+namespace {
+
+constexpr int BAR_POOL = 64;
+
+spd_status fail(spd_ctx* c, spd_status s, const std::string& msg) {
+  if (c) c->err = msg;
+  return s;
+}
+#define CU(call)                                                                              \
+  do {                                                                                        \
+    cudaError_t e_ = (call);                                                                  \
+    if (e_ != cudaSuccess)                                                                    \
+      return fail(ctx, e_ == cudaErrorMemoryAllocation ? SPD_ENOMEM : SPD_ECUDA,              \
+                  std::string(#call) + ": " + cudaGetErrorString(e_));                        \
+  } while (0)
+
+bool is_device_ptr(const void* p) {
+  cudaPointerAttributes at{};
+  if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return false; }
+  return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeManaged;
+}
+
+template <typename T>
+spd_status dalloc(spd_ctx* ctx, T** p, size_t n) {
+  void* q = nullptr;
+  CU(cudaMalloc(&q, n * sizeof(T) + 256));
+  CU(cudaMemsetAsync(q, 0, n * sizeof(T) + 256, ctx->stream));
+  ctx->allocs.push_back(q);
+  *p = static_cast<T*>(q);
+  return SPD_OK;
+}
+
+// dst row = map(src row) * dst_mul + dst_off; qk_dh > 0 interleaves rotary pairs:
+// source row h*dh + i + w*dh/2 goes to h*dh + 2i + w, so a thread that owns two
+// consecutive rows owns one (i, i + dh/2) pair.
+__global__ void copy_rows_kernel(char* dst, const char* src, int nrows, int row_bytes, int dst_mul, int dst_off,
+                                 int qk_dh) {
+  const int chunks = row_bytes >> 4;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < (size_t)nrows * chunks;
+       i += (size_t)gridDim.x * blockDim.x) {
+    const int r = (int)(i / chunks), c = (int)(i - (size_t)r * chunks);
+    int dr = r;
+    if (qk_dh > 0) {
+      const int h = r / qk_dh, e = r - h * qk_dh, half = qk_dh >> 1;
+      dr = h * qk_dh + ((e < half) ? 2 * e : 2 * (e - half) + 1);
+    }
+    dr = dr * dst_mul + dst_off;
+    reinterpret_cast<uint4*>(dst + (size_t)dr * row_bytes)[c] =
+        reinterpret_cast<const uint4*>(src + (size_t)r * row_bytes)[c];
+  }
+}
+
+spd_status put_rows(spd_ctx* ctx, void* dst, const void* src, void* staging, int nrows, int rowlen, size_t esz,
+                    int dst_mul, int dst_off, int qk_dh) {
+  if (!src) return fail(ctx, SPD_EINVAL, "missing weight pointer");
+  const size_t bytes = (size_t)nrows * rowlen * esz;
+  CU(cudaMemcpyAsync(staging, src, bytes, cudaMemcpyDefault, ctx->stream));
+  copy_rows_kernel<<<1184, 256, 0, ctx->stream>>>(static_cast<char*>(dst), static_cast<const char*>(staging), nrows,
+                                                  (int)(rowlen * esz), dst_mul, dst_off, qk_dh);
+  CU(cudaGetLastError());
+  CU(cudaStreamSynchronize(ctx->stream));  // staging is reused; host sources may be pageable
+  return SPD_OK;
+}
+
+spd_status check_model(spd_ctx* ctx, const spd_model_cfg& c, const char* who) {
+  auto bad = [&](const char* what) { return fail(ctx, SPD_EINVAL, std::string(who) + ": " + what); };
+  if (c.n_layers < 1 || c.d_model < 8 || c.n_heads < 1 || c.d_ffn < 8 || c.vocab < 2) return bad("non-positive shape");
+  if (c.d_model % c.n_heads) return bad("d_model not divisible by n_heads");
+  const int dh = c.d_model / c.n_heads;
+  if (dh != 32 && dh != 64 && dh != 128) return bad("d_head must be 32, 64 or 128");
+  if (c.d_model > KC_MAX) return bad("d_model > 4096 not supported");
+  if (c.d_model % 32 || c.d_ffn % 8) return bad("d_model must be a multiple of 32 and d_ffn of 8");
+  if (c.dtype != 0 && c.dtype != 1) return bad("dtype must be 0 (fp32) or 1 (bf16)");
+  if (!(c.rms_eps >= 0.f) || !(c.rope_theta > 0.f)) return bad("bad rms_eps / rope_theta");
+  return SPD_OK;
+}
+
+spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, const spd_weights* w, int adapter_in,
+                       void* staging) {
+  mh.cfg = c;
+  const size_t esz = c.dtype == 1 ? 2 : 4;
+  mh.esz = esz;
+  const int d = c.d_model, f = c.d_ffn, V = c.vocab, L = c.n_layers, H = c.n_heads, dh = d / H;
+  const int max_seq = ctx->cfg.max_seq;
+  ModelDev& md = mh.md;
+  md.L = L; md.d = d; md.H = H; md.dh = dh; md.f = f; md.V = V; md.max_seq = max_seq;
+  md.nsplit = ctx->n_sm / H > 0 ? ctx->n_sm / H : 1;
+  md.eps = c.rms_eps;
+  md.scale = (float)(1.0 / sqrt((double)dh));
+  spd_status s;
+  char* embed = nullptr;
+  if ((s = dalloc(ctx, &embed, (size_t)V * d * esz))) return s;
+  if ((s = put_rows(ctx, embed, w->tok_embed, staging, V, d, esz, 1, 0, 0))) return s;
+  md.embed = embed;
+  if (c.tied_embeddings) {
+    md.lm_head = embed;
+  } else {
+    char* lm = nullptr;
+    if ((s = dalloc(ctx, &lm, (size_t)V * d * esz))) return s;
+    if ((s = put_rows(ctx, lm, w->lm_head, staging, V, d, esz, 1, 0, 0))) return s;
+    md.lm_head = lm;
+  }
+  float* fn = nullptr;
+  if ((s = dalloc(ctx, &fn, (size_t)d))) return s;
+  if (!w->final_norm) return fail(ctx, SPD_EINVAL, "missing final_norm");
+  CU(cudaMemcpyAsync(fn, w->final_norm, d * sizeof(float), cudaMemcpyDefault, ctx->stream));
+  md.final_norm = fn;
+  if (adapter_in > 0) {
+    if (!w->adapter) return fail(ctx, SPD_EINVAL, "draft_adapter_in > 0 but no adapter weights");
+    char* ad = nullptr;
+    if ((s = dalloc(ctx, &ad, (size_t)d * adapter_in * esz))) return s;
+    if ((s = put_rows(ctx, ad, w->adapter, staging, d, adapter_in, esz, 1, 0, 0))) return s;
+    mh.adapter = ad;
+  }
+  std::vector<LayerDev> layers(L);
+  if (!w->attn_norm || !w->wq || !w->wk || !w->wv || !w->wo || !w->ffn_norm || !w->w_gate || !w->w_up || !w->w_down)
+    return fail(ctx, SPD_EINVAL, "missing per-layer weight array");
+  for (int l = 0; l < L; ++l) {
+    char *wqkv, *wo, *wgu, *wd;
+    float *an, *fnw;
+    if ((s = dalloc(ctx, &wqkv, (size_t)3 * d * d * esz))) return s;
+    if ((s = dalloc(ctx, &wo, (size_t)d * d * esz))) return s;
+    if ((s = dalloc(ctx, &wgu, (size_t)2 * f * d * esz))) return s;
+    if ((s = dalloc(ctx, &wd, (size_t)d * f * esz))) return s;
+    if ((s = dalloc(ctx, &an, (size_t)d))) return s;
+    if ((s = dalloc(ctx, &fnw, (size_t)d))) return s;
+    if ((s = put_rows(ctx, wqkv, w->wq[l], staging, d, d, esz, 1, 0, dh))) return s;
+    if ((s = put_rows(ctx, wqkv + (size_t)d * d * esz, w->wk[l], staging, d, d, esz, 1, 0, dh))) return s;
+    if ((s = put_rows(ctx, wqkv + (size_t)2 * d * d * esz, w->wv[l], staging, d, d, esz, 1, 0, 0))) return s;
+    if ((s = put_rows(ctx, wo, w->wo[l], staging, d, d, esz, 1, 0, 0))) return s;
+    if ((s = put_rows(ctx, wgu, w->w_gate[l], staging, f, d, esz, 2, 0, 0))) return s;
+    if ((s = put_rows(ctx, wgu, w->w_up[l], staging, f, d, esz, 2, 1, 0))) return s;
+    if ((s = put_rows(ctx, wd, w->w_down[l], staging, d, f, esz, 1, 0, 0))) return s;
+    if (!w->attn_norm[l] || !w->ffn_norm[l]) return fail(ctx, SPD_EINVAL, "missing norm gain");
+    CU(cudaMemcpyAsync(an, w->attn_norm[l], d * sizeof(float), cudaMemcpyDefault, ctx->stream));
+    CU(cudaMemcpyAsync(fnw, w->ffn_norm[l], d * sizeof(float), cudaMemcpyDefault, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    layers[l] = LayerDev{wqkv, wo, wgu, wd, an, fnw};
+  }
+  if ((s = dalloc(ctx, &mh.layers_dev, (size_t)L))) return s;
+  CU(cudaMemcpyAsync(mh.layers_dev, layers.data(), L * sizeof(LayerDev), cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  md.layers = mh.layers_dev;
+  // rotary table: cos/sin(pos * theta^(-2i/dh)) in double, stored fp32
+  {
+    const int half = dh / 2;
+    std::vector<float> cs((size_t)max_seq * half), sn((size_t)max_seq * half);
+    for (int i = 0; i < half; ++i) {
+      const double inv = pow((double)c.rope_theta, -2.0 * i / (double)dh);
+      for (int p = 0; p < max_seq; ++p) {
+        cs[(size_t)p * half + i] = (float)cos(p * inv);
+        sn[(size_t)p * half + i] = (float)sin(p * inv);
+      }
+    }
+    float *dc, *ds;
+    if ((s = dalloc(ctx, &dc, cs.size()))) return s;
+    if ((s = dalloc(ctx, &ds, sn.size()))) return s;
+    CU(cudaMemcpyAsync(dc, cs.data(), cs.size() * 4, cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaMemcpyAsync(ds, sn.data(), sn.size() * 4, cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    md.rope_cos = dc; md.rope_sin = ds;
+  }
+  char *kc, *vc;
+  if ((s = dalloc(ctx, &kc, (size_t)L * max_seq * d * esz))) return s;
+  if ((s = dalloc(ctx, &vc, (size_t)L * max_seq * d * esz))) return s;
+  md.kcache = kc; md.vcache = vc;
+  if ((s = dalloc(ctx, &md.x, (size_t)MAX_M * d))) return s;
+  if ((s = dalloc(ctx, &md.qbuf, (size_t)MAX_M * d))) return s;
+  if ((s = dalloc(ctx, &md.attn, (size_t)MAX_M * d))) return s;
+  if ((s = dalloc(ctx, &md.act, (size_t)MAX_M * f))) return s;
+  if ((s = dalloc(ctx, &md.apart, (size_t)H * md.nsplit * MAX_M * dh))) return s;
+  if ((s = dalloc(ctx, &md.aml, (size_t)H * md.nsplit * MAX_M * 2))) return s;
+  if ((s = dalloc(ctx, &md.head_cnt, (size_t)H))) return s;
+  if ((s = dalloc(ctx, &md.stat_part, (size_t)ctx->n_sm * MAX_M * 4))) return s;
+  if ((s = dalloc(ctx, &mh.logits, (size_t)MAX_M * V))) return s;
+  if ((s = dalloc(ctx, &mh.md_dev, (size_t)1))) return s;
+  CU(cudaMemcpyAsync(mh.md_dev, &md, sizeof(ModelDev), cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  mh.wbytes = ((size_t)L * (4ull * d * d + 3ull * d * f) + (size_t)V * d) * esz;
+  return SPD_OK;
+}
+
+// ---- kernel dispatch
+
+using KernelFn = void (*)(const StepArgs);
+
+template <typename WT>
+KernelFn pick_m(int M) {
+  switch (M) {
+    case 1: return forward_kernel<1, WT>;
+    case 2: return forward_kernel<2, WT>;
+    case 3: return forward_kernel<3, WT>;
+    case 4: return forward_kernel<4, WT>;
+    case 5: return forward_kernel<5, WT>;
+    case 6: return forward_kernel<6, WT>;
+    case 7: return forward_kernel<7, WT>;
+    default: return forward_kernel<8, WT>;
+  }
+}
+KernelFn pick_kernel(int M, int dtype) { return dtype == 1 ? pick_m<__nv_bfloat16>(M) : pick_m<float>(M); }
+
+struct LaunchCfg { int nstage; size_t smem; };
+
+spd_status launch_cfg(spd_ctx* ctx, KernelFn fn, int M, int n_sm, int smem_optin, LaunchCfg* lc) {
+  cudaFuncAttributes fa{};
+  CU(cudaFuncGetAttributes(&fa, (const void*)fn));
+  const size_t fixed = CTRL_BYTES + (size_t)M * KC_MAX * sizeof(float);
+  const size_t avail = (size_t)smem_optin - fa.sharedSizeBytes;
+  if (avail < fixed + 2 * STAGE_BYTES) return fail(ctx, SPD_ECUDA, "not enough shared memory per block");
+  int ns = (int)((avail - fixed) / STAGE_BYTES);
+  if (ns > NSTAGE_MAX) ns = NSTAGE_MAX;
+  lc->nstage = ns;
+  lc->smem = fixed + (size_t)ns * STAGE_BYTES;
+  CU(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lc->smem));
+  (void)n_sm;
+  return SPD_OK;
+}
+
+spd_status launch_forward(spd_ctx* ctx, int M, int dtype, StepArgs a, cudaStream_t stream, int n_sm, int smem_optin,
+                          unsigned* bar) {
+  KernelFn fn = pick_kernel(M, dtype);
+  LaunchCfg lc{};
+  spd_status s = launch_cfg(ctx, fn, M, n_sm, smem_optin, &lc);
+  if (s) return s;
+  a.nstage = lc.nstage;
+  a.bar = bar;
+  CU(cudaMemsetAsync(bar, 0, sizeof(unsigned), stream));
+  void* params[] = {&a};
+  CU(cudaLaunchCooperativeKernel((const void*)fn, dim3(n_sm), dim3(ENGINE_THREADS), params, lc.smem, stream));
+  return SPD_OK;
+}
+
+unsigned* next_bar(spd_ctx* ctx) {
+  unsigned* b = ctx->bars + 32 * (ctx->bar_next % BAR_POOL);  // 128 B apart
+  ctx->bar_next++;
+  return b;
+}
+
+spd_status check_dev_err(spd_ctx* ctx, int e) {
+  if (e == DEV_OK) return SPD_OK;
+  if (e == DEV_BAD_TOKEN) return fail(ctx, SPD_EINVAL, "token id out of range seen on the device");
+  return fail(ctx, SPD_ETIMEOUT, "device-side wait ran out (code " + std::to_string(e) + ")");
+}
+
+spd_status sync_state(spd_ctx* ctx) {
+  CU(cudaMemcpyAsync(ctx->st_host, ctx->st, sizeof(DevState), cudaMemcpyDeviceToHost, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  ctx->len_ub = ctx->st_host->n_text;
+  const int e = ctx->st_host->err;
+  if (e != DEV_OK) {
+    cudaMemsetAsync(&ctx->st->err, 0, sizeof(int), ctx->stream);
+    return check_dev_err(ctx, e);
+  }
+  return SPD_OK;
+}
+
+spd_status copy_out(spd_ctx* ctx, void* dst, const void* src_dev, size_t bytes, bool* need_sync) {
+  if (!dst) return SPD_OK;
+  if (is_device_ptr(dst)) {
+    CU(cudaMemcpyAsync(dst, src_dev, bytes, cudaMemcpyDeviceToDevice, ctx->stream));
+  } else {
+    CU(cudaMemcpyAsync(dst, src_dev, bytes, cudaMemcpyDeviceToHost, ctx->stream));
+    *need_sync = true;
+  }
+  return SPD_OK;
+}
+
+StepArgs base_args(spd_ctx* ctx, ModelHost& mh) {
+  StepArgs a{};
+  a.md = mh.md_dev;
+  a.st = ctx->st;
+  a.greedy = ctx->cfg.greedy;
+  a.temperature = ctx->cfg.temperature;
+  a.pos_base = mh.pos_base;
+  a.logits = mh.logits;
+  return a;
+}
+
+// Feed rows [r0, r1) of a prompt through a model in chunks of up to 8 rows.
+spd_status feed_rows(spd_ctx* ctx, ModelHost& mh, const float* rows_dev, const int* ids_dev, int r0, int r1,
+                     int pos0, bool sample_last, int init_n_text, int init_prev) {
+  const int d = mh.cfg.d_model;
+  for (int r = r0; r < r1; r += MAX_M) {
+    const int M = (r1 - r) < MAX_M ? (r1 - r) : MAX_M;
+    StepArgs a = base_args(ctx, mh);
+    a.mode = MODE_ROWS;
+    a.rows = rows_dev ? rows_dev + (size_t)r * d : nullptr;
+    a.row_ids = ids_dev ? ids_dev + r : nullptr;
+    a.rows_pos0 = pos0 + (r - r0);
+    a.want_sample = sample_last && (r + M >= r1);
+    a.init_n_text = init_n_text;
+    a.init_prev = init_prev;
+    a.uniforms = ctx->ubuf + 8;
+    a.out_ids = ctx->out_dev;
+    spd_status s = launch_forward(ctx, M, mh.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx));
+    if (s) return s;
+  }
+  return SPD_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------ C ABI
+
+extern "C" {
+
+const char* spd_last_error(const spd_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+void spd_destroy(spd_ctx* ctx) {
+  if (!ctx) return;
+  cudaStreamSynchronize(ctx->stream);
+  for (void* p : ctx->allocs) cudaFree(p);
+  if (ctx->st_host) cudaFreeHost(ctx->st_host);
+  for (auto& e : ctx->ev)
+    if (e) cudaEventDestroy(e);
+  delete ctx;
+}
+
+spd_status spd_create(const spd_weights* target_w, const spd_weights* draft_w, const spd_cfg* cfg, spd_ctx** out) {
+  if (out) *out = nullptr;
+  if (!target_w || !draft_w || !cfg || !out) return SPD_EINVAL;
+  spd_ctx* ctx = new (std::nothrow) spd_ctx();
+  if (!ctx) return SPD_ENOMEM;
+  auto bail = [&](spd_status s) {
+    fprintf(stderr, "spd_create: %s\n", ctx->err.c_str());
+    spd_destroy(ctx);
+    return s;
+  };
+  ctx->cfg = *cfg;
+  ctx->stream = static_cast<cudaStream_t>(cfg->stream);
+  spd_status s;
+  if ((s = check_model(ctx, cfg->target, "target"))) return bail(s);
+  if ((s = check_model(ctx, cfg->draft, "draft"))) return bail(s);
+  if (cfg->target.vocab != cfg->draft.vocab) return bail(fail(ctx, SPD_EINVAL, "target and draft vocab differ"));
+  if (cfg->gamma_max < 0 || cfg->gamma_max > MAX_M - 1) return bail(fail(ctx, SPD_EINVAL, "gamma_max must be 0..7"));
+  if (cfg->max_seq < 16) return bail(fail(ctx, SPD_EINVAL, "max_seq too small"));
+  if (!cfg->greedy && !(cfg->temperature > 0.f)) return bail(fail(ctx, SPD_EINVAL, "temperature must be > 0"));
+  if (cfg->draft_adapter_in < 0 || cfg->draft_adapter_in % 8) return bail(fail(ctx, SPD_EINVAL, "bad draft_adapter_in"));
+  if (cudaGetDevice(&ctx->device) != cudaSuccess) return bail(fail(ctx, SPD_ECUDA, "no CUDA device"));
+  cudaDeviceProp prop{};
+  if (cudaGetDeviceProperties(&prop, ctx->device) != cudaSuccess) return bail(fail(ctx, SPD_ECUDA, "no device properties"));
+  if (prop.major != 10) return bail(fail(ctx, SPD_ECUDA, "this library is built for sm_100a only"));
+  if (!prop.cooperativeLaunch) return bail(fail(ctx, SPD_ECUDA, "cooperative launch not supported"));
+  ctx->n_sm = prop.multiProcessorCount;
+  ctx->smem_optin = (int)prop.sharedMemPerBlockOptin;
+  // attention scratch must fit the activation region: M*4*(9*dh + Lc) <= M*16384
+  for (const spd_model_cfg* c : {&cfg->target, &cfg->draft}) {
+    const int nsplit = ctx->n_sm / c->n_heads > 0 ? ctx->n_sm / c->n_heads : 1;
+    const int dh = c->d_model / c->n_heads;
+    if ((cfg->max_seq + nsplit - 1) / nsplit + 4 + 9 * dh > KC_MAX)
+      return bail(fail(ctx, SPD_EINVAL, "max_seq too large for the attention scratch"));
+  }
+  if (cfg->temperature <= 0.f) ctx->cfg.temperature = 1.0f;
+  const size_t esz_t = cfg->target.dtype ? 2 : 4, esz_d = cfg->draft.dtype ? 2 : 4;
+  size_t stage_elems = 0;
+  for (const spd_model_cfg* c : {&cfg->target, &cfg->draft}) {
+    const size_t e = c->dtype ? 2 : 4;
+    const size_t big = (size_t)(c->vocab > c->d_ffn ? c->vocab : c->d_ffn) * c->d_model * e;
+    if (big > stage_elems) stage_elems = big;
+  }
+  (void)esz_t; (void)esz_d;
+  char* staging = nullptr;
+  if (cudaMalloc(&staging, stage_elems + 256) != cudaSuccess) return bail(fail(ctx, SPD_ENOMEM, "staging allocation failed"));
+  s = build_model(ctx, ctx->target, cfg->target, target_w, 0, staging);
+  if (!s) s = build_model(ctx, ctx->draft, cfg->draft, draft_w, cfg->draft_adapter_in, staging);
+  cudaFree(staging);
+  if (s) return bail(s);
+  const int V = cfg->target.vocab;
+  const int dmax = cfg->target.d_model > cfg->draft.d_model ? cfg->target.d_model : cfg->draft.d_model;
+  if ((s = dalloc(ctx, &ctx->st, 1))) return bail(s);
+  if ((s = dalloc(ctx, &ctx->bars, (size_t)32 * BAR_POOL))) return bail(s);
+  if ((s = dalloc(ctx, &ctx->ubuf, 16))) return bail(s);
+  if ((s = dalloc(ctx, &ctx->qbuf, (size_t)(cfg->gamma_max > 0 ? cfg->gamma_max : 1) * V))) return bail(s);
+  if ((s = dalloc(ctx, &ctx->rows, (size_t)cfg->max_seq * dmax))) return bail(s);
+  if ((s = dalloc(ctx, &ctx->ids_dev, (size_t)cfg->max_seq))) return bail(s);
+  ctx->out_cap = cfg->max_seq + MAX_M;
+  if ((s = dalloc(ctx, &ctx->out_dev, (size_t)ctx->out_cap))) return bail(s);
+  if (cudaMallocHost(&ctx->st_host, sizeof(DevState)) != cudaSuccess) return bail(fail(ctx, SPD_ENOMEM, "pinned allocation failed"));
+  for (auto& e : ctx->ev)
+    if (cudaEventCreate(&e) != cudaSuccess) return bail(fail(ctx, SPD_ECUDA, "event creation failed"));
+  // every kernel variant that can be launched must fit one CTA per SM
+  for (int M = 1; M <= MAX_M; ++M)
+    for (int dt : {cfg->target.dtype, cfg->draft.dtype}) {
+      KernelFn fn = pick_kernel(M, dt);
+      LaunchCfg lc{};
+      if ((s = launch_cfg(ctx, fn, M, ctx->n_sm, ctx->smem_optin, &lc))) return bail(s);
+      int nb = 0;
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, (const void*)fn, ENGINE_THREADS, lc.smem) != cudaSuccess || nb < 1)
+        return bail(fail(ctx, SPD_ECUDA, "forward kernel does not fit on an SM"));
+    }
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return bail(fail(ctx, SPD_ECUDA, "sync failed"));
+  *out = ctx;
+  return SPD_OK;
+}
+
+spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m, const float* draft_image_feats,
+                       const int32_t* prompt_ids, int n, const float* u0, int32_t* first_token) {
+  if (!ctx) return SPD_EINVAL;
+  if (n < 1 || m < 0 || !prompt_ids || (m > 0 && !image_embeds)) return fail(ctx, SPD_EINVAL, "bad prefill arguments");
+  if (!ctx->cfg.greedy && !u0) return fail(ctx, SPD_EINVAL, "u0 required when sampling");
+  const int ad = ctx->cfg.draft_adapter_in;
+  if (ad > 0 && (m == 0 || !draft_image_feats)) return fail(ctx, SPD_EINVAL, "draft adapter needs image features");
+  if (m + n + ctx->cfg.gamma_max + 1 > ctx->cfg.max_seq) return fail(ctx, SPD_EOVERFLOW, "prompt does not fit max_seq");
+  const int V = ctx->cfg.target.vocab;
+  std::vector<int32_t> ids_h;
+  if (!is_device_ptr(prompt_ids)) {
+    for (int i = 0; i < n; ++i)
+      if (prompt_ids[i] < 0 || prompt_ids[i] >= V) return fail(ctx, SPD_EINVAL, "prompt id out of range");
+  }
+  CU(cudaMemcpyAsync(ctx->ids_dev, prompt_ids, n * sizeof(int32_t), cudaMemcpyDefault, ctx->stream));
+  int32_t last_id = 0;
+  CU(cudaMemcpyAsync(&last_id, ctx->ids_dev + n - 1, sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream));
+  float u = u0 ? *u0 : 0.f;
+  if (u < 0.f || u >= 1.f) return fail(ctx, SPD_EINVAL, "uniform outside [0,1)");
+  CU(cudaMemcpyAsync(ctx->ubuf + 8, &u, sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaMemsetAsync(ctx->st, 0, sizeof(DevState), ctx->stream));
+  CU(cudaMemcpyAsync(&ctx->st->out_cap, &ctx->out_cap, sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  spd_status s;
+  // ---- draft: [adapter(features) ; embed(prompt)] or embed(prompt) alone (Sec. 3)
+  ModelHost& dm = ctx->draft;
+  dm.pos_base = 0;
+  if (ad > 0) {
+    const int dd = dm.cfg.d_model;
+    float* feats = ctx->rows;                 // [m][ad] staged behind the output rows
+    float* outrows = ctx->rows;
+    // stage features at the end of the rows buffer so that outputs can start at 0
+    float* fstage = ctx->rows + (size_t)ctx->cfg.max_seq * (ctx->target.cfg.d_model > dd ? ctx->target.cfg.d_model : dd) - (size_t)m * ad;
+    if ((size_t)m * ad + (size_t)m * dd > (size_t)ctx->cfg.max_seq * (ctx->target.cfg.d_model > dd ? ctx->target.cfg.d_model : dd))
+      return fail(ctx, SPD_EOVERFLOW, "image features do not fit the staging buffer");
+    (void)feats;
+    CU(cudaMemcpyAsync(fstage, draft_image_feats, (size_t)m * ad * sizeof(float), cudaMemcpyDefault, ctx->stream));
+    for (int r = 0; r < m; r += MAX_M) {
+      const int M = (m - r) < MAX_M ? (m - r) : MAX_M;
+      StepArgs a = base_args(ctx, dm);
+      a.mode = MODE_GEMM;
+      a.gx = fstage + (size_t)r * ad; a.gw = dm.adapter; a.gy = outrows + (size_t)r * dd; a.gN = dd; a.gK = ad;
+      if ((s = launch_forward(ctx, M, dm.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx)))) return s;
+    }
+    if ((s = feed_rows(ctx, dm, outrows, nullptr, 0, m, 0, false, 0, 0))) return s;
+    dm.pos_base = m;
+  }
+  if ((s = feed_rows(ctx, dm, nullptr, ctx->ids_dev, 0, n, dm.pos_base, false, 0, 0))) return s;
+  // ---- target: [V_1..V_m ; embed(prompt)] (Eq. 1); last row -> first generated token
+  ModelHost& tm = ctx->target;
+  tm.pos_base = m;
+  if (m > 0) {
+    CU(cudaMemcpyAsync(ctx->rows, image_embeds, (size_t)m * tm.cfg.d_model * sizeof(float), cudaMemcpyDefault, ctx->stream));
+    if ((s = feed_rows(ctx, tm, ctx->rows, nullptr, 0, m, 0, false, 0, 0))) return s;
+  }
+  if ((s = feed_rows(ctx, tm, nullptr, ctx->ids_dev, 0, n, m, true, n, last_id))) return s;
+  ctx->prefilled = true;
+  ctx->drafted_gamma = -1;
+  ctx->n_prompt = n; ctx->m_image = m;
+  ctx->last_verify_rows = 1; ctx->last_draft_rows = 0;
+  // the sampled row was row (chunk rows - 1) of the last chunk: move it to row 0
+  {
+    const int lastM = (n % MAX_M) ? (n % MAX_M) : MAX_M;
+    if (lastM > 1)
+      CU(cudaMemcpyAsync(tm.logits, tm.logits + (size_t)(lastM - 1) * V, V * sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));
+  }
+  if ((s = sync_state(ctx))) return s;
+  if (first_token) *first_token = ctx->st_host->pending;
+  return SPD_OK;
+}
+
+spd_status spd_draft(spd_ctx* ctx, int gamma, const float* uniforms, int32_t* draft_ids, float* draft_probs) {
+  if (!ctx) return SPD_EINVAL;
+  if (!ctx->prefilled) return fail(ctx, SPD_ESTATE, "spd_draft before spd_prefill");
+  if (gamma < 1 || gamma > ctx->cfg.gamma_max) return fail(ctx, SPD_EINVAL, "gamma out of range");
+  if (!ctx->cfg.greedy && !uniforms) return fail(ctx, SPD_EINVAL, "uniforms required when sampling");
+  if (draft_probs && !is_device_ptr(draft_probs)) return fail(ctx, SPD_EINVAL, "draft_probs must be device memory");
+  const int base = ctx->m_image > ctx->draft.pos_base ? ctx->m_image : ctx->draft.pos_base;
+  if (base + ctx->len_ub + gamma + 1 > ctx->cfg.max_seq) {
+    spd_status s = sync_state(ctx);
+    if (s) return s;
+    if (base + ctx->len_ub + gamma + 1 > ctx->cfg.max_seq) return fail(ctx, SPD_EOVERFLOW, "KV cache full");
+  }
+  if (uniforms) CU(cudaMemcpyAsync(ctx->ubuf, uniforms, gamma * sizeof(float), cudaMemcpyDefault, ctx->stream));
+  ModelHost& dm = ctx->draft;
+  for (int j = 0; j < gamma; ++j) {
+    StepArgs a = base_args(ctx, dm);
+    a.mode = MODE_DRAFT;
+    a.gamma = gamma; a.j = j;
+    a.uniforms = ctx->ubuf;
+    a.q_out = ctx->qbuf;
+    a.logits = dm.logits;
+    spd_status s = launch_forward(ctx, 2, dm.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx));
+    if (s) return s;
+    // keep this step's logits row (row 1) for spd_get_draft_logits: rows 2.. of the buffer
+    if (j + 2 < MAX_M)
+      CU(cudaMemcpyAsync(dm.logits + (size_t)(j + 2) * dm.cfg.vocab, dm.logits + (size_t)dm.cfg.vocab,
+                         dm.cfg.vocab * sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));
+  }
+  ctx->drafted_gamma = gamma;
+  ctx->last_draft_rows = gamma < MAX_M - 2 ? gamma : MAX_M - 2;
+  bool need_sync = false;
+  spd_status s;
+  if (draft_probs && !ctx->cfg.greedy)
+    CU(cudaMemcpyAsync(draft_probs, ctx->qbuf, (size_t)gamma * dm.cfg.vocab * sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));
+  if ((s = copy_out(ctx, draft_ids, ctx->st->d_ids, gamma * sizeof(int32_t), &need_sync))) return s;
+  if (need_sync) CU(cudaStreamSynchronize(ctx->stream));
+  return SPD_OK;
+}
+
+spd_status spd_verify(spd_ctx* ctx, int gamma, const int32_t* draft_ids, const float* draft_probs,
+                      const float* uniforms, int32_t* n_accepted, int32_t* next_token) {
+  if (!ctx) return SPD_EINVAL;
+  if (!ctx->prefilled) return fail(ctx, SPD_ESTATE, "spd_verify before spd_prefill");
+  if (gamma < 0 || gamma > ctx->cfg.gamma_max) return fail(ctx, SPD_EINVAL, "gamma out of range");
+  if (gamma > 0 && ctx->drafted_gamma != gamma && (!draft_ids || (!ctx->cfg.greedy && !draft_probs)))
+    return fail(ctx, SPD_ESTATE, "spd_verify needs the ids and probabilities of an spd_draft with the same gamma");
+  if (!ctx->cfg.greedy && !uniforms) return fail(ctx, SPD_EINVAL, "uniforms required when sampling");
+  if (draft_probs && !is_device_ptr(draft_probs)) return fail(ctx, SPD_EINVAL, "draft_probs must be device memory");
+  if (ctx->m_image + ctx->len_ub + gamma + 1 > ctx->cfg.max_seq) {
+    spd_status s = sync_state(ctx);
+    if (s) return s;
+    if (ctx->m_image + ctx->len_ub + gamma + 1 > ctx->cfg.max_seq) return fail(ctx, SPD_EOVERFLOW, "KV cache full");
+  }
+  const int V = ctx->cfg.target.vocab;
+  if (draft_ids && gamma > 0) {
+    if (!is_device_ptr(draft_ids))
+      for (int j = 0; j < gamma; ++j)
+        if (draft_ids[j] < 0 || draft_ids[j] >= V) return fail(ctx, SPD_EINVAL, "draft id out of range");
+    CU(cudaMemcpyAsync(ctx->st->d_ids, draft_ids, gamma * sizeof(int32_t), cudaMemcpyDefault, ctx->stream));
+  }
+  if (uniforms) CU(cudaMemcpyAsync(ctx->ubuf + 8, uniforms, (gamma + 1) * sizeof(float), cudaMemcpyDefault, ctx->stream));
+  ModelHost& tm = ctx->target;
+  StepArgs a = base_args(ctx, tm);
+  a.mode = MODE_VERIFY;
+  a.gamma = gamma;
+  a.uniforms = ctx->ubuf + 8;
+  a.q_in = draft_probs ? draft_probs : ctx->qbuf;
+  a.out_ids = nullptr;
+  spd_status s = launch_forward(ctx, gamma + 1, tm.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx));
+  if (s) return s;
+  ctx->drafted_gamma = -1;
+  ctx->len_ub += gamma + 1;
+  ctx->last_verify_rows = gamma + 1;
+  bool need_sync = false;
+  if ((s = copy_out(ctx, n_accepted, &ctx->st->n_acc, sizeof(int32_t), &need_sync))) return s;
+  if ((s = copy_out(ctx, next_token, &ctx->st->next, sizeof(int32_t), &need_sync))) return s;
+  if (need_sync) return sync_state(ctx);
+  return SPD_OK;
+}
+
+spd_status spd_generate(spd_ctx* ctx, int n_new, int gamma, const float* uniforms, int32_t* out_ids,
+                        spd_stats* stats) {
+  if (!ctx) return SPD_EINVAL;
+  if (!ctx->prefilled) return fail(ctx, SPD_ESTATE, "spd_generate before spd_prefill");
+  if (n_new < 1 || !out_ids) return fail(ctx, SPD_EINVAL, "bad n_new / out_ids");
+  if (gamma < 0 || gamma > ctx->cfg.gamma_max) return fail(ctx, SPD_EINVAL, "gamma out of range");
+  if (!ctx->cfg.greedy && !uniforms) return fail(ctx, SPD_EINVAL, "uniforms required when sampling");
+  if (n_new > ctx->out_cap) return fail(ctx, SPD_EOVERFLOW, "n_new exceeds the output buffer");
+  spd_status s = sync_state(ctx);
+  if (s) return s;
+  if (ctx->st_host->n_emitted != 1 || ctx->st_host->block != 0)
+    return fail(ctx, SPD_ESTATE, "spd_generate must follow spd_prefill directly");
+  if (ctx->m_image + ctx->len_ub + n_new + gamma + 1 > ctx->cfg.max_seq)
+    return fail(ctx, SPD_EOVERFLOW, "n_new does not fit max_seq");
+  const int us = 2 * gamma + 1;
+  if (uniforms) {
+    const size_t need = (size_t)n_new * us;
+    if (need > ctx->upool_cap) {
+      if ((s = dalloc(ctx, &ctx->upool, need))) return s;
+      ctx->upool_cap = need;
+    }
+    CU(cudaMemcpyAsync(ctx->upool, uniforms, need * sizeof(float), cudaMemcpyDefault, ctx->stream));
+  }
+  ModelHost &tm = ctx->target, &dm = ctx->draft;
+  float ms_d = 0.f, ms_v = 0.f;
+  CU(cudaEventRecord(ctx->ev[0], ctx->stream));
+  int blocks = 0;
+  while (ctx->st_host->n_emitted < n_new) {
+    CU(cudaEventRecord(ctx->ev[1], ctx->stream));
+    for (int j = 0; j < gamma; ++j) {
+      StepArgs a = base_args(ctx, dm);
+      a.mode = MODE_DRAFT; a.gamma = gamma; a.j = j;
+      a.uniforms = uniforms ? ctx->upool : nullptr; a.u_stride = us; a.u_by_block = 1;
+      a.q_out = ctx->qbuf; a.logits = dm.logits;
+      if ((s = launch_forward(ctx, 2, dm.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx)))) return s;
+    }
+    CU(cudaEventRecord(ctx->ev[2], ctx->stream));
+    StepArgs a = base_args(ctx, tm);
+    a.mode = MODE_VERIFY; a.gamma = gamma;
+    a.uniforms = uniforms ? ctx->upool : nullptr; a.u_stride = us; a.u_by_block = 1;
+    a.q_in = ctx->qbuf; a.out_ids = ctx->out_dev;
+    if ((s = launch_forward(ctx, gamma + 1, tm.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx)))) return s;
+    CU(cudaEventRecord(ctx->ev[3], ctx->stream));
+    if ((s = sync_state(ctx))) return s;
+    float t1 = 0.f, t2 = 0.f;
+    cudaEventElapsedTime(&t1, ctx->ev[1], ctx->ev[2]);
+    cudaEventElapsedTime(&t2, ctx->ev[2], ctx->ev[3]);
+    ms_d += t1; ms_v += t2;
+    ++blocks;
+    if (blocks > n_new + 1) return fail(ctx, SPD_ECUDA, "block loop made no progress");
+  }
+  CU(cudaEventRecord(ctx->ev[3], ctx->stream));
+  CU(cudaMemcpyAsync(out_ids, ctx->out_dev, n_new * sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  ctx->drafted_gamma = -1;
+  ctx->last_verify_rows = gamma + 1;
+  if (stats) {
+    float tot = 0.f;
+    cudaEventElapsedTime(&tot, ctx->ev[0], ctx->ev[3]);
+    stats->blocks = blocks;
+    stats->tokens = n_new;
+    const int emitted = ctx->st_host->n_emitted - 1;
+    stats->accepted = emitted - blocks;
+    stats->tau = blocks ? (float)emitted / blocks : 0.f;
+    stats->ms_total = tot; stats->ms_draft = ms_d; stats->ms_verify = ms_v;
+  }
+  return SPD_OK;
+}
+
+spd_status spd_get_logits(spd_ctx* ctx, float* logits, int rows) {
+  if (!ctx || !logits) return SPD_EINVAL;
+  if (rows < 1 || rows > ctx->last_verify_rows) return fail(ctx, SPD_EINVAL, "rows exceed the last verify call");
+  CU(cudaMemcpyAsync(logits, ctx->target.logits, (size_t)rows * ctx->cfg.target.vocab * sizeof(float), cudaMemcpyDefault, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  return SPD_OK;
+}
+
+spd_status spd_get_draft_logits(spd_ctx* ctx, float* logits, int rows) {
+  if (!ctx || !logits) return SPD_EINVAL;
+  if (rows < 1 || rows > ctx->last_draft_rows) return fail(ctx, SPD_EINVAL, "rows exceed the last draft call");
+  const int V = ctx->cfg.draft.vocab;
+  CU(cudaMemcpyAsync(logits, ctx->draft.logits + (size_t)2 * V, (size_t)rows * V * sizeof(float), cudaMemcpyDefault, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  return SPD_OK;
+}
+
+spd_status spd_rollback(spd_ctx* ctx, int n_text, int32_t prev_token, int32_t pending_token) {
+  if (!ctx) return SPD_EINVAL;
+  if (!ctx->prefilled) return fail(ctx, SPD_ESTATE, "spd_rollback before spd_prefill");
+  const int V = ctx->cfg.target.vocab;
+  if (n_text < 1 || ctx->m_image + n_text + 1 > ctx->cfg.max_seq || prev_token < 0 || prev_token >= V ||
+      pending_token < 0 || pending_token >= V)
+    return fail(ctx, SPD_EINVAL, "bad rollback arguments");
+  int v[3] = {n_text, pending_token, prev_token};
+  CU(cudaMemcpyAsync(&ctx->st->n_text, v, sizeof(v), cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  ctx->len_ub = n_text;
+  ctx->drafted_gamma = -1;
+  return SPD_OK;
+}
+
+spd_status spd_get_state(spd_ctx* ctx, int32_t* n_text, int32_t* pending_token) {
+  if (!ctx) return SPD_EINVAL;
+  if (!ctx->prefilled) return fail(ctx, SPD_ESTATE, "no sequence yet");
+  spd_status s = sync_state(ctx);
+  if (s) return s;
+  if (n_text) *n_text = ctx->st_host->n_text;
+  if (pending_token) *pending_token = ctx->st_host->pending;
+  return SPD_OK;
+}
+
+spd_status spd_reject_sample(const float* p, const float* q, const int32_t* ids, const float* u, int B, int gamma,
+                             int V, int greedy, int32_t* n_acc, int32_t* next, void* stream) {
+  if (!p || !n_acc || !next || B < 1 || gamma < 0 || V < 1) return SPD_EINVAL;
+  if (gamma > 0 && !ids) return SPD_EINVAL;
+  if (!greedy && (!u || (gamma > 0 && !q))) return SPD_EINVAL;
+  reject_sample_kernel<<<B, SAMPLE_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(p, q, ids, u, gamma, V, greedy,
+                                                                                    n_acc, next);
+  return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ECUDA;
+}
+
+spd_status spd_skinny_gemm(const float* x, const void* w, int dtype, int M, int N, int K, float* y, void* stream) {
+  if (!x || !w || !y || M < 1 || M > MAX_M || N < 1 || K < 8 || K % 8 || (dtype != 0 && dtype != 1)) return SPD_EINVAL;
+  static unsigned* bar = nullptr;
+  static DevState* st = nullptr;
+  static int n_sm = 0, smem_optin = 0;
+  spd_ctx* ctx = nullptr;
+  if (!bar) {
+    int dev = 0;
+    cudaDeviceProp prop{};
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return SPD_ECUDA;
+    if (prop.major != 10) return SPD_ECUDA;
+    n_sm = prop.multiProcessorCount;
+    smem_optin = (int)prop.sharedMemPerBlockOptin;
+    if (cudaMalloc(&bar, 256) != cudaSuccess || cudaMalloc(&st, sizeof(DevState)) != cudaSuccess) return SPD_ENOMEM;
+    cudaMemset(st, 0, sizeof(DevState));
+  }
+  StepArgs a{};
+  a.mode = MODE_GEMM;
+  a.st = st;
+  a.gx = x; a.gw = w; a.gy = y; a.gN = N; a.gK = K;
+  return launch_forward(ctx, M, dtype, a, static_cast<cudaStream_t>(stream), n_sm, smem_optin, bar);
+}
+
+spd_status spd_verify_bytes(spd_ctx* ctx, int gamma, double* bytes) {
+  if (!ctx || !bytes) return SPD_EINVAL;
+  if (!ctx->prefilled) return fail(ctx, SPD_ESTATE, "no sequence yet");
+  spd_status s = sync_state(ctx);
+  if (s) return s;
+  const ModelHost& tm = ctx->target;
+  const double C = ctx->m_image + ctx->st_host->n_text;
+  const double kv_row = 2.0 * tm.cfg.n_layers * tm.cfg.d_model * tm.esz;
+  *bytes = (double)tm.wbytes + kv_row * (C + gamma + 1) + kv_row * (gamma + 1);
+  return SPD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,726 @@
+// The forward engine: ONE persistent cooperative kernel runs a whole M-row forward pass
+// (M = gamma+1 rows for the verify step, 2 rows for a draft step, up to 8 rows for a
+// chunk of prompt rows) through every layer, the LM head and the sampling rule.
+//
+// Why one kernel: the step is bound by streaming the weights from HBM once (the paper's
+// "memory bandwidth bottleneck", Sec. 1); with a launch per operation the pipeline drains
+// at every boundary.  Here a producer warp per CTA streams weight tiles through a ring of
+// shared-memory stages with bulk async copies and runs AHEAD of the compute warps across
+// layer and phase boundaries (weights never depend on activations), so HBM stays busy
+// while the compute warps sit in a grid barrier, build their activation tile or run
+// attention.
+//
+// Per layer (Eq. 1's decoder, LLaMA architecture): RMSNorm -> QKV projection (+ RoPE and
+// KV-cache append in the epilogue) | attention of the M new rows over the cache, causal
+// within the block | output projection + residual | RMSNorm -> gate/up projection +
+// SwiGLU | down projection + residual.  "|" is a grid barrier.
+//
+// Skinny GEMM Y[M,N] = X[M,K] W[N,K]^T: a tile is 32 weight rows; each of 8 compute warps
+// owns 4 rows, its lanes split K in 16-byte pieces (one ring stage = 32 rows x 512 B).
+// X lives in shared memory as fp32, laid out so that a lane's 16-byte reads are
+// conflict-free; products accumulate in fp32 with packed two-wide FMAs; the 4*M sums per
+// warp are reduced across lanes by a halving butterfly.
+#pragma once
+#include "spd_device.cuh"
+#include "spd_sample.cuh"
+
+namespace spd {
+
+constexpr int MAX_M = 8;
+constexpr int KC_MAX = 4096;          // activation columns resident in shared memory
+constexpr int STAGE_BYTES = 16384;    // 32 rows x 512 B
+constexpr int NSTAGE_MAX = 12;
+constexpr int CONSUMER_THREADS = 256;
+constexpr int ENGINE_THREADS = CONSUMER_THREADS + 32;
+constexpr int CTRL_BYTES = 1024;
+
+enum : int { MODE_VERIFY = 0, MODE_DRAFT = 1, MODE_ROWS = 2, MODE_GEMM = 3 };
+enum : int { PRO_PLAIN = 0, PRO_NORM = 1 };
+enum : int { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_QKV = 3 };
+
+struct LayerDev {
+  const void *wqkv, *wo, *wgu, *wd;   // repacked: see spd_api.cu
+  const float *attn_norm, *ffn_norm;
+};
+
+struct ModelDev {
+  int L, d, H, dh, f, V, max_seq, nsplit;
+  float eps, scale;
+  const void* embed;
+  const void* lm_head;
+  const float* final_norm;
+  const float *rope_cos, *rope_sin;   // [max_seq][dh/2]
+  void *kcache, *vcache;              // [L][max_seq][d]
+  float *x, *qbuf, *attn, *act;       // [8][d], [8][d], [8][d], [8][f]
+  float *apart, *aml;                 // attention partials [H][nsplit][8][dh], [H][nsplit][8][2]
+  unsigned* head_cnt;                 // [H]
+  float* stat_part;                   // [grid][8][4]: row max, row sum, argmax value, argmax index
+  const LayerDev* layers;
+};
+
+struct DevState {
+  int n_text;     // committed text tokens, pending excluded = text position of pending
+  int pending, prev;
+  int block;      // blocks committed since prefill
+  int n_emitted;  // tokens written to out_ids
+  int err;
+  int n_acc, next;
+  int d_ids[MAX_M];
+  int out_cap;
+  int pad[3];
+};
+
+struct StepArgs {
+  const ModelDev* md;
+  DevState* st;
+  unsigned* bar;          // grid-barrier counter, zero at launch
+  int mode, gamma, j, pos_base, nstage, greedy;
+  float temperature;
+  // MODE_ROWS
+  const float* rows;      // fp32 [M, d] input rows (already embeddings), or NULL: ids
+  const int* row_ids;     // MODE_ROWS with rows == NULL: token ids [M]
+  int rows_pos0, want_sample, init_n_text, init_prev;
+  // uniforms
+  const float* uniforms;
+  int u_stride, u_by_block;
+  // draft distributions [gamma][V]
+  const float* q_in;
+  float* q_out;
+  float* logits;          // [M][V] LM-head output
+  int* out_ids;
+  // MODE_GEMM
+  const float* gx; const void* gw; float* gy; int gN, gK;
+};
+
+struct Ctrl {
+  uint64_t full[NSTAGE_MAX];
+  uint64_t empty[NSTAGE_MAX];
+  SampleScratch sc;
+  float red[8][MAX_M];
+  float rowmax[MAX_M], rowsum[MAX_M];
+  int flag;
+};
+static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
+
+struct Gemm {
+  const void* W;
+  int N, K, pro, epi, layer;
+};
+
+__device__ __forceinline__ Gemm get_gemm(const ModelDev& md, int idx) {
+  Gemm g;
+  const int l = idx >> 2, which = idx & 3;
+  g.layer = l;
+  if (l >= md.L) { g.W = md.lm_head; g.N = md.V; g.K = md.d; g.pro = PRO_NORM; g.epi = EPI_STORE; return g; }
+  const LayerDev& ly = md.layers[l];
+  switch (which) {
+    case 0: g.W = ly.wqkv; g.N = 3 * md.d; g.K = md.d; g.pro = PRO_NORM; g.epi = EPI_QKV; break;
+    case 1: g.W = ly.wo; g.N = md.d; g.K = md.d; g.pro = PRO_PLAIN; g.epi = EPI_RESID; break;
+    case 2: g.W = ly.wgu; g.N = 2 * md.f; g.K = md.d; g.pro = PRO_NORM; g.epi = EPI_SWIGLU; break;
+    default: g.W = ly.wd; g.N = md.d; g.K = md.f; g.pro = PRO_PLAIN; g.epi = EPI_RESID; break;
+  }
+  return g;
+}
+
+template <typename WT> struct WTraits;
+template <> struct WTraits<__nv_bfloat16> { static constexpr int EPL = 8; };
+template <> struct WTraits<float> { static constexpr int EPL = 4; };
+
+__device__ __forceinline__ void chunking(int K, int kstep, int& nchunk, int& kcl) {
+  nchunk = (K + KC_MAX - 1) / KC_MAX;
+  kcl = (K + nchunk - 1) / nchunk;
+  kcl = (kcl + kstep - 1) / kstep * kstep;
+}
+
+struct Ring {
+  int stage;
+  unsigned phase;
+  int nstage;
+  __device__ __forceinline__ void advance() {
+    if (++stage == nstage) { stage = 0; phase ^= 1u; }
+  }
+};
+
+// ------------------------------------------------------------------------------ producer
+
+template <typename WT>
+__device__ void produce_gemm(const Gemm& g, int cta, int G, int& off, Ring& ring, Ctrl* ctl, char* stages,
+                             uint64_t pol, volatile int* err) {
+  constexpr int EPL = WTraits<WT>::EPL, KSTEP = 32 * EPL;
+  const int lane = threadIdx.x & 31;
+  const int ntiles = (g.N + 31) >> 5;
+  int nchunk, kcl;
+  chunking(g.K, KSTEP, nchunk, kcl);
+  for (int t = (cta - off + G) % G; t < ntiles; t += G) {
+    const int row = t * 32 + lane;
+    const bool rv = row < g.N;
+    const unsigned nrows = min(32, g.N - t * 32);
+    const char* wrow = static_cast<const char*>(g.W) + (size_t)(rv ? row : 0) * g.K * sizeof(WT);
+    for (int c = 0; c < nchunk; ++c) {
+      const int k0 = c * kcl, klen = min(kcl, g.K - k0);
+      for (int s = 0; s * KSTEP < klen; ++s) {
+        const unsigned bytes = min(KSTEP, klen - s * KSTEP) * sizeof(WT);
+        mbar_wait(&ctl->empty[ring.stage], ring.phase ^ 1u, err, DEV_TIMEOUT_EMPTY);
+        if (*err != DEV_OK) return;
+        if (lane == 0) mbar_arrive_expect_tx(&ctl->full[ring.stage], bytes * nrows);
+        __syncwarp();
+        if (rv)
+          bulk_g2s(stages + (size_t)ring.stage * STAGE_BYTES + lane * 512,
+                   wrow + (size_t)(k0 + s * KSTEP) * sizeof(WT), bytes, &ctl->full[ring.stage], pol);
+        ring.advance();
+      }
+    }
+  }
+  off = (off + ntiles) % G;
+}
+
+// ------------------------------------------------------------------------------ X tile
+
+// destination float4 index of natural float4 index k4 inside the activation tile
+template <int EPL>
+__device__ __forceinline__ int perm4(int k4) {
+  if constexpr (EPL == 8) return (k4 & ~63) | ((k4 & 1) << 5) | ((k4 & 63) >> 1);
+  else return k4;
+}
+
+__device__ __forceinline__ float4 cvt4(const __nv_bfloat16* p) {
+  const uint2 r = *reinterpret_cast<const uint2*>(p);
+  return make_float4(bf16lo(r.x), bf16hi(r.x), bf16lo(r.y), bf16hi(r.y));
+}
+__device__ __forceinline__ float4 cvt4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+
+// Load rows [M][klen] (fetch(m, k) -> 4 consecutive values at column k) into X with the
+// lane-friendly permutation, zero padding up to kpad.  With NORM: RMSNorm in place.
+template <int M, int EPL, bool NORM, class Fetch>
+__device__ void load_x(float* X, int kpad, int klen, Fetch fetch, const float* norm_w, float eps, int Ktotal,
+                       Ctrl* ctl, float* copy_out, int copy_ld) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int kp4 = kpad >> 2, kl4 = klen >> 2;
+  float4* X4 = reinterpret_cast<float4*>(X);
+  float ss[M];
+#pragma unroll
+  for (int m = 0; m < M; ++m) {
+    ss[m] = 0.f;
+    for (int k4 = tid; k4 < kp4; k4 += CONSUMER_THREADS) {
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (k4 < kl4) {
+        v = fetch(m, k4 << 2);
+        if (copy_out) __stcg(reinterpret_cast<float4*>(copy_out + (size_t)m * copy_ld + (k4 << 2)), v);
+      }
+      if (NORM) ss[m] += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+      X4[m * kp4 + perm4<EPL>(k4)] = v;
+    }
+  }
+  if (NORM) {
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      float s = ss[m];
+#pragma unroll
+      for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      if (lane == 0) ctl->red[warp][m] = s;
+    }
+    named_sync(1, CONSUMER_THREADS);
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) s += ctl->red[w][m];
+      const float inv = 1.0f / sqrtf(s / (float)Ktotal + eps);
+      for (int k4 = tid; k4 < kl4; k4 += CONSUMER_THREADS) {
+        const float4 g = *reinterpret_cast<const float4*>(norm_w + (k4 << 2));
+        float4& v = X4[m * kp4 + perm4<EPL>(k4)];
+        v.x = (v.x * inv) * g.x; v.y = (v.y * inv) * g.y; v.z = (v.z * inv) * g.z; v.w = (v.w * inv) * g.w;
+      }
+    }
+  }
+  named_sync(1, CONSUMER_THREADS);
+}
+
+// ------------------------------------------------------------------------------ reduction
+
+// Sum each of CNT values over the 32 lanes.  While the count is a multiple of 4 the
+// lanes split the values (half kept, half sent); afterwards every value is all-reduced.
+// On return lane holds `final_cnt` sums starting at value index `base`.
+template <int CNT, int BIT>
+__device__ __forceinline__ void reduce_rec(float* v, int& base, int lane) {
+  if constexpr (BIT > 0) {
+    if constexpr (CNT % 4 == 0) {
+      constexpr int HALF = CNT / 2;
+      const bool up = (lane & BIT) != 0;
+#pragma unroll
+      for (int i = 0; i < HALF; ++i) {
+        const float keep = up ? v[i + HALF] : v[i];
+        const float send = up ? v[i] : v[i + HALF];
+        v[i] = keep + __shfl_xor_sync(0xffffffffu, send, BIT);
+      }
+      if (up) base += HALF;
+      reduce_rec<HALF, BIT / 2>(v, base, lane);
+    } else {
+#pragma unroll
+      for (int i = 0; i < CNT; ++i) v[i] += __shfl_xor_sync(0xffffffffu, v[i], BIT);
+      reduce_rec<CNT, BIT / 2>(v, base, lane);
+    }
+  }
+}
+constexpr int final_cnt(int cnt, int bit) { return bit == 0 ? cnt : (cnt % 4 == 0 ? final_cnt(cnt / 2, bit / 2) : cnt); }
+constexpr int dup_mask(int cnt, int bit) {
+  return bit == 0 ? 0 : (cnt % 4 == 0 ? dup_mask(cnt / 2, bit / 2) : (bit | dup_mask(cnt, bit / 2)));
+}
+
+// ------------------------------------------------------------------------------ epilogues
+
+struct EpiArgs {
+  float* out;     // STORE: [M][ldo]; RESID: x [M][ldo]; SWIGLU: act [M][ldo]
+  int ldo;
+  // QKV
+  float* qbuf; void* kc; void* vc;  // cache bases already offset to the layer
+  const float *cs, *sn;
+  int pos0, d, dh;
+};
+
+__device__ __forceinline__ void cache_store(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+__device__ __forceinline__ void cache_store(float* p, float v) { *p = v; }
+
+template <typename WT>
+__device__ __forceinline__ void epilogue_pair(int epi, const EpiArgs& e, int m, int n, int N, float a, float b) {
+  if (n >= N) return;
+  if (epi == EPI_STORE) {
+    stcg(e.out + (size_t)m * e.ldo + n, a);
+    if (n + 1 < N) stcg(e.out + (size_t)m * e.ldo + n + 1, b);
+  } else if (epi == EPI_RESID) {
+    float* p = e.out + (size_t)m * e.ldo + n;
+    stcg(p, ldcg(p) + a);
+    if (n + 1 < N) stcg(p + 1, ldcg(p + 1) + b);
+  } else if (epi == EPI_SWIGLU) {
+    const float s = a / (1.0f + expf(-a));
+    stcg(e.out + (size_t)m * e.ldo + (n >> 1), s * b);
+  } else {  // EPI_QKV: rows are [q | k | v]; q and k rows are stored pair-interleaved
+    const int region = n / e.d, c = n - region * e.d;
+    const int pos = e.pos0 + m;
+    if (region == 2) {
+      WT* vp = static_cast<WT*>(e.vc) + (size_t)pos * e.d + c;
+      cache_store(vp, a);
+      cache_store(vp + 1, b);
+    } else {
+      const int h = c / e.dh, i = (c - h * e.dh) >> 1, half = e.dh >> 1;
+      const float cs = e.cs[pos * half + i], sn = e.sn[pos * half + i];
+      const float ra = a * cs - b * sn, rb = b * cs + a * sn;
+      const int c0 = h * e.dh + i;
+      if (region == 0) {
+        stcg(e.qbuf + (size_t)m * e.d + c0, ra);
+        stcg(e.qbuf + (size_t)m * e.d + c0 + half, rb);
+      } else {
+        WT* kp = static_cast<WT*>(e.kc) + (size_t)pos * e.d + c0;
+        cache_store(kp, ra);
+        cache_store(kp + half, rb);
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------ consumer
+
+template <int M, typename WT>
+__device__ __forceinline__ void compute_step(const char* stage, const float* X, int kp4, int s, int len, int warp,
+                                             int lane, float2 (&acc)[4][M]) {
+  constexpr int EPL = WTraits<WT>::EPL;
+  const bool active = lane * EPL < len;
+  const uint4* wp = reinterpret_cast<const uint4*>(stage + warp * 2048 + lane * 16);
+  if constexpr (EPL == 8) {
+    float2 w[4][4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      uint4 q = wp[r * 32];
+      if (!active) q = make_uint4(0, 0, 0, 0);
+      w[r][0] = make_float2(bf16lo(q.x), bf16hi(q.x));
+      w[r][1] = make_float2(bf16lo(q.y), bf16hi(q.y));
+      w[r][2] = make_float2(bf16lo(q.z), bf16hi(q.z));
+      w[r][3] = make_float2(bf16lo(q.w), bf16hi(q.w));
+    }
+    const float4* xp = reinterpret_cast<const float4*>(X) + s * 64 + lane;
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      const float4 xa = xp[m * kp4], xb = xp[m * kp4 + 32];
+      const float2 x0 = make_float2(xa.x, xa.y), x1 = make_float2(xa.z, xa.w);
+      const float2 x2 = make_float2(xb.x, xb.y), x3 = make_float2(xb.z, xb.w);
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        float2 a = acc[r][m];
+        a = __ffma2_rn(w[r][0], x0, a);
+        a = __ffma2_rn(w[r][1], x1, a);
+        a = __ffma2_rn(w[r][2], x2, a);
+        a = __ffma2_rn(w[r][3], x3, a);
+        acc[r][m] = a;
+      }
+    }
+  } else {
+    float2 w[4][2];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      uint4 q = wp[r * 32];
+      if (!active) q = make_uint4(0, 0, 0, 0);
+      w[r][0] = make_float2(__uint_as_float(q.x), __uint_as_float(q.y));
+      w[r][1] = make_float2(__uint_as_float(q.z), __uint_as_float(q.w));
+    }
+    const float4* xp = reinterpret_cast<const float4*>(X) + s * 32 + lane;
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      const float4 xa = xp[m * kp4];
+      const float2 x0 = make_float2(xa.x, xa.y), x1 = make_float2(xa.z, xa.w);
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        float2 a = acc[r][m];
+        a = __ffma2_rn(w[r][0], x0, a);
+        a = __ffma2_rn(w[r][1], x1, a);
+        acc[r][m] = a;
+      }
+    }
+  }
+}
+
+// xsrc(m, k) fetches 4 activation values; used for every chunk.
+template <int M, typename WT, class Fetch>
+__device__ void consume_gemm(const Gemm& g, const EpiArgs& e, Fetch fetch, const float* norm_w, float eps,
+                             float* copy_out, int cta, int G, int& off, Ring& ring, Ctrl* ctl, float* X,
+                             const char* stages, volatile int* err) {
+  constexpr int EPL = WTraits<WT>::EPL, KSTEP = 32 * EPL;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int ntiles = (g.N + 31) >> 5;
+  int nchunk, kcl;
+  chunking(g.K, KSTEP, nchunk, kcl);
+  const int kp4 = kcl >> 2;
+  const int t0 = (cta - off + G) % G;
+  off = (off + ntiles) % G;
+  if (t0 >= ntiles) return;
+  if (nchunk == 1) {
+    if (g.pro == PRO_NORM) load_x<M, EPL, true>(X, kcl, g.K, fetch, norm_w, eps, g.K, ctl, copy_out, g.K);
+    else load_x<M, EPL, false>(X, kcl, g.K, fetch, nullptr, 0.f, g.K, ctl, copy_out, g.K);
+  }
+  for (int t = t0; t < ntiles; t += G) {
+    float2 acc[4][M];
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int m = 0; m < M; ++m) acc[r][m] = make_float2(0.f, 0.f);
+    for (int c = 0; c < nchunk; ++c) {
+      const int k0 = c * kcl, klen = min(kcl, g.K - k0);
+      if (nchunk > 1) {
+        named_sync(1, CONSUMER_THREADS);  // everyone is done with the previous chunk
+        load_x<M, EPL, false>(X, kcl, klen, [&](int m, int k) { return fetch(m, k0 + k); }, nullptr, 0.f, g.K, ctl,
+                              nullptr, 0);
+      }
+      for (int s = 0; s * KSTEP < klen; ++s) {
+        mbar_wait(&ctl->full[ring.stage], ring.phase, err, DEV_TIMEOUT_FULL);
+        compute_step<M, WT>(stages + (size_t)ring.stage * STAGE_BYTES, X, kp4, s, min(KSTEP, klen - s * KSTEP), warp,
+                            lane, acc);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ctl->empty[ring.stage]);
+        ring.advance();
+      }
+    }
+    // 4*M sums per warp, value index m*4 + r
+    float v[4 * M];
+#pragma unroll
+    for (int m = 0; m < M; ++m)
+#pragma unroll
+      for (int r = 0; r < 4; ++r) v[m * 4 + r] = acc[r][m].x + acc[r][m].y;
+    int base = 0;
+    reduce_rec<4 * M, 16>(v, base, lane);
+    constexpr int FC = final_cnt(4 * M, 16), DUP = dup_mask(4 * M, 16);
+    if ((lane & DUP) == 0) {
+#pragma unroll
+      for (int i = 0; i < FC; i += 2) {
+        const int vi = base + i, m = vi >> 2, r = vi & 3;
+        epilogue_pair<WT>(g.epi, e, m, t * 32 + warp * 4 + r, g.N, v[i], v[i + 1]);
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------ grid barrier
+
+__device__ __forceinline__ void grid_barrier(unsigned* counter, unsigned& target, unsigned G, volatile int* err) {
+  named_sync(1, CONSUMER_THREADS);
+  if (threadIdx.x == 0) {
+    target += G;
+    __threadfence();
+    atomicAdd(counter, 1u);
+    unsigned it = 0;
+    while (ld_acquire(counter) < target) {
+      if (++it > SPIN_LIMIT_GRID || ((it & 255u) == 0 && *err != DEV_OK)) {
+        atomicCAS(const_cast<int*>(err), DEV_OK, DEV_TIMEOUT_GRID);
+        break;
+      }
+    }
+    __threadfence();
+  }
+  named_sync(1, CONSUMER_THREADS);
+}
+
+// ------------------------------------------------------------------------------ attention
+
+template <typename CT> struct CTraits;
+template <> struct CTraits<__nv_bfloat16> {
+  static constexpr int E = 8;
+  static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&f)[8]) {
+    const uint4 r = __ldcg(reinterpret_cast<const uint4*>(p));
+    f[0] = bf16lo(r.x); f[1] = bf16hi(r.x); f[2] = bf16lo(r.y); f[3] = bf16hi(r.y);
+    f[4] = bf16lo(r.z); f[5] = bf16hi(r.z); f[6] = bf16lo(r.w); f[7] = bf16hi(r.w);
+  }
+};
+template <> struct CTraits<float> {
+  static constexpr int E = 4;
+  static __device__ __forceinline__ void load(const float* p, float (&f)[4]) {
+    const float4 r = __ldcg(reinterpret_cast<const float4*>(p));
+    f[0] = r.x; f[1] = r.y; f[2] = r.z; f[3] = r.w;
+  }
+};
+
+// Query row m (position pos0+m) attends cache rows 0..pos0+m.  Work unit = (head, KV
+// split); each unit leaves an unnormalised partial output with its row max and sum; the
+// CTA that finishes a head's last split merges them (no waiting).
+template <int M, typename CT>
+__device__ void attn_phase(const ModelDev& md, int layer, int pos0, int cta, int G, float* xs, Ctrl* ctl) {
+  constexpr int E = CTraits<CT>::E;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int H = md.H, dh = md.dh, d = md.d, nsplit = md.nsplit;
+  const int len = pos0 + M;
+  const int Lc = (len + nsplit - 1) / nsplit;
+  const int Lcp = (Lc + 3) & ~3;
+  const int LPP = dh / E, PPI = 32 / LPP;
+  const int sub = lane / LPP, li = lane - sub * LPP;
+  float* qs = xs;                   // [M][dh]
+  float* S = qs + M * dh;           // [M][Lcp]
+  float* red = S + M * Lcp;         // [8][M][dh]
+  const CT* Kl = static_cast<const CT*>(md.kcache) + (size_t)layer * md.max_seq * d;
+  const CT* Vl = static_cast<const CT*>(md.vcache) + (size_t)layer * md.max_seq * d;
+
+  for (int unit = cta; unit < H * nsplit; unit += G) {
+    const int h = unit / nsplit, sp = unit - h * nsplit;
+    const int p0 = sp * Lc, p1 = min(len, p0 + Lc);
+    for (int i = tid; i < M * dh; i += CONSUMER_THREADS) {
+      const int m = i / dh, c = i - m * dh;
+      qs[i] = ldcg(md.qbuf + (size_t)m * d + h * dh + c) * md.scale;
+    }
+    named_sync(1, CONSUMER_THREADS);
+    float qr[M][E];
+#pragma unroll
+    for (int m = 0; m < M; ++m)
+#pragma unroll
+      for (int e = 0; e < E; ++e) qr[m][e] = qs[m * dh + li * E + e];
+    // scores
+    for (int pb = p0 + warp * PPI; pb < p1; pb += 8 * PPI) {
+      const int p = pb + sub;
+      const bool valid = p < p1;
+      float kf[E];
+#pragma unroll
+      for (int e = 0; e < E; ++e) kf[e] = 0.f;
+      if (valid) CTraits<CT>::load(Kl + (size_t)p * d + h * dh + li * E, kf);
+      float part[M];
+#pragma unroll
+      for (int m = 0; m < M; ++m) {
+        float s = 0.f;
+#pragma unroll
+        for (int e = 0; e < E; ++e) s = fmaf(kf[e], qr[m][e], s);
+        part[m] = s;
+      }
+      for (int o = LPP >> 1; o; o >>= 1)
+#pragma unroll
+        for (int m = 0; m < M; ++m) part[m] += __shfl_xor_sync(0xffffffffu, part[m], o);
+      if (valid && li == 0) {
+#pragma unroll
+        for (int m = 0; m < M; ++m) S[m * Lcp + (p - p0)] = (p <= pos0 + m) ? part[m] : -INFINITY;
+      }
+    }
+    named_sync(1, CONSUMER_THREADS);
+    // per-row max, exponentials, sum: warp m takes row m
+    if (warp < M) {
+      const int n = p1 - p0;
+      float* row = S + warp * Lcp;
+      float mx = -INFINITY;
+      for (int i = lane; i < n; i += 32) mx = fmaxf(mx, row[i]);
+#pragma unroll
+      for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      float sum = 0.f;
+      for (int i = lane; i < n; i += 32) {
+        const float ex = (mx == -INFINITY) ? 0.f : expf(row[i] - mx);
+        row[i] = ex;
+        sum += ex;
+      }
+#pragma unroll
+      for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      if (lane == 0) { ctl->rowmax[warp] = mx; ctl->rowsum[warp] = sum; }
+    }
+    named_sync(1, CONSUMER_THREADS);
+    // weighted sum of V rows
+    float acc[M][E];
+#pragma unroll
+    for (int m = 0; m < M; ++m)
+#pragma unroll
+      for (int e = 0; e < E; ++e) acc[m][e] = 0.f;
+    for (int pb = p0 + warp * PPI; pb < p1; pb += 8 * PPI) {
+      const int p = pb + sub;
+      if (p < p1) {
+        float vf[E];
+        CTraits<CT>::load(Vl + (size_t)p * d + h * dh + li * E, vf);
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+          const float w = S[m * Lcp + (p - p0)];
+#pragma unroll
+          for (int e = 0; e < E; ++e) acc[m][e] = fmaf(w, vf[e], acc[m][e]);
+        }
+      }
+    }
+    for (int o = LPP; o < 32; o <<= 1)
+#pragma unroll
+      for (int m = 0; m < M; ++m)
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[m][e] += __shfl_xor_sync(0xffffffffu, acc[m][e], o);
+    if (sub == 0) {
+#pragma unroll
+      for (int m = 0; m < M; ++m)
+#pragma unroll
+        for (int e = 0; e < E; ++e) red[(warp * M + m) * dh + li * E + e] = acc[m][e];
+    }
+    named_sync(1, CONSUMER_THREADS);
+    float* part_out = md.apart + ((size_t)(h * nsplit + sp) * MAX_M) * dh;
+    for (int i = tid; i < M * dh; i += CONSUMER_THREADS) {
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) s += red[w * M * dh + i];
+      stcg(part_out + i, s);
+    }
+    if (tid < M) {
+      float* ml = md.aml + ((size_t)(h * nsplit + sp) * MAX_M + tid) * 2;
+      stcg(ml, ctl->rowmax[tid]);
+      stcg(ml + 1, ctl->rowsum[tid]);
+    }
+    __threadfence();
+    named_sync(1, CONSUMER_THREADS);
+    if (tid == 0) {
+      const unsigned old = atomicAdd(md.head_cnt + h, 1u);
+      ctl->flag = (old == (unsigned)nsplit - 1u);
+      __threadfence();
+    }
+    named_sync(1, CONSUMER_THREADS);
+    if (ctl->flag) {
+      for (int i = tid; i < M * dh; i += CONSUMER_THREADS) {
+        const int m = i / dh, c = i - m * dh;
+        float gmax = -INFINITY;
+        for (int s2 = 0; s2 < nsplit; ++s2)
+          gmax = fmaxf(gmax, ldcg(md.aml + ((size_t)(h * nsplit + s2) * MAX_M + m) * 2));
+        float num = 0.f, den = 0.f;
+        for (int s2 = 0; s2 < nsplit; ++s2) {
+          const float* ml = md.aml + ((size_t)(h * nsplit + s2) * MAX_M + m) * 2;
+          const float mx = ldcg(ml);
+          const float w = (mx == -INFINITY) ? 0.f : expf(mx - gmax);
+          den = fmaf(w, ldcg(ml + 1), den);
+          num = fmaf(w, ldcg(md.apart + ((size_t)(h * nsplit + s2) * MAX_M) * dh + i), num);
+        }
+        stcg(md.attn + (size_t)m * d + h * dh + c, num / den);
+      }
+      if (tid == 0) md.head_cnt[h] = 0u;
+    }
+    named_sync(1, CONSUMER_THREADS);
+  }
+}
+
+// ------------------------------------------------------------------------------ sampling
+
+// Row statistics of logits/T over a slice of the vocabulary, one slice per CTA.
+template <int M>
+__device__ void stats_phase(const float* logits, int V, int rows0, int nrows, float temperature, int cta, int G,
+                            float* stat_part, Ctrl* ctl) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int VS = (V + G - 1) / G;
+  const int k0 = cta * VS, k1 = min(V, k0 + VS);
+  for (int r = 0; r < nrows; ++r) {
+    const float* row = logits + (size_t)(rows0 + r) * V;
+    float mx = -INFINITY, av = -INFINITY;
+    int ai = 0x7fffffff;
+    for (int k = k0 + tid; k < k1; k += CONSUMER_THREADS) {
+      const float l = ldcg(row + k);
+      const float s = __fdiv_rn(l, temperature);
+      mx = fmaxf(mx, s);
+      if (l > av || ai == 0x7fffffff) { av = l; ai = k; }
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      const float ov = __shfl_xor_sync(0xffffffffu, av, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, ai, o);
+      if (oi != 0x7fffffff && (ai == 0x7fffffff || ov > av || (ov == av && oi < ai))) { av = ov; ai = oi; }
+    }
+    if (lane == 0) { ctl->sc.fval[warp] = mx; ctl->sc.amax[warp] = av; ctl->sc.aidx[warp] = ai; }
+    named_sync(1, CONSUMER_THREADS);
+    float cmx = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) cmx = fmaxf(cmx, ctl->sc.fval[w]);
+    float sum = 0.f;
+    for (int k = k0 + tid; k < k1; k += CONSUMER_THREADS)
+      sum += expf(__fdiv_rn(ldcg(row + k), temperature) - cmx);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    named_sync(1, CONSUMER_THREADS);
+    if (lane == 0) ctl->sc.fval[warp] = sum;
+    named_sync(1, CONSUMER_THREADS);
+    if (tid == 0) {
+      float tot = 0.f;
+      float bv = ctl->sc.amax[0];
+      int bi = ctl->sc.aidx[0];
+#pragma unroll
+      for (int w = 0; w < 8; ++w) {
+        tot += ctl->sc.fval[w];
+        const int oi = ctl->sc.aidx[w];
+        if (oi != 0x7fffffff && (bi == 0x7fffffff || ctl->sc.amax[w] > bv || (ctl->sc.amax[w] == bv && oi < bi))) {
+          bv = ctl->sc.amax[w];
+          bi = oi;
+        }
+      }
+      float* o = stat_part + ((size_t)cta * MAX_M + r) * 4;
+      stcg(o, cmx); stcg(o + 1, tot); stcg(o + 2, bv); stcg(o + 3, __int_as_float(bi));
+    }
+    named_sync(1, CONSUMER_THREADS);
+  }
+}
+
+// Merge the per-CTA slices: row max, sum of exp, argmax (lowest index on ties).
+__device__ void merge_stats(const float* stat_part, int G, int nrows, Ctrl* ctl, float* rmax, float* rsum,
+                            int* rarg) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (warp < nrows) {
+    const int r = warp;
+    float mx = -INFINITY, av = -INFINITY;
+    int ai = 0x7fffffff;
+    for (int c = lane; c < G; c += 32) {
+      const float* o = stat_part + ((size_t)c * MAX_M + r) * 4;
+      mx = fmaxf(mx, ldcg(o));
+      const float ov = ldcg(o + 2);
+      const int oi = __float_as_int(ldcg(o + 3));
+      if (oi != 0x7fffffff && (ai == 0x7fffffff || ov > av || (ov == av && oi < ai))) { av = ov; ai = oi; }
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      const float ov = __shfl_xor_sync(0xffffffffu, av, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, ai, o);
+      if (oi != 0x7fffffff && (ai == 0x7fffffff || ov > av || (ov == av && oi < ai))) { av = ov; ai = oi; }
+    }
+    float sum = 0.f;
+    for (int c = lane; c < G; c += 32) {
+      const float* o = stat_part + ((size_t)c * MAX_M + r) * 4;
+      const float cm = ldcg(o);
+      if (cm != -INFINITY) sum += ldcg(o + 1) * expf(cm - mx);
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) { rmax[r] = mx; rsum[r] = sum; rarg[r] = ai; }
+  }
+  named_sync(1, CONSUMER_THREADS);
+}
+
+__device__ __noinline__ float prob_of(float logit, float temperature, float rmax, float rsum) {
+  return __fdiv_rn(expf(__fsub_rn(__fdiv_rn(logit, temperature), rmax)), rsum);
+}
+
+}  // namespace spd
