@@ -90,18 +90,26 @@ class SpdOracle:
 
     # ---- step 2
     def draft(self, gamma: int, u_draft):
-        ids, probs, raw = [], [], []
+        ids, probs, raw, used = [], [], [], []
         feed = self.seq[self.d_fed:]                    # pending, plus an unseen accepted token
         pos0 = self.off + self.d_fed
         for j in range(gamma):
             logits = self.d.forward(self.dc, self.d.embed(feed), pos0)
             raw.append(logits[-1])
-            x, prob = self._pick(logits[-1], None if self.greedy else u_draft[j])
+            if self.greedy:
+                uj = None
+            elif callable(u_draft):      # the caller picks u after seeing q_j (test harness)
+                uj = u_draft(j, S.softmax_t(logits[-1], self.temperature))
+            else:
+                uj = u_draft[j]
+            x, prob = self._pick(logits[-1], uj)
+            used.append(0.0 if uj is None else float(uj))
             ids.append(x)
             probs.append(prob)
             pos0 += len(feed)
             feed = [x]
         self.last_draft_logits = np.stack(raw) if raw else None
+        self.last_draft_u = np.asarray(used, dtype=F32)
         q = None if (self.greedy or gamma == 0) else np.stack(probs).astype(F32)
         return np.asarray(ids, dtype=np.int32), q
 
@@ -117,6 +125,9 @@ class SpdOracle:
         else:
             p = S.softmax_t(logits, self.temperature)
             self.last_p = p
+            if callable(u):              # the caller picks the uniforms after seeing p and q
+                u = u(p, q, ids)
+            self.last_u = np.asarray(u, dtype=F32)
             a, nxt = S.reject_sample(p, q, ids, u, greedy=False)
         old_len = len(self.seq)
         self.seq += ids[:a] + [nxt]

@@ -160,8 +160,7 @@ __device__ void produce_gemm(const Gemm& g, int cta, int G, int& off, Ring& ring
       const int k0 = c * kcl, klen = min(kcl, g.K - k0);
       for (int s = 0; s * KSTEP < klen; ++s) {
         const unsigned bytes = min(KSTEP, klen - s * KSTEP) * sizeof(WT);
-        mbar_wait(&ctl->empty[ring.stage], ring.phase ^ 1u, err, DEV_TIMEOUT_EMPTY);
-        if (*err != DEV_OK) return;
+        if (!mbar_wait(&ctl->empty[ring.stage], ring.phase ^ 1u, err, DEV_TIMEOUT_EMPTY)) return;
         if (lane == 0) mbar_arrive_expect_tx(&ctl->full[ring.stage], bytes * nrows);
         __syncwarp();
         if (rv)

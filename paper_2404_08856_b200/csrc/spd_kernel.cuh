@@ -123,7 +123,6 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
       for (int i = 0; i < n_gemm; ++i) {
         const Gemm g = get_gemm(md, i);
         produce_gemm<WT>(g, cta, G, off, ring, ctl, stages, pol, err);
-        if (*err != DEV_OK) break;
       }
     }
   } else {

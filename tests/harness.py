@@ -1,0 +1,99 @@
+"""Shared helpers of the GPU parity tests: build the CUDA context and the CPU oracle from
+the same seeded inputs, and drive both in lock-step.
+
+Sampling decisions compare a floating-point quantity with a uniform.  The two sides agree
+bit for bit only when that quantity is not within rounding distance of the uniform, so the
+harness lets the ORACLE choose each uniform from a seeded stream and skip candidates that
+fall too close to a decision boundary (the margins below).  Inputs therefore depend on the
+oracle and the seed only, never on the CUDA path, and every compared decision has exactly
+one correct answer.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+import synth
+from oracle import llama, sampling as S
+from oracle.spd import SpdOracle
+
+F32 = np.float32
+
+
+def build_weights(wl, std=0.02):
+    tw = synth.Weights(wl.target, wl.seeds["weights"], "target", std=std)
+    dw = synth.Weights(wl.draft, wl.seeds["weights"], "draft", adapter_in=wl.adapter_in, std=std)
+    return tw, dw
+
+
+def make_oracle(wl, tw, dw, max_seq, temperature=1.0, greedy=False):
+    t = llama.Model(wl.target, tw, max_seq)
+    d = llama.Model(wl.draft, dw, max_seq)
+    ad = dw.f32("adapter") if wl.adapter_in else None
+    return SpdOracle(t, d, temperature, greedy, adapter_w=ad)
+
+
+def make_gpu(wl, tw, dw, max_seq, temperature=1.0, greedy=False, gamma_max=7):
+    import paper_2404_08856_b200 as spd
+    return spd.Spd(wl.target, wl.draft, tw.stored, dw.stored, max_seq, gamma_max, temperature, greedy,
+                   adapter_in=wl.adapter_in)
+
+
+class SafeUniforms:
+    """Seeded stream of uniforms on the 2^-24 grid from which the oracle side picks the
+    first candidate that keeps a decision away from its boundary."""
+
+    def __init__(self, seed, tag, accept_margin=2e-3, cdf_margin=2e-6, n=1 << 16):
+        self.pool = synth.uniforms(seed, tag, n)
+        self.i = 0
+        self.skipped = 0
+        self.accept_margin, self.cdf_margin = accept_margin, cdf_margin
+
+    def _next(self):
+        u = self.pool[self.i]
+        self.i += 1
+        return F32(u)
+
+    def for_cdf(self, w):
+        """u whose inverse-CDF threshold is at least cdf_margin * Z from both ends of the
+        selected token's interval."""
+        W = S.fixed_point(w).astype(np.float64)
+        cum = np.cumsum(W)
+        Z = cum[-1]
+        while True:
+            u = self._next()
+            t = Z * float(u)
+            k = int(np.searchsorted(cum, t, side="right"))
+            lo = cum[k - 1] if k else 0.0
+            if t - lo > self.cdf_margin * Z and cum[k] - t > self.cdf_margin * Z:
+                return u
+            self.skipped += 1
+
+    def for_accept(self, p_x, q_x):
+        a = float(S.accept_prob(p_x, q_x))
+        while True:
+            u = self._next()
+            if abs(float(u) - a) > self.accept_margin or (a >= 1.0):
+                return u
+            self.skipped += 1
+
+    # hooks for SpdOracle.draft / SpdOracle.verify
+    def draft_hook(self, j, prob):
+        return self.for_cdf(prob)
+
+    def verify_hook(self, p, q, ids):
+        gamma = len(ids)
+        u = np.zeros(gamma + 1, dtype=F32)
+        r = gamma
+        for j in range(gamma):
+            x = int(ids[j])
+            u[j] = self.for_accept(p[j, x], q[j, x])
+            if r == gamma and not (u[j] < S.accept_prob(p[j, x], q[j, x])):
+                r = j
+        w = p[gamma] if r == gamma else np.maximum(F32(0), p[r] - q[r])
+        u[gamma] = self.for_cdf(w)
+        return u
+
+
+def top2_gap(row):
+    part = np.partition(row, -2)[-2:]
+    return float(part[1] - part[0])
