@@ -241,7 +241,29 @@ def test_tiny_lockstep(greedy):
     wl = synth.tiny_workload(4)
     r = lockstep(wl, greedy, 1.0, 10, 2e-4, std=0.2 if greedy else 0.1, gammas=[4, 1, 7, 3, 2, 5, 6])
     assert r["blocks"] >= 8
-    assert r["accepted"] > 0, "accept path not exercised"
+    if not greedy:
+        assert r["accepted"] > 0, "accept path not exercised"
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("greedy", [True, False])
+def test_tiny_identical_draft_accepts_everything(greedy):
+    """Draft == target and no image: every draft token is accepted, tau = gamma + 1."""
+    spd = _lib()
+    wl = synth.Workload("same", synth.TINY_TARGET, synth.TINY_TARGET, 0, 16, 3, 24)
+    tw = synth.Weights(wl.target, 1, "target", std=0.2)
+    gpu = spd.Spd(wl.target, wl.target, tw.stored, tw.stored, 128, 7, 1.0, greedy)
+    ids = synth.prompt_ids(wl)
+    gpu.prefill(None, ids, u0=0.3)
+    u = synth.uniforms(3, "same.gpu", (24, 7))
+    out, st = gpu.generate(24, 3, None if greedy else u)
+    assert st["accepted"] == 3 * st["blocks"] and st["tau"] == 4.0
+    orc = H.make_oracle(wl, tw, tw, 128, 1.0, greedy)
+    orc.prefill(None, ids, u0=0.3)
+    want, _ = orc.generate(24, 3, None if greedy else u)
+    if greedy:
+        assert np.array_equal(out, want)
+    gpu.close()
 
 
 @pytest.mark.gpu
@@ -354,6 +376,6 @@ def test_state_and_overflow_errors():
     out, st = gpu.generate(8, 4)          # still usable afterwards
     assert len(out) == 8
     gpu.close()
-    bad = synth.ModelCfg(1, 100, 3, 64, 64, dtype="fp32")
+    bad = synth.ModelCfg(2, 100, 3, 64, 64, dtype="fp32")   # d_model not divisible by heads
     with pytest.raises(spd.SpdError):
-        H.make_gpu(synth.Workload("bad", bad, bad, 0, 4, 1, 4), tw, dw, 48)
+        H.make_gpu(synth.Workload("bad", bad, bad, 0, 4, 1, 4), tw, tw, 48)
