@@ -145,7 +145,7 @@ spd_status spd_verify(spd_ctx* ctx, int gamma, const int32_t* draft_ids,
                       int32_t* n_accepted, int32_t* next_token);
 
 /* Block loop (Fig. 1): repeats draft + verify until n_new tokens exist after the prompt;
- * the token produced by spd_prefill is the first of them.
+ * the pending token (after spd_prefill: the token it produced) is the first of them.
  *   uniforms  fp32 [n_new, 2*gamma+1], host or device: per block gamma draft draws, then
  *             gamma+1 verification uniforms; may be NULL when greedy
  *   out_ids   int32 [n_new], HOST

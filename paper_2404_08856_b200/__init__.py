@@ -166,6 +166,10 @@ class Spd:
                                      C.byref(nxt)))
         return a.value, nxt.value
 
+    def draft_async(self, gamma: int, uniforms_dev=None):
+        """Enqueue gamma draft steps with device-resident uniforms; nothing is read back."""
+        self._check(lib().spd_draft(self._ctx, gamma, _ptr(uniforms_dev), None, None))
+
     def verify_async(self, gamma: int, uniforms_dev=None):
         """Enqueue a verify step with device-resident uniforms; nothing is read back."""
         self._check(lib().spd_verify(self._ctx, gamma, None, None, _ptr(uniforms_dev), None, None))

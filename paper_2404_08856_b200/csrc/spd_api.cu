@@ -260,6 +260,10 @@ KernelFn pick_kernel(int M, int dtype) { return dtype == 1 ? pick_m<__nv_bfloat1
 struct LaunchCfg { int nstage; size_t smem; };
 
 spd_status launch_cfg(spd_ctx* ctx, KernelFn fn, int M, int n_sm, int smem_optin, LaunchCfg* lc) {
+  static LaunchCfg cache[2 * (MAX_M + 1)];   // per kernel variant; filled on first use
+  static KernelFn cache_fn[2 * (MAX_M + 1)];
+  for (int i = 0; i < 2 * (MAX_M + 1); ++i)
+    if (cache_fn[i] == fn) { *lc = cache[i]; return SPD_OK; }
   cudaFuncAttributes fa{};
   CU(cudaFuncGetAttributes(&fa, (const void*)fn));
   const size_t fixed = CTRL_BYTES + (size_t)M * KC_MAX * sizeof(float);
@@ -271,6 +275,8 @@ spd_status launch_cfg(spd_ctx* ctx, KernelFn fn, int M, int n_sm, int smem_optin
   lc->smem = fixed + (size_t)ns * STAGE_BYTES;
   CU(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lc->smem));
   (void)n_sm;
+  for (int i = 0; i < 2 * (MAX_M + 1); ++i)
+    if (!cache_fn[i]) { cache[i] = *lc; cache_fn[i] = fn; break; }
   return SPD_OK;
 }
 
@@ -612,8 +618,14 @@ spd_status spd_generate(spd_ctx* ctx, int n_new, int gamma, const float* uniform
   if (n_new > ctx->out_cap) return fail(ctx, SPD_EOVERFLOW, "n_new exceeds the output buffer");
   spd_status s = sync_state(ctx);
   if (s) return s;
-  if (ctx->st_host->n_emitted != 1 || ctx->st_host->block != 0)
-    return fail(ctx, SPD_ESTATE, "spd_generate must follow spd_prefill directly");
+  {  // the pending token is the first output; uniforms are indexed by block from 0
+    int head[2] = {0, 1};   // block, n_emitted
+    CU(cudaMemcpyAsync(&ctx->st->block, head, sizeof(head), cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaMemcpyAsync(ctx->out_dev, &ctx->st->pending, sizeof(int), cudaMemcpyDeviceToDevice, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    ctx->st_host->n_emitted = 1;
+    ctx->st_host->block = 0;
+  }
   if (ctx->m_image + ctx->len_ub + n_new + gamma + 1 > ctx->cfg.max_seq)
     return fail(ctx, SPD_EOVERFLOW, "n_new does not fit max_seq");
   const int us = 2 * gamma + 1;
