@@ -278,13 +278,49 @@ def run_gpu(args, rank, world):
         dist.destroy_process_group()
 
 
+def run_micro(args):
+    """Times the weight-streaming GEMM alone (the projections of one verify step):
+    y[M,N] = x[M,K] w[N,K]^T, bf16 weights larger than L2, CUDA events, prints one JSON line."""
+    import torch
+    import paper_2404_08856_b200 as spd
+    from paper_2404_08856_b200 import build
+    build.build()
+    M, N, K = args.M, args.N, args.K
+    g = torch.Generator(device="cuda").manual_seed(0)
+    x = torch.randn(M, K, device="cuda", generator=g)
+    w = (torch.randn(N, K, device="cuda", generator=g) * 0.02).to(torch.bfloat16)
+    y = torch.empty(M, N, device="cuda")
+    for _ in range(max(args.warmup, 1)):
+        spd.skinny_gemm(x, w, y, 1)
+    torch.cuda.synchronize()
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    e[0].record()
+    for i in range(args.steps):
+        spd.skinny_gemm(x, w, y, 1)
+        e[i + 1].record()
+    torch.cuda.synchronize()
+    ms = sorted(e[i].elapsed_time(e[i + 1]) for i in range(args.steps))
+    med = ms[len(ms) // 2]
+    peak, kind = measured_peak()
+    gbs = N * K * 2 / (med * 1e-3) / 1e9
+    print(json.dumps({"micro": "skinny_gemm (includes the tile-packing pass of w)", "M": M, "N": N, "K": K,
+                      "ms_median": med, "ms_min": ms[0], "weight_GBs": gbs, "frac_of_peak": gbs / peak,
+                      "peak_kind": kind}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--micro", default=None, choices=["gemm"], help="time one kernel alone instead of the path")
+    ap.add_argument("--M", type=int, default=6)
+    ap.add_argument("--N", type=int, default=32768)
+    ap.add_argument("--K", type=int, default=4096)
     args = ap.parse_args()
+    if args.micro:
+        return run_micro(args)
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
     if args.impl == "reference":

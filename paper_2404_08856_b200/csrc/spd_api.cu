@@ -120,6 +120,34 @@ spd_status put_rows(spd_ctx* ctx, void* dst, const void* src, void* staging, int
   return SPD_OK;
 }
 
+// Row-major [N][K] -> tile-packed [ceil(N/32)][ceil(K/kstep)][32][kstep], zero padded, where
+// kstep elements are 512 bytes.  16 bytes per thread-iteration.
+__global__ void pack_tiles_kernel(char* dst, const char* src, int N, int K, int esz) {
+  const int kstep = 512 / esz, nsteps = (K + kstep - 1) / kstep, ntiles = (N + 31) >> 5;
+  const size_t total = (size_t)ntiles * nsteps * 1024;   // 16-byte chunks
+  const int epc = 16 / esz;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int c = (int)(i & 31), r = (int)((i >> 5) & 31);
+    const size_t blk = i >> 10;
+    const int st = (int)(blk % nsteps), t = (int)(blk / nsteps);
+    const int row = t * 32 + r, k = st * kstep + c * epc;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (row < N && k < K) v = *reinterpret_cast<const uint4*>(src + ((size_t)row * K + k) * esz);
+    reinterpret_cast<uint4*>(dst)[i] = v;
+  }
+}
+
+size_t packed_bytes(int N, int K, size_t esz) {
+  const int kstep = (int)(512 / esz);
+  return (size_t)((N + 31) / 32) * ((K + kstep - 1) / kstep) * STAGE_BYTES;
+}
+
+spd_status pack_tiles(spd_ctx* ctx, void* dst, const void* src_rowmajor, int N, int K, size_t esz, cudaStream_t st) {
+  pack_tiles_kernel<<<1184, 256, 0, st>>>(static_cast<char*>(dst), static_cast<const char*>(src_rowmajor), N, K, (int)esz);
+  CU(cudaGetLastError());
+  return SPD_OK;
+}
+
 spd_status check_model(spd_ctx* ctx, const spd_model_cfg& c, const char* who) {
   auto bad = [&](const char* what) { return fail(ctx, SPD_EINVAL, std::string(who) + ": " + what); };
   if (c.n_layers < 1 || c.d_model < 8 || c.n_heads < 1 || c.d_ffn < 8 || c.vocab < 2) return bad("non-positive shape");
@@ -134,7 +162,7 @@ spd_status check_model(spd_ctx* ctx, const spd_model_cfg& c, const char* who) {
 }
 
 spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, const spd_weights* w, int adapter_in,
-                       void* staging) {
+                       void* staging, char* rm) {
   mh.cfg = c;
   const size_t esz = c.dtype == 1 ? 2 : 4;
   mh.esz = esz;
@@ -150,12 +178,11 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
   if ((s = dalloc(ctx, &embed, (size_t)V * d * esz))) return s;
   if ((s = put_rows(ctx, embed, w->tok_embed, staging, V, d, esz, 1, 0, 0))) return s;
   md.embed = embed;
-  if (c.tied_embeddings) {
-    md.lm_head = embed;
-  } else {
+  {  // the LM head is streamed tile-packed; a tied head is a packed copy of the table
     char* lm = nullptr;
-    if ((s = dalloc(ctx, &lm, (size_t)V * d * esz))) return s;
-    if ((s = put_rows(ctx, lm, w->lm_head, staging, V, d, esz, 1, 0, 0))) return s;
+    if ((s = dalloc(ctx, &lm, packed_bytes(V, d, esz)))) return s;
+    if ((s = put_rows(ctx, rm, c.tied_embeddings ? w->tok_embed : w->lm_head, staging, V, d, esz, 1, 0, 0))) return s;
+    if ((s = pack_tiles(ctx, lm, rm, V, d, esz, ctx->stream))) return s;
     md.lm_head = lm;
   }
   float* fn = nullptr;
@@ -166,8 +193,9 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
   if (adapter_in > 0) {
     if (!w->adapter) return fail(ctx, SPD_EINVAL, "draft_adapter_in > 0 but no adapter weights");
     char* ad = nullptr;
-    if ((s = dalloc(ctx, &ad, (size_t)d * adapter_in * esz))) return s;
-    if ((s = put_rows(ctx, ad, w->adapter, staging, d, adapter_in, esz, 1, 0, 0))) return s;
+    if ((s = dalloc(ctx, &ad, packed_bytes(d, adapter_in, esz)))) return s;
+    if ((s = put_rows(ctx, rm, w->adapter, staging, d, adapter_in, esz, 1, 0, 0))) return s;
+    if ((s = pack_tiles(ctx, ad, rm, d, adapter_in, esz, ctx->stream))) return s;
     mh.adapter = ad;
   }
   std::vector<LayerDev> layers(L);
@@ -176,19 +204,24 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
   for (int l = 0; l < L; ++l) {
     char *wqkv, *wo, *wgu, *wd;
     float *an, *fnw;
-    if ((s = dalloc(ctx, &wqkv, (size_t)3 * d * d * esz))) return s;
-    if ((s = dalloc(ctx, &wo, (size_t)d * d * esz))) return s;
-    if ((s = dalloc(ctx, &wgu, (size_t)2 * f * d * esz))) return s;
-    if ((s = dalloc(ctx, &wd, (size_t)d * f * esz))) return s;
+    if ((s = dalloc(ctx, &wqkv, packed_bytes(3 * d, d, esz)))) return s;
+    if ((s = dalloc(ctx, &wo, packed_bytes(d, d, esz)))) return s;
+    if ((s = dalloc(ctx, &wgu, packed_bytes(2 * f, d, esz)))) return s;
+    if ((s = dalloc(ctx, &wd, packed_bytes(d, f, esz)))) return s;
     if ((s = dalloc(ctx, &an, (size_t)d))) return s;
     if ((s = dalloc(ctx, &fnw, (size_t)d))) return s;
-    if ((s = put_rows(ctx, wqkv, w->wq[l], staging, d, d, esz, 1, 0, dh))) return s;
-    if ((s = put_rows(ctx, wqkv + (size_t)d * d * esz, w->wk[l], staging, d, d, esz, 1, 0, dh))) return s;
-    if ((s = put_rows(ctx, wqkv + (size_t)2 * d * d * esz, w->wv[l], staging, d, d, esz, 1, 0, 0))) return s;
-    if ((s = put_rows(ctx, wo, w->wo[l], staging, d, d, esz, 1, 0, 0))) return s;
-    if ((s = put_rows(ctx, wgu, w->w_gate[l], staging, f, d, esz, 2, 0, 0))) return s;
-    if ((s = put_rows(ctx, wgu, w->w_up[l], staging, f, d, esz, 2, 1, 0))) return s;
-    if ((s = put_rows(ctx, wd, w->w_down[l], staging, d, f, esz, 1, 0, 0))) return s;
+    // compose the permuted row-major matrix in `rm`, then tile-pack it
+    if ((s = put_rows(ctx, rm, w->wq[l], staging, d, d, esz, 1, 0, dh))) return s;
+    if ((s = put_rows(ctx, rm + (size_t)d * d * esz, w->wk[l], staging, d, d, esz, 1, 0, dh))) return s;
+    if ((s = put_rows(ctx, rm + (size_t)2 * d * d * esz, w->wv[l], staging, d, d, esz, 1, 0, 0))) return s;
+    if ((s = pack_tiles(ctx, wqkv, rm, 3 * d, d, esz, ctx->stream))) return s;
+    if ((s = put_rows(ctx, rm, w->wo[l], staging, d, d, esz, 1, 0, 0))) return s;
+    if ((s = pack_tiles(ctx, wo, rm, d, d, esz, ctx->stream))) return s;
+    if ((s = put_rows(ctx, rm, w->w_gate[l], staging, f, d, esz, 2, 0, 0))) return s;
+    if ((s = put_rows(ctx, rm, w->w_up[l], staging, f, d, esz, 2, 1, 0))) return s;
+    if ((s = pack_tiles(ctx, wgu, rm, 2 * f, d, esz, ctx->stream))) return s;
+    if ((s = put_rows(ctx, rm, w->w_down[l], staging, d, f, esz, 1, 0, 0))) return s;
+    if ((s = pack_tiles(ctx, wd, rm, d, f, esz, ctx->stream))) return s;
     if (!w->attn_norm[l] || !w->ffn_norm[l]) return fail(ctx, SPD_EINVAL, "missing norm gain");
     CU(cudaMemcpyAsync(an, w->attn_norm[l], d * sizeof(float), cudaMemcpyDefault, ctx->stream));
     CU(cudaMemcpyAsync(fnw, w->ffn_norm[l], d * sizeof(float), cudaMemcpyDefault, ctx->stream));
@@ -423,11 +456,17 @@ spd_status spd_create(const spd_weights* target_w, const spd_weights* draft_w, c
     if (big > stage_elems) stage_elems = big;
   }
   (void)esz_t; (void)esz_d;
-  char* staging = nullptr;
-  if (cudaMalloc(&staging, stage_elems + 256) != cudaSuccess) return bail(fail(ctx, SPD_ENOMEM, "staging allocation failed"));
-  s = build_model(ctx, ctx->target, cfg->target, target_w, 0, staging);
-  if (!s) s = build_model(ctx, ctx->draft, cfg->draft, draft_w, cfg->draft_adapter_in, staging);
+  char *staging = nullptr, *rowmajor = nullptr;
+  if (cudaMalloc(&staging, stage_elems + 256) != cudaSuccess ||
+      cudaMalloc(&rowmajor, 3 * stage_elems + 256) != cudaSuccess) {
+    cudaFree(staging);
+    return bail(fail(ctx, SPD_ENOMEM, "staging allocation failed"));
+  }
+  s = build_model(ctx, ctx->target, cfg->target, target_w, 0, staging, rowmajor);
+  if (!s) s = build_model(ctx, ctx->draft, cfg->draft, draft_w, cfg->draft_adapter_in, staging, rowmajor);
+  cudaStreamSynchronize(ctx->stream);
   cudaFree(staging);
+  cudaFree(rowmajor);
   if (s) return bail(s);
   const int V = cfg->target.vocab;
   const int dmax = cfg->target.d_model > cfg->draft.d_model ? cfg->target.d_model : cfg->draft.d_model;
@@ -737,10 +776,14 @@ spd_status spd_reject_sample(const float* p, const float* q, const int32_t* ids,
 
 spd_status spd_skinny_gemm(const float* x, const void* w, int dtype, int M, int N, int K, float* y, void* stream) {
   if (!x || !w || !y || M < 1 || M > MAX_M || N < 1 || K < 8 || K % 8 || (dtype != 0 && dtype != 1)) return SPD_EINVAL;
+  // per-process scratch: a grid-barrier word, a status block and the tile-packed copy of w
   static unsigned* bar = nullptr;
   static DevState* st = nullptr;
+  static char* packed = nullptr;
+  static size_t packed_cap = 0;
   static int n_sm = 0, smem_optin = 0;
   spd_ctx* ctx = nullptr;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
   if (!bar) {
     int dev = 0;
     cudaDeviceProp prop{};
@@ -751,11 +794,22 @@ spd_status spd_skinny_gemm(const float* x, const void* w, int dtype, int M, int 
     if (cudaMalloc(&bar, 256) != cudaSuccess || cudaMalloc(&st, sizeof(DevState)) != cudaSuccess) return SPD_ENOMEM;
     cudaMemset(st, 0, sizeof(DevState));
   }
+  const size_t esz = dtype == 1 ? 2 : 4;
+  const size_t need = packed_bytes(N, K, esz);
+  if (need > packed_cap) {
+    cudaStreamSynchronize(cs);
+    if (packed) cudaFree(packed);
+    packed = nullptr; packed_cap = 0;
+    if (cudaMalloc(&packed, need) != cudaSuccess) return SPD_ENOMEM;
+    packed_cap = need;
+  }
+  spd_status s = pack_tiles(ctx, packed, w, N, K, esz, cs);
+  if (s) return s;
   StepArgs a{};
   a.mode = MODE_GEMM;
   a.st = st;
-  a.gx = x; a.gw = w; a.gy = y; a.gN = N; a.gK = K;
-  return launch_forward(ctx, M, dtype, a, static_cast<cudaStream_t>(stream), n_sm, smem_optin, bar);
+  a.gx = x; a.gw = packed; a.gy = y; a.gN = N; a.gK = K;
+  return launch_forward(ctx, M, dtype, a, cs, n_sm, smem_optin, bar);
 }
 
 spd_status spd_verify_bytes(spd_ctx* ctx, int gamma, double* bytes) {

@@ -143,31 +143,26 @@ struct Ring {
 
 // ------------------------------------------------------------------------------ producer
 
+// Weights are stored tile-packed: for each tile of 32 rows, for each K step of 512 bytes
+// per row, one contiguous 16 KB block [32 rows][512 B] (rows beyond N and columns beyond K
+// are zero).  One bulk copy moves a whole ring stage.
 template <typename WT>
 __device__ void produce_gemm(const Gemm& g, int cta, int G, int& off, Ring& ring, Ctrl* ctl, char* stages,
                              uint64_t pol, volatile int* err) {
   constexpr int EPL = WTraits<WT>::EPL, KSTEP = 32 * EPL;
   const int lane = threadIdx.x & 31;
   const int ntiles = (g.N + 31) >> 5;
-  int nchunk, kcl;
-  chunking(g.K, KSTEP, nchunk, kcl);
+  const int nsteps = (g.K + KSTEP - 1) / KSTEP;
   for (int t = (cta - off + G) % G; t < ntiles; t += G) {
-    const int row = t * 32 + lane;
-    const bool rv = row < g.N;
-    const unsigned nrows = min(32, g.N - t * 32);
-    const char* wrow = static_cast<const char*>(g.W) + (size_t)(rv ? row : 0) * g.K * sizeof(WT);
-    for (int c = 0; c < nchunk; ++c) {
-      const int k0 = c * kcl, klen = min(kcl, g.K - k0);
-      for (int s = 0; s * KSTEP < klen; ++s) {
-        const unsigned bytes = min(KSTEP, klen - s * KSTEP) * sizeof(WT);
-        if (!mbar_wait(&ctl->empty[ring.stage], ring.phase ^ 1u, err, DEV_TIMEOUT_EMPTY)) return;
-        if (lane == 0) mbar_arrive_expect_tx(&ctl->full[ring.stage], bytes * nrows);
-        __syncwarp();
-        if (rv)
-          bulk_g2s(stages + (size_t)ring.stage * STAGE_BYTES + lane * 512,
-                   wrow + (size_t)(k0 + s * KSTEP) * sizeof(WT), bytes, &ctl->full[ring.stage], pol);
-        ring.advance();
+    const char* src = static_cast<const char*>(g.W) + (size_t)t * nsteps * STAGE_BYTES;
+    for (int s = 0; s < nsteps; ++s) {
+      if (!mbar_wait(&ctl->empty[ring.stage], ring.phase ^ 1u, err, DEV_TIMEOUT_EMPTY)) return;
+      if (lane == 0) {
+        mbar_arrive_expect_tx(&ctl->full[ring.stage], STAGE_BYTES);
+        bulk_g2s(stages + (size_t)ring.stage * STAGE_BYTES, src + (size_t)s * STAGE_BYTES, STAGE_BYTES,
+                 &ctl->full[ring.stage], pol);
       }
+      ring.advance();
     }
   }
   off = (off + ntiles) % G;
@@ -320,17 +315,15 @@ __device__ __forceinline__ void epilogue_pair(int epi, const EpiArgs& e, int m, 
 // ------------------------------------------------------------------------------ consumer
 
 template <int M, typename WT>
-__device__ __forceinline__ void compute_step(const char* stage, const float* X, int kp4, int s, int len, int warp,
+__device__ __forceinline__ void compute_step(const char* stage, const float* X, int kp4, int s, int warp,
                                              int lane, float2 (&acc)[4][M]) {
   constexpr int EPL = WTraits<WT>::EPL;
-  const bool active = lane * EPL < len;
   const uint4* wp = reinterpret_cast<const uint4*>(stage + warp * 2048 + lane * 16);
   if constexpr (EPL == 8) {
     float2 w[4][4];
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
-      uint4 q = wp[r * 32];
-      if (!active) q = make_uint4(0, 0, 0, 0);
+      const uint4 q = wp[r * 32];
       w[r][0] = make_float2(bf16lo(q.x), bf16hi(q.x));
       w[r][1] = make_float2(bf16lo(q.y), bf16hi(q.y));
       w[r][2] = make_float2(bf16lo(q.z), bf16hi(q.z));
@@ -356,8 +349,7 @@ __device__ __forceinline__ void compute_step(const char* stage, const float* X, 
     float2 w[4][2];
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
-      uint4 q = wp[r * 32];
-      if (!active) q = make_uint4(0, 0, 0, 0);
+      const uint4 q = wp[r * 32];
       w[r][0] = make_float2(__uint_as_float(q.x), __uint_as_float(q.y));
       w[r][1] = make_float2(__uint_as_float(q.z), __uint_as_float(q.w));
     }
@@ -410,8 +402,7 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, Fetch fetch, const
       }
       for (int s = 0; s * KSTEP < klen; ++s) {
         mbar_wait(&ctl->full[ring.stage], ring.phase, err, DEV_TIMEOUT_FULL);
-        compute_step<M, WT>(stages + (size_t)ring.stage * STAGE_BYTES, X, kp4, s, min(KSTEP, klen - s * KSTEP), warp,
-                            lane, acc);
+        compute_step<M, WT>(stages + (size_t)ring.stage * STAGE_BYTES, X, kp4, s, warp, lane, acc);
         __syncwarp();
         if (lane == 0) mbar_arrive(&ctl->empty[ring.stage]);
         ring.advance();
