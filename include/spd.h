@@ -169,6 +169,14 @@ spd_status spd_get_draft_logits(spd_ctx* ctx, float* logits, int rows);
 spd_status spd_rollback(spd_ctx* ctx, int n_text, int32_t prev_token, int32_t pending_token);
 spd_status spd_get_state(spd_ctx* ctx, int32_t* n_text, int32_t* pending_token);
 
+/* Phase trace of spd_verify.  The first call switches tracing on (returns *n = 0).  Later
+ * calls copy the trace of the last spd_verify into stamps[cap] (HOST).  Each entry is
+ * (%globaltimer in ns << 8) | id, written by CTA 0: id 0 kernel start, 1 activation tile of
+ * a projection built, 2 its last weight stage consumed, 3 phase finished, 4 grid barrier
+ * passed.  Per layer the phases are QKV, attention, O-projection, gate/up, down; then LM
+ * head, row statistics, sampling. */
+spd_status spd_trace(spd_ctx* ctx, uint64_t* stamps, int cap, int* n);
+
 /* The rejection rule alone (Sec. 2.1) on given probabilities, B independent sequences:
  *   p [B, gamma+1, V], q [B, gamma, V] fp32 DEVICE (q may be NULL when greedy)
  *   ids int32 [B, gamma], u fp32 [B, gamma+1] DEVICE (u may be NULL when greedy)

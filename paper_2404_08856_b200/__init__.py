@@ -20,7 +20,7 @@ STATUS_NAMES = ["SPD_OK", "SPD_EINVAL", "SPD_ESTATE", "SPD_ENOMEM", "SPD_EOVERFL
 
 EXPORTS = ["spd_create", "spd_destroy", "spd_last_error", "spd_prefill", "spd_draft", "spd_verify",
            "spd_generate", "spd_get_logits", "spd_get_draft_logits", "spd_rollback", "spd_get_state",
-           "spd_reject_sample", "spd_skinny_gemm", "spd_verify_bytes"]
+           "spd_reject_sample", "spd_skinny_gemm", "spd_verify_bytes", "spd_trace"]
 
 
 class SpdError(RuntimeError):
@@ -200,6 +200,13 @@ class Spd:
         n, p = C.c_int32(0), C.c_int32(0)
         self._check(lib().spd_get_state(self._ctx, C.byref(n), C.byref(p)))
         return n.value, p.value
+
+    def trace(self) -> np.ndarray:
+        """Phase timestamps (ns) of the last verify step; the first call enables tracing."""
+        out = np.zeros(1024, dtype=np.uint64)
+        n = C.c_int(0)
+        self._check(lib().spd_trace(self._ctx, _ptr(out), 1024, C.byref(n)))
+        return out[: n.value].copy()
 
     def verify_bytes(self, gamma: int) -> float:
         b = C.c_double(0)

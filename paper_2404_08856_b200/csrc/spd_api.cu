@@ -53,6 +53,8 @@ struct spd_ctx {
   int len_ub = 0;               // upper bound of n_text known to the host
   int n_prompt = 0, m_image = 0;
   int last_verify_rows = 0, last_draft_rows = 0;
+  unsigned long long* trace = nullptr;   // device buffer of phase timestamps (verify steps)
+  int trace_cap = 0;
   cudaEvent_t ev[4]{};
 };
 
@@ -120,30 +122,43 @@ spd_status put_rows(spd_ctx* ctx, void* dst, const void* src, void* staging, int
   return SPD_OK;
 }
 
-// Row-major [N][K] -> tile-packed [ceil(N/32)][ceil(K/kstep)][32][kstep], zero padded, where
-// kstep elements are 512 bytes.  16 bytes per thread-iteration.
-__global__ void pack_tiles_kernel(char* dst, const char* src, int N, int K, int esz) {
-  const int kstep = 512 / esz, nsteps = (K + kstep - 1) / kstep, ntiles = (N + 31) >> 5;
-  const size_t total = (size_t)ntiles * nsteps * 1024;   // 16-byte chunks
-  const int epc = 16 / esz;
+// Row-major [N][K] -> the streaming layout of spd_engine.cuh: rows dealt to the G CTAs in
+// quads, each CTA's rows cut into tiles of up to 32 rows, a tile stored step by step
+// ([step][row][512 B]); zero padding for rows >= N and columns >= K; for 2-byte elements the
+// 16-byte chunks of a row are XOR-swizzled with (row-in-tile & 7).
+__global__ void pack_tiles_kernel(char* dst, const char* src, int N, int K, int esz, int G) {
+  const int kstep = 512 / esz, nsteps = (K + kstep - 1) / kstep, epc = 16 / esz;
+  const long long Q = (N + 3) >> 2;
+  const size_t total = (size_t)Q * 4 * nsteps * 32;   // 16-byte chunks
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-    const int c = (int)(i & 31), r = (int)((i >> 5) & 31);
-    const size_t blk = i >> 10;
-    const int st = (int)(blk % nsteps), t = (int)(blk / nsteps);
-    const int row = t * 32 + r, k = st * kstep + c * epc;
+    const int kc = (int)(i & 31);
+    const size_t rs = i >> 5;
+    const int s = (int)(rs % nsteps), n = (int)(rs / nsteps);
+    const long long q = n >> 2;
+    int c = (int)(((q + 1) * G + Q - 1) / Q) - 1;
+    while (c > 0 && Q * c / G > q) --c;
+    while (c < G - 1 && Q * (c + 1) / G <= q) ++c;
+    const int q0 = (int)(Q * c / G), q1 = (int)(Q * (c + 1) / G);
+    const int rl = n - q0 * 4, t = rl >> 5, ri = rl & 31;
+    const int nr = min(32, (q1 - q0) * 4 - t * 32);
+    const int phys = esz == 2 ? (kc ^ (ri & 7)) : kc;
+    const int k = s * kstep + kc * epc;
     uint4 v = make_uint4(0, 0, 0, 0);
-    if (row < N && k < K) v = *reinterpret_cast<const uint4*>(src + ((size_t)row * K + k) * esz);
-    reinterpret_cast<uint4*>(dst)[i] = v;
+    if (n < N && k < K) v = *reinterpret_cast<const uint4*>(src + ((size_t)n * K + k) * esz);
+    const size_t off = (((size_t)(q0 * 4 + t * 32) * nsteps + (size_t)s * nr + ri) * 512) + (size_t)phys * 16;
+    *reinterpret_cast<uint4*>(dst + off) = v;
   }
 }
 
 size_t packed_bytes(int N, int K, size_t esz) {
   const int kstep = (int)(512 / esz);
-  return (size_t)((N + 31) / 32) * ((K + kstep - 1) / kstep) * STAGE_BYTES;
+  return (size_t)((N + 3) / 4) * 4 * ((K + kstep - 1) / kstep) * 512;
 }
 
-spd_status pack_tiles(spd_ctx* ctx, void* dst, const void* src_rowmajor, int N, int K, size_t esz, cudaStream_t st) {
-  pack_tiles_kernel<<<1184, 256, 0, st>>>(static_cast<char*>(dst), static_cast<const char*>(src_rowmajor), N, K, (int)esz);
+spd_status pack_tiles(spd_ctx* ctx, void* dst, const void* src_rowmajor, int N, int K, size_t esz, int G,
+                      cudaStream_t st) {
+  pack_tiles_kernel<<<1184, 256, 0, st>>>(static_cast<char*>(dst), static_cast<const char*>(src_rowmajor), N, K,
+                                          (int)esz, G);
   CU(cudaGetLastError());
   return SPD_OK;
 }
@@ -182,7 +197,7 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
     char* lm = nullptr;
     if ((s = dalloc(ctx, &lm, packed_bytes(V, d, esz)))) return s;
     if ((s = put_rows(ctx, rm, c.tied_embeddings ? w->tok_embed : w->lm_head, staging, V, d, esz, 1, 0, 0))) return s;
-    if ((s = pack_tiles(ctx, lm, rm, V, d, esz, ctx->stream))) return s;
+    if ((s = pack_tiles(ctx, lm, rm, V, d, esz, ctx->n_sm, ctx->stream))) return s;
     md.lm_head = lm;
   }
   float* fn = nullptr;
@@ -195,7 +210,7 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
     char* ad = nullptr;
     if ((s = dalloc(ctx, &ad, packed_bytes(d, adapter_in, esz)))) return s;
     if ((s = put_rows(ctx, rm, w->adapter, staging, d, adapter_in, esz, 1, 0, 0))) return s;
-    if ((s = pack_tiles(ctx, ad, rm, d, adapter_in, esz, ctx->stream))) return s;
+    if ((s = pack_tiles(ctx, ad, rm, d, adapter_in, esz, ctx->n_sm, ctx->stream))) return s;
     mh.adapter = ad;
   }
   std::vector<LayerDev> layers(L);
@@ -214,14 +229,14 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
     if ((s = put_rows(ctx, rm, w->wq[l], staging, d, d, esz, 1, 0, dh))) return s;
     if ((s = put_rows(ctx, rm + (size_t)d * d * esz, w->wk[l], staging, d, d, esz, 1, 0, dh))) return s;
     if ((s = put_rows(ctx, rm + (size_t)2 * d * d * esz, w->wv[l], staging, d, d, esz, 1, 0, 0))) return s;
-    if ((s = pack_tiles(ctx, wqkv, rm, 3 * d, d, esz, ctx->stream))) return s;
+    if ((s = pack_tiles(ctx, wqkv, rm, 3 * d, d, esz, ctx->n_sm, ctx->stream))) return s;
     if ((s = put_rows(ctx, rm, w->wo[l], staging, d, d, esz, 1, 0, 0))) return s;
-    if ((s = pack_tiles(ctx, wo, rm, d, d, esz, ctx->stream))) return s;
+    if ((s = pack_tiles(ctx, wo, rm, d, d, esz, ctx->n_sm, ctx->stream))) return s;
     if ((s = put_rows(ctx, rm, w->w_gate[l], staging, f, d, esz, 2, 0, 0))) return s;
     if ((s = put_rows(ctx, rm, w->w_up[l], staging, f, d, esz, 2, 1, 0))) return s;
-    if ((s = pack_tiles(ctx, wgu, rm, 2 * f, d, esz, ctx->stream))) return s;
+    if ((s = pack_tiles(ctx, wgu, rm, 2 * f, d, esz, ctx->n_sm, ctx->stream))) return s;
     if ((s = put_rows(ctx, rm, w->w_down[l], staging, d, f, esz, 1, 0, 0))) return s;
-    if ((s = pack_tiles(ctx, wd, rm, d, f, esz, ctx->stream))) return s;
+    if ((s = pack_tiles(ctx, wd, rm, d, f, esz, ctx->n_sm, ctx->stream))) return s;
     if (!w->attn_norm[l] || !w->ffn_norm[l]) return fail(ctx, SPD_EINVAL, "missing norm gain");
     CU(cudaMemcpyAsync(an, w->attn_norm[l], d * sizeof(float), cudaMemcpyDefault, ctx->stream));
     CU(cudaMemcpyAsync(fnw, w->ffn_norm[l], d * sizeof(float), cudaMemcpyDefault, ctx->stream));
@@ -299,7 +314,7 @@ spd_status launch_cfg(spd_ctx* ctx, KernelFn fn, int M, int n_sm, int smem_optin
     if (cache_fn[i] == fn) { *lc = cache[i]; return SPD_OK; }
   cudaFuncAttributes fa{};
   CU(cudaFuncGetAttributes(&fa, (const void*)fn));
-  const size_t fixed = CTRL_BYTES + (size_t)M * KC_MAX * sizeof(float);
+  const size_t fixed = FIXED_SMEM + (size_t)x_bytes(M);
   const size_t avail = (size_t)smem_optin - fa.sharedSizeBytes;
   if (avail < fixed + 2 * STAGE_BYTES) return fail(ctx, SPD_ECUDA, "not enough shared memory per block");
   int ns = (int)((avail - fixed) / STAGE_BYTES);
@@ -440,13 +455,6 @@ spd_status spd_create(const spd_weights* target_w, const spd_weights* draft_w, c
   if (!prop.cooperativeLaunch) return bail(fail(ctx, SPD_ECUDA, "cooperative launch not supported"));
   ctx->n_sm = prop.multiProcessorCount;
   ctx->smem_optin = (int)prop.sharedMemPerBlockOptin;
-  // attention scratch must fit the activation region: M*4*(9*dh + Lc) <= M*16384
-  for (const spd_model_cfg* c : {&cfg->target, &cfg->draft}) {
-    const int nsplit = ctx->n_sm / c->n_heads > 0 ? ctx->n_sm / c->n_heads : 1;
-    const int dh = c->d_model / c->n_heads;
-    if ((cfg->max_seq + nsplit - 1) / nsplit + 4 + 9 * dh > KC_MAX)
-      return bail(fail(ctx, SPD_EINVAL, "max_seq too large for the attention scratch"));
-  }
   if (cfg->temperature <= 0.f) ctx->cfg.temperature = 1.0f;
   const size_t esz_t = cfg->target.dtype ? 2 : 4, esz_d = cfg->draft.dtype ? 2 : 4;
   size_t stage_elems = 0;
@@ -635,6 +643,7 @@ spd_status spd_verify(spd_ctx* ctx, int gamma, const int32_t* draft_ids, const f
   a.uniforms = ctx->ubuf + 8;
   a.q_in = draft_probs ? draft_probs : ctx->qbuf;
   a.out_ids = nullptr;
+  a.trace = ctx->trace;
   spd_status s = launch_forward(ctx, gamma + 1, tm.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx));
   if (s) return s;
   ctx->drafted_gamma = -1;
@@ -739,6 +748,25 @@ spd_status spd_get_draft_logits(spd_ctx* ctx, float* logits, int rows) {
   return SPD_OK;
 }
 
+spd_status spd_trace(spd_ctx* ctx, uint64_t* stamps, int cap, int* n) {
+  if (!ctx || !n) return SPD_EINVAL;
+  const int need = 2 + ctx->cfg.target.n_layers * 18 + 16;
+  if (!ctx->trace) {   // first call switches tracing on for later spd_verify calls
+    spd_status s = dalloc(ctx, &ctx->trace, (size_t)need);
+    if (s) return s;
+    ctx->trace_cap = need;
+    *n = 0;
+    return SPD_OK;
+  }
+  const int cnt = 1 + ctx->cfg.target.n_layers * 18 + 7;
+  *n = cnt < cap ? cnt : cap;
+  if (stamps && *n > 0) {
+    CU(cudaMemcpyAsync(stamps, ctx->trace, (size_t)*n * sizeof(uint64_t), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+  }
+  return SPD_OK;
+}
+
 spd_status spd_rollback(spd_ctx* ctx, int n_text, int32_t prev_token, int32_t pending_token) {
   if (!ctx) return SPD_EINVAL;
   if (!ctx->prefilled) return fail(ctx, SPD_ESTATE, "spd_rollback before spd_prefill");
@@ -803,7 +831,7 @@ spd_status spd_skinny_gemm(const float* x, const void* w, int dtype, int M, int 
     if (cudaMalloc(&packed, need) != cudaSuccess) return SPD_ENOMEM;
     packed_cap = need;
   }
-  spd_status s = pack_tiles(ctx, packed, w, N, K, esz, cs);
+  spd_status s = pack_tiles(ctx, packed, w, N, K, esz, n_sm, cs);
   if (s) return s;
   StepArgs a{};
   a.mode = MODE_GEMM;

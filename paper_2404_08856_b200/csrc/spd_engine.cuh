@@ -33,6 +33,12 @@ constexpr int NSTAGE_MAX = 12;
 constexpr int CONSUMER_THREADS = 256;
 constexpr int ENGINE_THREADS = CONSUMER_THREADS + 32;
 constexpr int CTRL_BYTES = 1024;
+constexpr int ZERO_BYTES = 512;         // a row of zeros for out-of-range ldmatrix lanes
+constexpr int RED_BYTES = 8192;         // cross-warp partial sums of one tile
+constexpr int FIXED_SMEM = CTRL_BYTES + ZERO_BYTES + RED_BYTES;
+// activation region: M rows of KC_MAX fp32 (or two bf16 planes), at least 64 KB so that the
+// attention phase can stage its K/V tiles there
+__host__ __device__ constexpr int x_bytes(int M) { return M * KC_MAX * 4 > 65536 ? M * KC_MAX * 4 : 65536; }
 
 enum : int { MODE_VERIFY = 0, MODE_DRAFT = 1, MODE_ROWS = 2, MODE_GEMM = 3 };
 enum : int { PRO_PLAIN = 0, PRO_NORM = 1 };
@@ -90,6 +96,8 @@ struct StepArgs {
   int* out_ids;
   // MODE_GEMM
   const float* gx; const void* gw; float* gy; int gN, gK;
+  // optional phase trace: CTA 0 stores %globaltimer after every phase and every barrier
+  unsigned long long* trace;
 };
 
 struct Ctrl {
@@ -97,9 +105,18 @@ struct Ctrl {
   uint64_t empty[NSTAGE_MAX];
   SampleScratch sc;
   float red[8][MAX_M];
+  float inv[MAX_M];
   float rowmax[MAX_M], rowsum[MAX_M];
   int flag;
+  int trace_n;                      // entries written so far (CTA 0 only)
+  unsigned long long* trace;        // NULL: tracing off
 };
+
+// Trace entry = (%globaltimer ns << 8) | id.  ids: 0 kernel start, 1 activation tile built,
+// 2 last weight stage consumed, 3 phase finished, 4 grid barrier passed.
+__device__ __forceinline__ void trace_stamp(Ctrl* ctl, int id) {
+  if (ctl->trace && threadIdx.x == 0) ctl->trace[ctl->trace_n++] = (globaltimer() << 8) | (unsigned)id;
+}
 static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
 
 struct Gemm {
@@ -132,6 +149,14 @@ __device__ __forceinline__ void chunking(int K, int kstep, int& nchunk, int& kcl
   kcl = (kcl + kstep - 1) / kstep * kstep;
 }
 
+// Rows are dealt to CTAs in quads of 4, as evenly as integers allow: CTA c owns quads
+// [Q*c/G, Q*(c+1)/G).  Streamed bytes per CTA then differ by at most one quad.
+__device__ __forceinline__ void cta_quads(int N, int cta, int G, int& q0, int& q1) {
+  const long long Q = (N + 3) >> 2;
+  q0 = (int)(Q * cta / G);
+  q1 = (int)(Q * (cta + 1) / G);
+}
+
 struct Ring {
   int stage;
   unsigned phase;
@@ -143,39 +168,37 @@ struct Ring {
 
 // ------------------------------------------------------------------------------ producer
 
-// Weights are stored tile-packed: for each tile of 32 rows, for each K step of 512 bytes
-// per row, one contiguous 16 KB block [32 rows][512 B] (rows beyond N and columns beyond K
-// are zero).  One bulk copy moves a whole ring stage.
+// Packed weight layout (built once at set-up): the rows of a CTA are contiguous; they are
+// cut into tiles of up to 32 rows; a tile is stored step by step, one step = 512 bytes of
+// every row of the tile ([row][512 B], so a step of an nr-row tile is one contiguous block
+// of nr*512 bytes = one bulk copy = one ring stage).  For bf16 the 16-byte chunks of a row
+// are XOR-swizzled with (row & 7) so that ldmatrix reads are bank-conflict free.
 template <typename WT>
-__device__ void produce_gemm(const Gemm& g, int cta, int G, int& off, Ring& ring, Ctrl* ctl, char* stages,
-                             uint64_t pol, volatile int* err) {
+__device__ void produce_gemm(const Gemm& g, int cta, int G, Ring& ring, Ctrl* ctl, char* stages, uint64_t pol,
+                             volatile int* err) {
   constexpr int EPL = WTraits<WT>::EPL, KSTEP = 32 * EPL;
   const int lane = threadIdx.x & 31;
-  const int ntiles = (g.N + 31) >> 5;
+  int q0, q1;
+  cta_quads(g.N, cta, G, q0, q1);
+  const int rows = (q1 - q0) * 4;
   const int nsteps = (g.K + KSTEP - 1) / KSTEP;
-  for (int t = (cta - off + G) % G; t < ntiles; t += G) {
-    const char* src = static_cast<const char*>(g.W) + (size_t)t * nsteps * STAGE_BYTES;
+  for (int t = 0; t * 32 < rows; ++t) {
+    const int nr = min(32, rows - t * 32);
+    const char* src = static_cast<const char*>(g.W) + ((size_t)(q0 * 4 + t * 32) * nsteps) * 512;
+    const unsigned bytes = nr * 512;
     for (int s = 0; s < nsteps; ++s) {
       if (!mbar_wait(&ctl->empty[ring.stage], ring.phase ^ 1u, err, DEV_TIMEOUT_EMPTY)) return;
       if (lane == 0) {
-        mbar_arrive_expect_tx(&ctl->full[ring.stage], STAGE_BYTES);
-        bulk_g2s(stages + (size_t)ring.stage * STAGE_BYTES, src + (size_t)s * STAGE_BYTES, STAGE_BYTES,
-                 &ctl->full[ring.stage], pol);
+        mbar_arrive_expect_tx(&ctl->full[ring.stage], bytes);
+        bulk_g2s(stages + (size_t)ring.stage * STAGE_BYTES, src + (size_t)s * bytes, bytes, &ctl->full[ring.stage],
+                 pol);
       }
       ring.advance();
     }
   }
-  off = (off + ntiles) % G;
 }
 
 // ------------------------------------------------------------------------------ X tile
-
-// destination float4 index of natural float4 index k4 inside the activation tile
-template <int EPL>
-__device__ __forceinline__ int perm4(int k4) {
-  if constexpr (EPL == 8) return (k4 & ~63) | ((k4 & 1) << 5) | ((k4 & 63) >> 1);
-  else return k4;
-}
 
 __device__ __forceinline__ float4 cvt4(const __nv_bfloat16* p) {
   const uint2 r = *reinterpret_cast<const uint2*>(p);
@@ -183,26 +206,71 @@ __device__ __forceinline__ float4 cvt4(const __nv_bfloat16* p) {
 }
 __device__ __forceinline__ float4 cvt4(const float* p) { return *reinterpret_cast<const float4*>(p); }
 
-// Load rows [M][klen] (fetch(m, k) -> 4 consecutive values at column k) into X with the
-// lane-friendly permutation, zero padding up to kpad.  With NORM: RMSNorm in place.
-template <int M, int EPL, bool NORM, class Fetch>
-__device__ void load_x(float* X, int kpad, int klen, Fetch fetch, const float* norm_w, float eps, int Ktotal,
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+// Activation rows [M][klen] into shared memory (fetch(m, k) -> 4 consecutive values).
+// With NORM the RMSNorm gain is multiplied in here and 1/rms is left in ctl->inv[m] for
+// the epilogue (a per-row scalar commutes with the contraction).
+//  * fp32 weights: X is fp32 [M][kpad], natural order.
+//  * bf16 weights: X is split into two bf16 planes, x = hi + lo (error 2^-17 |x|), each
+//    [M][kpad] with 16-byte chunks XOR-swizzled by the row, read by ldmatrix as the
+//    B operand of the tensor-core MMA.
+template <int M, typename WT, bool NORM, class Fetch>
+__device__ void load_x(char* X, int kpad, int klen, Fetch fetch, const float* norm_w, float eps, int Ktotal,
                        Ctrl* ctl, float* copy_out, int copy_ld) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int kp4 = kpad >> 2, kl4 = klen >> 2;
-  float4* X4 = reinterpret_cast<float4*>(X);
   float ss[M];
 #pragma unroll
-  for (int m = 0; m < M; ++m) {
-    ss[m] = 0.f;
-    for (int k4 = tid; k4 < kp4; k4 += CONSUMER_THREADS) {
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (k4 < kl4) {
-        v = fetch(m, k4 << 2);
-        if (copy_out) __stcg(reinterpret_cast<float4*>(copy_out + (size_t)m * copy_ld + (k4 << 2)), v);
+  for (int m = 0; m < M; ++m) ss[m] = 0.f;
+  // all loads of a pass are issued before the first is used (KC_MAX / 4 / 256 = 4 per row)
+  constexpr int PER = KC_MAX / 4 / CONSUMER_THREADS;
+  constexpr int MB = M >= 2 ? 2 : 1;   // rows per pass
+#pragma unroll
+  for (int m0 = 0; m0 < M; m0 += MB) {
+    float4 v[MB][PER];
+#pragma unroll
+    for (int mm = 0; mm < MB; ++mm)
+#pragma unroll
+      for (int i = 0; i < PER; ++i) {
+        const int k4 = tid + i * CONSUMER_THREADS;
+        v[mm][i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (m0 + mm < M && k4 < kl4) v[mm][i] = fetch(m0 + mm, k4 << 2);
       }
-      if (NORM) ss[m] += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-      X4[m * kp4 + perm4<EPL>(k4)] = v;
+#pragma unroll
+    for (int mm = 0; mm < MB; ++mm) {
+      const int m = m0 + mm;
+      if (m < M) {
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+          const int k4 = tid + i * CONSUMER_THREADS;
+          if (k4 < kp4) {
+            float4 x = v[mm][i];
+            if (k4 < kl4) {
+              if (copy_out) __stcg(reinterpret_cast<float4*>(copy_out + (size_t)m * copy_ld + (k4 << 2)), x);
+              if (NORM) {
+                ss[m] += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+                const float4 g = *reinterpret_cast<const float4*>(norm_w + (k4 << 2));
+                x.x *= g.x; x.y *= g.y; x.z *= g.z; x.w *= g.w;
+              }
+            }
+            if constexpr (sizeof(WT) == 4) {
+              reinterpret_cast<float4*>(X)[m * kp4 + k4] = x;
+            } else {
+              const uint32_t h0 = pack_bf16(x.x, x.y), h1 = pack_bf16(x.z, x.w);
+              const float rx = x.x - bf16lo(h0), ry = x.y - bf16hi(h0), rz = x.z - bf16lo(h1), rw = x.w - bf16hi(h1);
+              const int chunk = k4 >> 1, phys = (chunk & ~7) | ((chunk ^ m) & 7);
+              const size_t off = (size_t)m * kpad * 2 + phys * 16 + (k4 & 1) * 8;
+              *reinterpret_cast<uint2*>(X + off) = make_uint2(h0, h1);
+              *reinterpret_cast<uint2*>(X + (size_t)M * kpad * 2 + off) =
+                  make_uint2(pack_bf16(rx, ry), pack_bf16(rz, rw));
+            }
+          }
+        }
+      }
     }
   }
   if (NORM) {
@@ -214,18 +282,14 @@ __device__ void load_x(float* X, int kpad, int klen, Fetch fetch, const float* n
       if (lane == 0) ctl->red[warp][m] = s;
     }
     named_sync(1, CONSUMER_THREADS);
-#pragma unroll
-    for (int m = 0; m < M; ++m) {
+    if (tid < M) {
       float s = 0.f;
 #pragma unroll
-      for (int w = 0; w < 8; ++w) s += ctl->red[w][m];
-      const float inv = 1.0f / sqrtf(s / (float)Ktotal + eps);
-      for (int k4 = tid; k4 < kl4; k4 += CONSUMER_THREADS) {
-        const float4 g = *reinterpret_cast<const float4*>(norm_w + (k4 << 2));
-        float4& v = X4[m * kp4 + perm4<EPL>(k4)];
-        v.x = (v.x * inv) * g.x; v.y = (v.y * inv) * g.y; v.z = (v.z * inv) * g.z; v.w = (v.w * inv) * g.w;
-      }
+      for (int w = 0; w < 8; ++w) s += ctl->red[w][tid];
+      ctl->inv[tid] = 1.0f / sqrtf(s / (float)Ktotal + eps);
     }
+  } else if (tid < M) {
+    ctl->inv[tid] = 1.0f;
   }
   named_sync(1, CONSUMER_THREADS);
 }
@@ -275,6 +339,7 @@ struct EpiArgs {
 __device__ __forceinline__ void cache_store(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 __device__ __forceinline__ void cache_store(float* p, float v) { *p = v; }
 
+// (a, b) are the results of rows n and n+1 (n even) for activation row m.
 template <typename WT>
 __device__ __forceinline__ void epilogue_pair(int epi, const EpiArgs& e, int m, int n, int N, float a, float b) {
   if (n >= N) return;
@@ -312,117 +377,179 @@ __device__ __forceinline__ void epilogue_pair(int epi, const EpiArgs& e, int m, 
   }
 }
 
-// ------------------------------------------------------------------------------ consumer
+// ------------------------------------------------------------------------------ consumers
 
-template <int M, typename WT>
-__device__ __forceinline__ void compute_step(const char* stage, const float* X, int kp4, int s, int warp,
-                                             int lane, float2 (&acc)[4][M]) {
-  constexpr int EPL = WTraits<WT>::EPL;
+// fp32 weights: warp w owns rows 4w..4w+3 of the tile, lanes split K, packed fp32 FMAs.
+template <int M>
+__device__ __forceinline__ void compute_step_f32(const char* stage, const float* X, int kp4, int s, int warp,
+                                                 int lane, float2 (&acc)[4][M]) {
   const uint4* wp = reinterpret_cast<const uint4*>(stage + warp * 2048 + lane * 16);
-  if constexpr (EPL == 8) {
-    float2 w[4][4];
+  float2 w[4][2];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const uint4 q = wp[r * 32];
+    w[r][0] = make_float2(__uint_as_float(q.x), __uint_as_float(q.y));
+    w[r][1] = make_float2(__uint_as_float(q.z), __uint_as_float(q.w));
+  }
+  const float4* xp = reinterpret_cast<const float4*>(X) + s * 32 + lane;
+#pragma unroll
+  for (int m = 0; m < M; ++m) {
+    const float4 xa = xp[m * kp4];
+    const float2 x0 = make_float2(xa.x, xa.y), x1 = make_float2(xa.z, xa.w);
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
-      const uint4 q = wp[r * 32];
-      w[r][0] = make_float2(bf16lo(q.x), bf16hi(q.x));
-      w[r][1] = make_float2(bf16lo(q.y), bf16hi(q.y));
-      w[r][2] = make_float2(bf16lo(q.z), bf16hi(q.z));
-      w[r][3] = make_float2(bf16lo(q.w), bf16hi(q.w));
-    }
-    const float4* xp = reinterpret_cast<const float4*>(X) + s * 64 + lane;
-#pragma unroll
-    for (int m = 0; m < M; ++m) {
-      const float4 xa = xp[m * kp4], xb = xp[m * kp4 + 32];
-      const float2 x0 = make_float2(xa.x, xa.y), x1 = make_float2(xa.z, xa.w);
-      const float2 x2 = make_float2(xb.x, xb.y), x3 = make_float2(xb.z, xb.w);
-#pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        float2 a = acc[r][m];
-        a = __ffma2_rn(w[r][0], x0, a);
-        a = __ffma2_rn(w[r][1], x1, a);
-        a = __ffma2_rn(w[r][2], x2, a);
-        a = __ffma2_rn(w[r][3], x3, a);
-        acc[r][m] = a;
-      }
-    }
-  } else {
-    float2 w[4][2];
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      const uint4 q = wp[r * 32];
-      w[r][0] = make_float2(__uint_as_float(q.x), __uint_as_float(q.y));
-      w[r][1] = make_float2(__uint_as_float(q.z), __uint_as_float(q.w));
-    }
-    const float4* xp = reinterpret_cast<const float4*>(X) + s * 32 + lane;
-#pragma unroll
-    for (int m = 0; m < M; ++m) {
-      const float4 xa = xp[m * kp4];
-      const float2 x0 = make_float2(xa.x, xa.y), x1 = make_float2(xa.z, xa.w);
-#pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        float2 a = acc[r][m];
-        a = __ffma2_rn(w[r][0], x0, a);
-        a = __ffma2_rn(w[r][1], x1, a);
-        acc[r][m] = a;
-      }
+      float2 a = acc[r][m];
+      a = __ffma2_rn(w[r][0], x0, a);
+      a = __ffma2_rn(w[r][1], x1, a);
+      acc[r][m] = a;
     }
   }
 }
 
-// xsrc(m, k) fetches 4 activation values; used for every chunk.
+__device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// One K-chunk or whole GEMM for this CTA's rows.  fetch(m, k) reads 4 activation values.
 template <int M, typename WT, class Fetch>
 __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, Fetch fetch, const float* norm_w, float eps,
-                             float* copy_out, int cta, int G, int& off, Ring& ring, Ctrl* ctl, float* X,
-                             const char* stages, volatile int* err) {
+                             float* copy_out, int cta, int G, Ring& ring, Ctrl* ctl, char* X, float* red,
+                             uint32_t zero_addr, const char* stages, volatile int* err) {
   constexpr int EPL = WTraits<WT>::EPL, KSTEP = 32 * EPL;
+  constexpr bool BF = sizeof(WT) == 2;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int ntiles = (g.N + 31) >> 5;
+  int q0, q1;
+  cta_quads(g.N, cta, G, q0, q1);
+  const int rows = (q1 - q0) * 4;
+  if (rows == 0) {
+    if (copy_out) {   // this CTA only has to publish the input rows (residual stream)
+      for (int i = tid; i < M * (g.K >> 2); i += CONSUMER_THREADS) {
+        const int m = i / (g.K >> 2), k = (i - m * (g.K >> 2)) << 2;
+        __stcg(reinterpret_cast<float4*>(copy_out + (size_t)m * g.K + k), fetch(m, k));
+      }
+    }
+    return;
+  }
   int nchunk, kcl;
   chunking(g.K, KSTEP, nchunk, kcl);
   const int kp4 = kcl >> 2;
-  const int t0 = (cta - off + G) % G;
-  off = (off + ntiles) % G;
-  if (t0 >= ntiles) return;
   if (nchunk == 1) {
-    if (g.pro == PRO_NORM) load_x<M, EPL, true>(X, kcl, g.K, fetch, norm_w, eps, g.K, ctl, copy_out, g.K);
-    else load_x<M, EPL, false>(X, kcl, g.K, fetch, nullptr, 0.f, g.K, ctl, copy_out, g.K);
+    if (g.pro == PRO_NORM) load_x<M, WT, true>(X, kcl, g.K, fetch, norm_w, eps, g.K, ctl, copy_out, g.K);
+    else load_x<M, WT, false>(X, kcl, g.K, fetch, nullptr, 0.f, g.K, ctl, copy_out, g.K);
   }
-  for (int t = t0; t < ntiles; t += G) {
-    float2 acc[4][M];
+  trace_stamp(ctl, 1);
+  const uint32_t x_addr = smem_u32(X);
+  for (int t = 0; t * 32 < rows; ++t) {
+    const int nr = min(32, rows - t * 32);
+    const int n0 = q0 * 4 + t * 32;
+    float2 acc[4][M];       // fp32 path
+    float dacc[2][4];       // bf16 path: two 16-row groups x (16 rows x 8 columns) fragment
 #pragma unroll
     for (int r = 0; r < 4; ++r)
 #pragma unroll
       for (int m = 0; m < M; ++m) acc[r][m] = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) dacc[i][j] = 0.f;
     for (int c = 0; c < nchunk; ++c) {
       const int k0 = c * kcl, klen = min(kcl, g.K - k0);
       if (nchunk > 1) {
         named_sync(1, CONSUMER_THREADS);  // everyone is done with the previous chunk
-        load_x<M, EPL, false>(X, kcl, klen, [&](int m, int k) { return fetch(m, k0 + k); }, nullptr, 0.f, g.K, ctl,
-                              nullptr, 0);
+        load_x<M, WT, false>(X, kcl, klen, [&](int m, int k) { return fetch(m, k0 + k); }, nullptr, 0.f, g.K, ctl,
+                             nullptr, 0);
       }
       for (int s = 0; s * KSTEP < klen; ++s) {
         mbar_wait(&ctl->full[ring.stage], ring.phase, err, DEV_TIMEOUT_FULL);
-        compute_step<M, WT>(stages + (size_t)ring.stage * STAGE_BYTES, X, kp4, s, warp, lane, acc);
+        const char* stage = stages + (size_t)ring.stage * STAGE_BYTES;
+        if constexpr (!BF) {
+          if (warp * 4 < nr) compute_step_f32<M>(stage, reinterpret_cast<const float*>(X), kp4, s, warp, lane, acc);
+        } else {
+          // warp w takes the two 16-wide K slices 2w, 2w+1 of this 256-wide step
+          const uint32_t st_addr = smem_u32(stage);
+          const int mat = lane >> 3, rr = lane & 7;
+#pragma unroll
+          for (int kk = 0; kk < 2; ++kk) {
+            const int c16 = (warp * 2 + kk) * 2;     // first 16-byte chunk of the slice (of 32)
+            // B: matrices {hi k0-7, hi k8-15, lo k0-7, lo k8-15}, row = activation row
+            uint32_t b0, b1, b2, b3;
+            {
+              const int chunk = s * 32 + c16 + (mat & 1);
+              const int phys = (chunk & ~7) | ((chunk ^ rr) & 7);
+              const uint32_t addr = rr < M ? x_addr + (uint32_t)(((mat >> 1) * M + rr) * kcl * 2 + phys * 16) : zero_addr;
+              ldsm4(addr, b0, b1, b2, b3);
+            }
+#pragma unroll
+            for (int gi = 0; gi < 2; ++gi) {
+              if (gi * 16 < nr) {
+                // A: matrices {rows 0-7 k0-7, rows 8-15 k0-7, rows 0-7 k8-15, rows 8-15 k8-15}
+                const int r = gi * 16 + (mat & 1) * 8 + rr;
+                const int ch = (c16 + (mat >> 1)) ^ (r & 7);
+                const uint32_t addr = r < nr ? st_addr + (uint32_t)(r * 512 + ch * 16) : zero_addr;
+                uint32_t a0, a1, a2, a3;
+                ldsm4(addr, a0, a1, a2, a3);
+                mma_bf16(dacc[gi], a0, a1, a2, a3, b0, b1);
+                mma_bf16(dacc[gi], a0, a1, a2, a3, b2, b3);
+              }
+            }
+          }
+        }
         __syncwarp();
         if (lane == 0) mbar_arrive(&ctl->empty[ring.stage]);
         ring.advance();
       }
     }
-    // 4*M sums per warp, value index m*4 + r
-    float v[4 * M];
+    if (t * 32 + 32 >= rows) trace_stamp(ctl, 2);
+    if constexpr (!BF) {
+      // 4*M sums per warp, value index m*4 + r
+      float v[4 * M];
 #pragma unroll
-    for (int m = 0; m < M; ++m)
+      for (int m = 0; m < M; ++m)
 #pragma unroll
-      for (int r = 0; r < 4; ++r) v[m * 4 + r] = acc[r][m].x + acc[r][m].y;
-    int base = 0;
-    reduce_rec<4 * M, 16>(v, base, lane);
-    constexpr int FC = final_cnt(4 * M, 16), DUP = dup_mask(4 * M, 16);
-    if ((lane & DUP) == 0) {
+        for (int r = 0; r < 4; ++r) v[m * 4 + r] = acc[r][m].x + acc[r][m].y;
+      int base = 0;
+      reduce_rec<4 * M, 16>(v, base, lane);
+      constexpr int FC = final_cnt(4 * M, 16), DUP = dup_mask(4 * M, 16);
+      if ((lane & DUP) == 0 && warp * 4 < nr) {
 #pragma unroll
-      for (int i = 0; i < FC; i += 2) {
-        const int vi = base + i, m = vi >> 2, r = vi & 3;
-        epilogue_pair<WT>(g.epi, e, m, t * 32 + warp * 4 + r, g.N, v[i], v[i + 1]);
+        for (int i = 0; i < FC; i += 2) {
+          const int vi = base + i, m = vi >> 2, r = vi & 3;
+          const float sc = ctl->inv[m];
+          epilogue_pair<WT>(g.epi, e, m, n0 + warp * 4 + r, g.N, v[i] * sc, v[i + 1] * sc);
+        }
       }
+    } else {
+      // partial sums of the 8 warps (each had its own K slices) meet in shared memory
+      const int gq = lane >> 2, tq = lane & 3;
+#pragma unroll
+      for (int gi = 0; gi < 2; ++gi) {
+        float* rp = red + ((warp * 2 + gi) * 16) * 8;
+        *reinterpret_cast<float2*>(rp + gq * 8 + tq * 2) = make_float2(dacc[gi][0], dacc[gi][1]);
+        *reinterpret_cast<float2*>(rp + (gq + 8) * 8 + tq * 2) = make_float2(dacc[gi][2], dacc[gi][3]);
+      }
+      named_sync(1, CONSUMER_THREADS);
+      {
+        // thread -> (row of the tile, activation row): tid = row*8 + m
+        float v = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) v += red[w * 256 + tid];
+        const int row = tid >> 3, m = tid & 7;
+        const float partner = __shfl_down_sync(0xffffffffu, v, 8);
+        if ((row & 1) == 0 && m < M && row < nr) {
+          const float sc = ctl->inv[m];
+          epilogue_pair<WT>(g.epi, e, m, n0 + row, g.N, v * sc, partner * sc);
+        }
+      }
+      named_sync(1, CONSUMER_THREADS);
     }
   }
 }
@@ -466,24 +593,51 @@ template <> struct CTraits<float> {
   }
 };
 
+__device__ __forceinline__ void cp_async16(void* dst_smem, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+
+template <typename CT>
+__device__ __forceinline__ void frag_from_smem(const char* p, float (&f)[CTraits<CT>::E]) {
+  const uint4 r = *reinterpret_cast<const uint4*>(p);
+  if constexpr (sizeof(CT) == 2) {
+    f[0] = bf16lo(r.x); f[1] = bf16hi(r.x); f[2] = bf16lo(r.y); f[3] = bf16hi(r.y);
+    f[4] = bf16lo(r.z); f[5] = bf16hi(r.z); f[6] = bf16lo(r.w); f[7] = bf16hi(r.w);
+  } else {
+    f[0] = __uint_as_float(r.x); f[1] = __uint_as_float(r.y); f[2] = __uint_as_float(r.z); f[3] = __uint_as_float(r.w);
+  }
+}
+
 // Query row m (position pos0+m) attends cache rows 0..pos0+m.  Work unit = (head, KV
-// split); each unit leaves an unnormalised partial output with its row max and sum; the
-// CTA that finishes a head's last split merges them (no waiting).
+// split).  The unit's K and V rows are brought into shared memory with asynchronous
+// 16-byte copies, all in flight at once (one memory latency), in sub-chunks that fit the
+// scratch region, with a running (online) softmax across sub-chunks.  Each unit leaves an
+// unnormalised partial output with its row max and sum; the CTA that finishes a head's
+// last split merges them (no waiting).
 template <int M, typename CT>
-__device__ void attn_phase(const ModelDev& md, int layer, int pos0, int cta, int G, float* xs, Ctrl* ctl) {
+__device__ void attn_phase(const ModelDev& md, int layer, int pos0, int cta, int G, char* xs, int xbytes, Ctrl* ctl) {
   constexpr int E = CTraits<CT>::E;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int H = md.H, dh = md.dh, d = md.d, nsplit = md.nsplit;
   const int len = pos0 + M;
   const int Lc = (len + nsplit - 1) / nsplit;
-  const int Lcp = (Lc + 3) & ~3;
   const int LPP = dh / E, PPI = 32 / LPP;
   const int sub = lane / LPP, li = lane - sub * LPP;
-  float* qs = xs;                   // [M][dh]
-  float* S = qs + M * dh;           // [M][Lcp]
-  float* red = S + M * Lcp;         // [8][M][dh]
+  const int rowb = dh * (int)sizeof(CT);                     // bytes of one head row
+  // scratch: q [M][dh] | K tile [SC][rowb] (later the cross-warp buffer) | V tile | S [M][SC]
+  int SC = (xbytes - M * dh * 4) / (2 * rowb + M * 4);
+  SC = min(SC & ~7, (Lc + 7) & ~7);
+  float* qs = reinterpret_cast<float*>(xs);
+  char* Kt = xs + M * dh * 4;
+  char* Vt = Kt + (size_t)SC * rowb;
+  float* S = reinterpret_cast<float*>(Vt + (size_t)SC * rowb);
+  float* red = reinterpret_cast<float*>(Kt);                 // [8][M][dh], needs SC*rowb >= 32*M*dh
   const CT* Kl = static_cast<const CT*>(md.kcache) + (size_t)layer * md.max_seq * d;
   const CT* Vl = static_cast<const CT*>(md.vcache) + (size_t)layer * md.max_seq * d;
+  const int cpr = rowb >> 4;                                  // 16-byte copies per row
 
   for (int unit = cta; unit < H * nsplit; unit += G) {
     const int h = unit / nsplit, sp = unit - h * nsplit;
@@ -492,74 +646,99 @@ __device__ void attn_phase(const ModelDev& md, int layer, int pos0, int cta, int
       const int m = i / dh, c = i - m * dh;
       qs[i] = ldcg(md.qbuf + (size_t)m * d + h * dh + c) * md.scale;
     }
+    if (tid < M) { ctl->rowmax[tid] = -INFINITY; ctl->rowsum[tid] = 0.f; }
+    float acc[M][E];
+#pragma unroll
+    for (int m = 0; m < M; ++m)
+#pragma unroll
+      for (int e = 0; e < E; ++e) acc[m][e] = 0.f;
     named_sync(1, CONSUMER_THREADS);
     float qr[M][E];
 #pragma unroll
     for (int m = 0; m < M; ++m)
 #pragma unroll
       for (int e = 0; e < E; ++e) qr[m][e] = qs[m * dh + li * E + e];
-    // scores
-    for (int pb = p0 + warp * PPI; pb < p1; pb += 8 * PPI) {
-      const int p = pb + sub;
-      const bool valid = p < p1;
-      float kf[E];
-#pragma unroll
-      for (int e = 0; e < E; ++e) kf[e] = 0.f;
-      if (valid) CTraits<CT>::load(Kl + (size_t)p * d + h * dh + li * E, kf);
-      float part[M];
-#pragma unroll
-      for (int m = 0; m < M; ++m) {
-        float s = 0.f;
-#pragma unroll
-        for (int e = 0; e < E; ++e) s = fmaf(kf[e], qr[m][e], s);
-        part[m] = s;
+
+    for (int c0 = p0; c0 < p1; c0 += SC) {
+      const int n = min(SC, p1 - c0);
+      for (int i = tid; i < n * cpr; i += CONSUMER_THREADS) {
+        const int r = i / cpr, cc = i - r * cpr;
+        const size_t g = ((size_t)(c0 + r) * d + h * dh) * sizeof(CT) + (size_t)cc * 16;
+        cp_async16(Kt + (size_t)r * rowb + cc * 16, reinterpret_cast<const char*>(Kl) + g);
+        cp_async16(Vt + (size_t)r * rowb + cc * 16, reinterpret_cast<const char*>(Vl) + g);
       }
-      for (int o = LPP >> 1; o; o >>= 1)
+      cp_async_wait_all();
+      named_sync(1, CONSUMER_THREADS);
+      // scores
+      for (int pb = warp * PPI; pb < n; pb += 8 * PPI) {
+        const int r = pb + sub;
+        float kf[E];
 #pragma unroll
-        for (int m = 0; m < M; ++m) part[m] += __shfl_xor_sync(0xffffffffu, part[m], o);
-      if (valid && li == 0) {
-#pragma unroll
-        for (int m = 0; m < M; ++m) S[m * Lcp + (p - p0)] = (p <= pos0 + m) ? part[m] : -INFINITY;
-      }
-    }
-    named_sync(1, CONSUMER_THREADS);
-    // per-row max, exponentials, sum: warp m takes row m
-    if (warp < M) {
-      const int n = p1 - p0;
-      float* row = S + warp * Lcp;
-      float mx = -INFINITY;
-      for (int i = lane; i < n; i += 32) mx = fmaxf(mx, row[i]);
-#pragma unroll
-      for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      float sum = 0.f;
-      for (int i = lane; i < n; i += 32) {
-        const float ex = (mx == -INFINITY) ? 0.f : expf(row[i] - mx);
-        row[i] = ex;
-        sum += ex;
-      }
-#pragma unroll
-      for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-      if (lane == 0) { ctl->rowmax[warp] = mx; ctl->rowsum[warp] = sum; }
-    }
-    named_sync(1, CONSUMER_THREADS);
-    // weighted sum of V rows
-    float acc[M][E];
-#pragma unroll
-    for (int m = 0; m < M; ++m)
-#pragma unroll
-      for (int e = 0; e < E; ++e) acc[m][e] = 0.f;
-    for (int pb = p0 + warp * PPI; pb < p1; pb += 8 * PPI) {
-      const int p = pb + sub;
-      if (p < p1) {
-        float vf[E];
-        CTraits<CT>::load(Vl + (size_t)p * d + h * dh + li * E, vf);
+        for (int e = 0; e < E; ++e) kf[e] = 0.f;
+        if (r < n) frag_from_smem<CT>(Kt + (size_t)r * rowb + li * 16, kf);
+        float part[M];
 #pragma unroll
         for (int m = 0; m < M; ++m) {
-          const float w = S[m * Lcp + (p - p0)];
+          float sacc = 0.f;
 #pragma unroll
-          for (int e = 0; e < E; ++e) acc[m][e] = fmaf(w, vf[e], acc[m][e]);
+          for (int e = 0; e < E; ++e) sacc = fmaf(kf[e], qr[m][e], sacc);
+          part[m] = sacc;
+        }
+        for (int o = LPP >> 1; o; o >>= 1)
+#pragma unroll
+          for (int m = 0; m < M; ++m) part[m] += __shfl_xor_sync(0xffffffffu, part[m], o);
+        if (r < n && li == 0) {
+#pragma unroll
+          for (int m = 0; m < M; ++m) S[m * SC + r] = (c0 + r <= pos0 + m) ? part[m] : -INFINITY;
         }
       }
+      named_sync(1, CONSUMER_THREADS);
+      // online softmax: warp m owns row m
+      if (warp < M) {
+        float* row = S + warp * SC;
+        float mx = -INFINITY;
+        for (int i = lane; i < n; i += 32) mx = fmaxf(mx, row[i]);
+#pragma unroll
+        for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        const float old = ctl->rowmax[warp];
+        const float nm = fmaxf(old, mx);
+        float sum = 0.f;
+        for (int i = lane; i < n; i += 32) {
+          const float ex = (nm == -INFINITY) ? 0.f : expf(row[i] - nm);
+          row[i] = ex;
+          sum += ex;
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (lane == 0) {
+          const float rescale = (old == -INFINITY) ? 0.f : expf(old - nm);
+          ctl->red[0][warp] = rescale;
+          ctl->rowsum[warp] = ctl->rowsum[warp] * rescale + sum;
+          ctl->rowmax[warp] = nm;
+        }
+      }
+      named_sync(1, CONSUMER_THREADS);
+      // rescale what was accumulated so far, add this sub-chunk's weighted V rows
+#pragma unroll
+      for (int m = 0; m < M; ++m) {
+        const float rs = ctl->red[0][m];
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[m][e] *= rs;
+      }
+      for (int pb = warp * PPI; pb < n; pb += 8 * PPI) {
+        const int r = pb + sub;
+        if (r < n) {
+          float vf[E];
+          frag_from_smem<CT>(Vt + (size_t)r * rowb + li * 16, vf);
+#pragma unroll
+          for (int m = 0; m < M; ++m) {
+            const float w = S[m * SC + r];
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[m][e] = fmaf(w, vf[e], acc[m][e]);
+          }
+        }
+      }
+      named_sync(1, CONSUMER_THREADS);   // tiles and S are free again
     }
     for (int o = LPP; o < 32; o <<= 1)
 #pragma unroll

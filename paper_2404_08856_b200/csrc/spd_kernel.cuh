@@ -91,8 +91,10 @@ template <int M, typename WT>
 __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepArgs a) {
   extern __shared__ __align__(1024) char smem[];
   Ctrl* ctl = reinterpret_cast<Ctrl*>(smem);
-  float* X = reinterpret_cast<float*>(smem + CTRL_BYTES);
-  char* stages = smem + CTRL_BYTES + (size_t)M * KC_MAX * sizeof(float);
+  float* red = reinterpret_cast<float*>(smem + CTRL_BYTES + ZERO_BYTES);
+  char* X = smem + FIXED_SMEM;
+  char* stages = smem + FIXED_SMEM + x_bytes(M);
+  const uint32_t zero_addr = smem_u32(smem + CTRL_BYTES);
   const ModelDev& md = *a.md;
   DevState* st = a.st;
   volatile int* err = &st->err;
@@ -105,6 +107,7 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
     }
     mbar_fence_init();
   }
+  if (tid < ZERO_BYTES / 4) reinterpret_cast<uint32_t*>(smem + CTRL_BYTES)[tid] = 0u;
   __syncthreads();
 
   const bool gemm_only = a.mode == MODE_GEMM;
@@ -114,29 +117,31 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
   if (tid >= CONSUMER_THREADS) {
     // ---------------- producer warp: stream every weight tile of this CTA, in order
     Ring ring{0, 0u, a.nstage};
-    int off = 0;
     const uint64_t pol = policy_evict_first();
     if (gemm_only) {
       Gemm g{a.gw, a.gN, a.gK, PRO_PLAIN, EPI_STORE, 0};
-      produce_gemm<WT>(g, cta, G, off, ring, ctl, stages, pol, err);
+      produce_gemm<WT>(g, cta, G, ring, ctl, stages, pol, err);
     } else {
       for (int i = 0; i < n_gemm; ++i) {
         const Gemm g = get_gemm(md, i);
-        produce_gemm<WT>(g, cta, G, off, ring, ctl, stages, pol, err);
+        produce_gemm<WT>(g, cta, G, ring, ctl, stages, pol, err);
       }
     }
   } else {
     // ---------------- compute warps
     Ring ring{0, 0u, a.nstage};
-    int off = 0;
     unsigned bar_target = 0;
+    if (tid == 0) { ctl->trace = cta == 0 ? a.trace : nullptr; ctl->trace_n = 0; }
+    named_sync(1, CONSUMER_THREADS);
+    auto stamp = [&](int id = 3) { trace_stamp(ctl, id); };
+    stamp(0);
     if (gemm_only) {
       Gemm g{a.gw, a.gN, a.gK, PRO_PLAIN, EPI_STORE, 0};
       EpiArgs e{};
       e.out = a.gy; e.ldo = a.gN;
       const float* gx = a.gx; const int K = a.gK;
       consume_gemm<M, WT>(g, e, [&](int m, int k) { return ldcg4(gx + (size_t)m * K + k); }, nullptr, 0.f, nullptr,
-                          cta, G, off, ring, ctl, X, stages, err);
+                          cta, G, ring, ctl, X, red, zero_addr, stages, err);
     } else {
       // positions and token ids of the M rows
       int pos0, pending = 0;
@@ -185,44 +190,44 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
         e.vc = static_cast<WT*>(md.vcache) + (size_t)l * md.max_seq * d;
         if (l == 0)
           consume_gemm<M, WT>(get_gemm(md, 0), e, fetch_in, ly.attn_norm, md.eps, cta == 0 ? md.x : nullptr, cta, G,
-                              off, ring, ctl, X, stages, err);
+                              ring, ctl, X, red, zero_addr, stages, err);
         else
-          consume_gemm<M, WT>(get_gemm(md, l * 4), e, fetch_x, ly.attn_norm, md.eps, nullptr, cta, G, off, ring, ctl,
-                              X, stages, err);
-        grid_barrier(a.bar, bar_target, G, err);
-        attn_phase<M, WT>(md, l, pos0, cta, G, X, ctl);
-        grid_barrier(a.bar, bar_target, G, err);
+          consume_gemm<M, WT>(get_gemm(md, l * 4), e, fetch_x, ly.attn_norm, md.eps, nullptr, cta, G, ring, ctl,
+                              X, red, zero_addr, stages, err);
+        stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
+        attn_phase<M, WT>(md, l, pos0, cta, G, X, x_bytes(M), ctl);
+        stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         // output projection + residual
         e.out = md.x; e.ldo = d;
         consume_gemm<M, WT>(get_gemm(md, l * 4 + 1), e,
                             [&](int m, int k) { return ldcg4(md.attn + (size_t)m * d + k); }, nullptr, 0.f, nullptr,
-                            cta, G, off, ring, ctl, X, stages, err);
-        grid_barrier(a.bar, bar_target, G, err);
+                            cta, G, ring, ctl, X, red, zero_addr, stages, err);
+        stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         // gate/up + SwiGLU
         e.out = md.act; e.ldo = md.f;
-        consume_gemm<M, WT>(get_gemm(md, l * 4 + 2), e, fetch_x, ly.ffn_norm, md.eps, nullptr, cta, G, off, ring, ctl,
-                            X, stages, err);
-        grid_barrier(a.bar, bar_target, G, err);
+        consume_gemm<M, WT>(get_gemm(md, l * 4 + 2), e, fetch_x, ly.ffn_norm, md.eps, nullptr, cta, G, ring, ctl,
+                            X, red, zero_addr, stages, err);
+        stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         // down projection + residual
         e.out = md.x; e.ldo = d;
         const int f = md.f;
         consume_gemm<M, WT>(get_gemm(md, l * 4 + 3), e,
                             [&](int m, int k) { return ldcg4(md.act + (size_t)m * f + k); }, nullptr, 0.f, nullptr,
-                            cta, G, off, ring, ctl, X, stages, err);
-        grid_barrier(a.bar, bar_target, G, err);
+                            cta, G, ring, ctl, X, red, zero_addr, stages, err);
+        stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
       }
       if (want_head) {
         EpiArgs e{};
         e.out = a.logits; e.ldo = md.V;
-        consume_gemm<M, WT>(get_gemm(md, md.L * 4), e, fetch_x, md.final_norm, md.eps, nullptr, cta, G, off, ring, ctl,
-                            X, stages, err);
-        grid_barrier(a.bar, bar_target, G, err);
+        consume_gemm<M, WT>(get_gemm(md, md.L * 4), e, fetch_x, md.final_norm, md.eps, nullptr, cta, G, ring, ctl,
+                            X, red, zero_addr, stages, err);
+        stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         // row statistics over vocabulary slices, then CTA 0 applies the sampling rule
         int r0, nrows;
         if (a.mode == MODE_VERIFY) { r0 = 0; nrows = a.gamma + 1; }
         else { r0 = M - 1; nrows = 1; }
         stats_phase<M>(a.logits, md.V, r0, nrows, a.temperature, cta, G, md.stat_part, ctl);
-        grid_barrier(a.bar, bar_target, G, err);
+        stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         if (cta == 0) {
           const float* u = a.uniforms ? a.uniforms + (a.u_by_block ? (size_t)st->block * a.u_stride : 0) : nullptr;
           if (a.mode == MODE_VERIFY) {
@@ -234,6 +239,7 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
             verify_sample<M>(a, md, st, ctl, G, M - 1, 0, u, ids, 0);
           }
         }
+        stamp();
       }
     }
   }
