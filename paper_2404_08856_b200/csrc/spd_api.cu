@@ -150,6 +150,11 @@ __global__ void pack_tiles_kernel(char* dst, const char* src, int N, int K, int 
   }
 }
 
+__global__ void widen_bf16_kernel(float* dst, const uint16_t* src, size_t n) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = __uint_as_float((uint32_t)src[i] << 16);
+}
+
 size_t packed_bytes(int N, int K, size_t esz) {
   const int kstep = (int)(512 / esz);
   return (size_t)((N + 3) / 4) * 4 * ((K + kstep - 1) / kstep) * 512;
@@ -189,10 +194,20 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
   md.eps = c.rms_eps;
   md.scale = (float)(1.0 / sqrt((double)dh));
   spd_status s;
-  char* embed = nullptr;
-  if ((s = dalloc(ctx, &embed, (size_t)V * d * esz))) return s;
-  if ((s = put_rows(ctx, embed, w->tok_embed, staging, V, d, esz, 1, 0, 0))) return s;
-  md.embed = embed;
+  {  // the embedding table is kept in fp32 so that rows can be bulk-copied as activations
+    float* embed = nullptr;
+    if ((s = dalloc(ctx, &embed, (size_t)V * d))) return s;
+    if (!w->tok_embed) return fail(ctx, SPD_EINVAL, "missing tok_embed");
+    if (esz == 4) {
+      CU(cudaMemcpyAsync(embed, w->tok_embed, (size_t)V * d * 4, cudaMemcpyDefault, ctx->stream));
+    } else {
+      CU(cudaMemcpyAsync(staging, w->tok_embed, (size_t)V * d * 2, cudaMemcpyDefault, ctx->stream));
+      widen_bf16_kernel<<<1184, 256, 0, ctx->stream>>>(embed, reinterpret_cast<const uint16_t*>(staging), (size_t)V * d);
+      CU(cudaGetLastError());
+    }
+    CU(cudaStreamSynchronize(ctx->stream));
+    md.embed = embed;
+  }
   {  // the LM head is streamed tile-packed; a tied head is a packed copy of the table
     char* lm = nullptr;
     if ((s = dalloc(ctx, &lm, packed_bytes(V, d, esz)))) return s;

@@ -38,7 +38,10 @@ constexpr int RED_BYTES = 8192;         // cross-warp partial sums of one tile
 constexpr int FIXED_SMEM = CTRL_BYTES + ZERO_BYTES + RED_BYTES;
 // activation region: M rows of KC_MAX fp32 (or two bf16 planes), at least 64 KB so that the
 // attention phase can stage its K/V tiles there
-__host__ __device__ constexpr int x_bytes(int M) { return M * KC_MAX * 4 > 65536 ? M * KC_MAX * 4 : 65536; }
+constexpr int X_PAD = 8;                // floats of padding per activation row (bank spread)
+__host__ __device__ constexpr int x_bytes(int M) {
+  return M * (KC_MAX + X_PAD) * 4 > 65536 ? M * (KC_MAX + X_PAD) * 4 : 65536;
+}
 
 enum : int { MODE_VERIFY = 0, MODE_DRAFT = 1, MODE_ROWS = 2, MODE_GEMM = 3 };
 enum : int { PRO_PLAIN = 0, PRO_NORM = 1 };
@@ -52,7 +55,7 @@ struct LayerDev {
 struct ModelDev {
   int L, d, H, dh, f, V, max_seq, nsplit;
   float eps, scale;
-  const void* embed;
+  const float* embed;                 // token embedding table, fp32 [V][d]
   const void* lm_head;
   const float* final_norm;
   const float *rope_cos, *rope_sin;   // [max_seq][dh/2]
@@ -103,6 +106,7 @@ struct StepArgs {
 struct Ctrl {
   uint64_t full[NSTAGE_MAX];
   uint64_t empty[NSTAGE_MAX];
+  uint64_t xbar;                    // completion of the activation rows' bulk copies
   SampleScratch sc;
   float red[8][MAX_M];
   float inv[MAX_M];
@@ -200,86 +204,62 @@ __device__ void produce_gemm(const Gemm& g, int cta, int G, Ring& ring, Ctrl* ct
 
 // ------------------------------------------------------------------------------ X tile
 
-__device__ __forceinline__ float4 cvt4(const __nv_bfloat16* p) {
-  const uint2 r = *reinterpret_cast<const uint2*>(p);
-  return make_float4(bf16lo(r.x), bf16hi(r.x), bf16lo(r.y), bf16hi(r.y));
-}
-__device__ __forceinline__ float4 cvt4(const float* p) { return *reinterpret_cast<const float4*>(p); }
-
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-// Activation rows [M][klen] into shared memory (fetch(m, k) -> 4 consecutive values).
-// With NORM the RMSNorm gain is multiplied in here and 1/rms is left in ctl->inv[m] for
-// the epilogue (a per-row scalar commutes with the contraction).
-//  * fp32 weights: X is fp32 [M][kpad], natural order.
-//  * bf16 weights: X is split into two bf16 planes, x = hi + lo (error 2^-17 |x|), each
-//    [M][kpad] with 16-byte chunks XOR-swizzled by the row, read by ldmatrix as the
-//    B operand of the tensor-core MMA.
-template <int M, typename WT, bool NORM, class Fetch>
-__device__ void load_x(char* X, int kpad, int klen, Fetch fetch, const float* norm_w, float eps, int Ktotal,
-                       Ctrl* ctl, float* copy_out, int copy_ld) {
+// Source rows of an activation tile: row m starts at row[m] (fp32, 16-byte aligned).
+template <int M>
+struct XSrc {
+  const float* row[M];
+};
+
+// Activation rows [M][klen] -> shared memory, fp32, row stride kcl + X_PAD floats.  The rows
+// arrive by bulk async copies (one per row, all in flight together); columns klen..kcl are
+// zeroed.  With NORM one pass over the tile accumulates sum(x^2), multiplies the RMSNorm
+// gain in and leaves 1/rms in ctl->inv[m] for the epilogue (a per-row scalar commutes with
+// the contraction).  `copy_out`: also publish the raw rows to global memory.
+template <int M, bool NORM>
+__device__ void load_x(float* X, int kcl, int klen, const XSrc<M>& src, int k0, const float* norm_w, float eps,
+                       int Ktotal, Ctrl* ctl, unsigned& xphase, float* copy_out, volatile int* err) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int kp4 = kpad >> 2, kl4 = klen >> 2;
-  float ss[M];
+  const int xs = kcl + X_PAD;
+  if (tid == 0) {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    mbar_arrive_expect_tx(&ctl->xbar, (unsigned)(M * klen * 4));
 #pragma unroll
-  for (int m = 0; m < M; ++m) ss[m] = 0.f;
-  // all loads of a pass are issued before the first is used (KC_MAX / 4 / 256 = 4 per row)
-  constexpr int PER = KC_MAX / 4 / CONSUMER_THREADS;
-  constexpr int MB = M >= 2 ? 2 : 1;   // rows per pass
-#pragma unroll
-  for (int m0 = 0; m0 < M; m0 += MB) {
-    float4 v[MB][PER];
-#pragma unroll
-    for (int mm = 0; mm < MB; ++mm)
-#pragma unroll
-      for (int i = 0; i < PER; ++i) {
-        const int k4 = tid + i * CONSUMER_THREADS;
-        v[mm][i] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (m0 + mm < M && k4 < kl4) v[mm][i] = fetch(m0 + mm, k4 << 2);
-      }
-#pragma unroll
-    for (int mm = 0; mm < MB; ++mm) {
-      const int m = m0 + mm;
-      if (m < M) {
-#pragma unroll
-        for (int i = 0; i < PER; ++i) {
-          const int k4 = tid + i * CONSUMER_THREADS;
-          if (k4 < kp4) {
-            float4 x = v[mm][i];
-            if (k4 < kl4) {
-              if (copy_out) __stcg(reinterpret_cast<float4*>(copy_out + (size_t)m * copy_ld + (k4 << 2)), x);
-              if (NORM) {
-                ss[m] += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
-                const float4 g = *reinterpret_cast<const float4*>(norm_w + (k4 << 2));
-                x.x *= g.x; x.y *= g.y; x.z *= g.z; x.w *= g.w;
-              }
-            }
-            if constexpr (sizeof(WT) == 4) {
-              reinterpret_cast<float4*>(X)[m * kp4 + k4] = x;
-            } else {
-              const uint32_t h0 = pack_bf16(x.x, x.y), h1 = pack_bf16(x.z, x.w);
-              const float rx = x.x - bf16lo(h0), ry = x.y - bf16hi(h0), rz = x.z - bf16lo(h1), rw = x.w - bf16hi(h1);
-              const int chunk = k4 >> 1, phys = (chunk & ~7) | ((chunk ^ m) & 7);
-              const size_t off = (size_t)m * kpad * 2 + phys * 16 + (k4 & 1) * 8;
-              *reinterpret_cast<uint2*>(X + off) = make_uint2(h0, h1);
-              *reinterpret_cast<uint2*>(X + (size_t)M * kpad * 2 + off) =
-                  make_uint2(pack_bf16(rx, ry), pack_bf16(rz, rw));
-            }
-          }
-        }
-      }
-    }
+    for (int m = 0; m < M; ++m)
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(smem_u32(X + m * xs)), "l"(src.row[m] + k0), "r"((unsigned)(klen * 4)),
+                     "r"(smem_u32(&ctl->xbar))
+                   : "memory");
   }
+  // zero the padding columns meanwhile (weights are zero there, but 0 * garbage may be NaN)
+  const int padq = (kcl - klen) >> 2;
+  for (int i = tid; i < M * padq; i += CONSUMER_THREADS) {
+    const int m = i / padq, c = i - m * padq;
+    reinterpret_cast<float4*>(X + m * xs + klen)[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  mbar_wait(&ctl->xbar, xphase, err, DEV_TIMEOUT_FULL);
+  xphase ^= 1u;
   if (NORM) {
+    const int kl4 = klen >> 2;
 #pragma unroll
     for (int m = 0; m < M; ++m) {
-      float s = ss[m];
+      float ss = 0.f;
+      float4* xr = reinterpret_cast<float4*>(X + m * xs);
+      for (int k4 = tid; k4 < kl4; k4 += CONSUMER_THREADS) {
+        float4 x = xr[k4];
+        if (copy_out) __stcg(reinterpret_cast<float4*>(copy_out + (size_t)m * Ktotal + (k4 << 2)), x);
+        ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+        const float4 g = *reinterpret_cast<const float4*>(norm_w + (k4 << 2));
+        x.x *= g.x; x.y *= g.y; x.z *= g.z; x.w *= g.w;
+        xr[k4] = x;
+      }
 #pragma unroll
-      for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-      if (lane == 0) ctl->red[warp][m] = s;
+      for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      if (lane == 0) ctl->red[warp][m] = ss;
     }
     named_sync(1, CONSUMER_THREADS);
     if (tid < M) {
@@ -381,7 +361,7 @@ __device__ __forceinline__ void epilogue_pair(int epi, const EpiArgs& e, int m, 
 
 // fp32 weights: warp w owns rows 4w..4w+3 of the tile, lanes split K, packed fp32 FMAs.
 template <int M>
-__device__ __forceinline__ void compute_step_f32(const char* stage, const float* X, int kp4, int s, int warp,
+__device__ __forceinline__ void compute_step_f32(const char* stage, const float* X, int xs, int s, int warp,
                                                  int lane, float2 (&acc)[4][M]) {
   const uint4* wp = reinterpret_cast<const uint4*>(stage + warp * 2048 + lane * 16);
   float2 w[4][2];
@@ -391,10 +371,9 @@ __device__ __forceinline__ void compute_step_f32(const char* stage, const float*
     w[r][0] = make_float2(__uint_as_float(q.x), __uint_as_float(q.y));
     w[r][1] = make_float2(__uint_as_float(q.z), __uint_as_float(q.w));
   }
-  const float4* xp = reinterpret_cast<const float4*>(X) + s * 32 + lane;
 #pragma unroll
   for (int m = 0; m < M; ++m) {
-    const float4 xa = xp[m * kp4];
+    const float4 xa = reinterpret_cast<const float4*>(X + m * xs)[s * 32 + lane];
     const float2 x0 = make_float2(xa.x, xa.y), x1 = make_float2(xa.z, xa.w);
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
@@ -419,11 +398,11 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// One K-chunk or whole GEMM for this CTA's rows.  fetch(m, k) reads 4 activation values.
-template <int M, typename WT, class Fetch>
-__device__ void consume_gemm(const Gemm& g, const EpiArgs& e, Fetch fetch, const float* norm_w, float eps,
-                             float* copy_out, int cta, int G, Ring& ring, Ctrl* ctl, char* X, float* red,
-                             uint32_t zero_addr, const char* stages, volatile int* err) {
+// This CTA's share of one projection.  src gives the M activation rows (fp32).
+template <int M, typename WT>
+__device__ void consume_gemm(const Gemm& g, const EpiArgs& e, const XSrc<M>& src, const float* norm_w, float eps,
+                             float* copy_out, int cta, int G, Ring& ring, Ctrl* ctl, float* X, unsigned& xphase,
+                             float* red, uint32_t zero_addr, const char* stages, volatile int* err) {
   constexpr int EPL = WTraits<WT>::EPL, KSTEP = 32 * EPL;
   constexpr bool BF = sizeof(WT) == 2;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -434,20 +413,21 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, Fetch fetch, const
     if (copy_out) {   // this CTA only has to publish the input rows (residual stream)
       for (int i = tid; i < M * (g.K >> 2); i += CONSUMER_THREADS) {
         const int m = i / (g.K >> 2), k = (i - m * (g.K >> 2)) << 2;
-        __stcg(reinterpret_cast<float4*>(copy_out + (size_t)m * g.K + k), fetch(m, k));
+        __stcg(reinterpret_cast<float4*>(copy_out + (size_t)m * g.K + k),
+               __ldcg(reinterpret_cast<const float4*>(src.row[m] + k)));
       }
     }
     return;
   }
   int nchunk, kcl;
   chunking(g.K, KSTEP, nchunk, kcl);
-  const int kp4 = kcl >> 2;
+  const int xs = kcl + X_PAD;
   if (nchunk == 1) {
-    if (g.pro == PRO_NORM) load_x<M, WT, true>(X, kcl, g.K, fetch, norm_w, eps, g.K, ctl, copy_out, g.K);
-    else load_x<M, WT, false>(X, kcl, g.K, fetch, nullptr, 0.f, g.K, ctl, copy_out, g.K);
+    if (g.pro == PRO_NORM) load_x<M, true>(X, kcl, g.K, src, 0, norm_w, eps, g.K, ctl, xphase, copy_out, err);
+    else load_x<M, false>(X, kcl, g.K, src, 0, nullptr, 0.f, g.K, ctl, xphase, nullptr, err);
   }
   trace_stamp(ctl, 1);
-  const uint32_t x_addr = smem_u32(X);
+  const int gq = lane >> 2, tq = lane & 3;
   for (int t = 0; t * 32 < rows; ++t) {
     const int nr = min(32, rows - t * 32);
     const int n0 = q0 * 4 + t * 32;
@@ -461,18 +441,23 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, Fetch fetch, const
     for (int i = 0; i < 2; ++i)
 #pragma unroll
       for (int j = 0; j < 4; ++j) dacc[i][j] = 0.f;
+    // the residual this thread will add in the epilogue is requested now (bf16 path)
+    float resid = 0.f;
+    if (BF && g.epi == EPI_RESID) {
+      const int row = tid >> 3, m = tid & 7;
+      if (m < M && row < nr && n0 + row < g.N) resid = ldcg(e.out + (size_t)m * e.ldo + n0 + row);
+    }
     for (int c = 0; c < nchunk; ++c) {
       const int k0 = c * kcl, klen = min(kcl, g.K - k0);
       if (nchunk > 1) {
         named_sync(1, CONSUMER_THREADS);  // everyone is done with the previous chunk
-        load_x<M, WT, false>(X, kcl, klen, [&](int m, int k) { return fetch(m, k0 + k); }, nullptr, 0.f, g.K, ctl,
-                             nullptr, 0);
+        load_x<M, false>(X, kcl, klen, src, k0, nullptr, 0.f, g.K, ctl, xphase, nullptr, err);
       }
       for (int s = 0; s * KSTEP < klen; ++s) {
         mbar_wait(&ctl->full[ring.stage], ring.phase, err, DEV_TIMEOUT_FULL);
         const char* stage = stages + (size_t)ring.stage * STAGE_BYTES;
         if constexpr (!BF) {
-          if (warp * 4 < nr) compute_step_f32<M>(stage, reinterpret_cast<const float*>(X), kp4, s, warp, lane, acc);
+          if (warp * 4 < nr) compute_step_f32<M>(stage, X, xs, s, warp, lane, acc);
         } else {
           // warp w takes the two 16-wide K slices 2w, 2w+1 of this 256-wide step
           const uint32_t st_addr = smem_u32(stage);
@@ -480,14 +465,16 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, Fetch fetch, const
 #pragma unroll
           for (int kk = 0; kk < 2; ++kk) {
             const int c16 = (warp * 2 + kk) * 2;     // first 16-byte chunk of the slice (of 32)
-            // B: matrices {hi k0-7, hi k8-15, lo k0-7, lo k8-15}, row = activation row
-            uint32_t b0, b1, b2, b3;
-            {
-              const int chunk = s * 32 + c16 + (mat & 1);
-              const int phys = (chunk & ~7) | ((chunk ^ rr) & 7);
-              const uint32_t addr = rr < M ? x_addr + (uint32_t)(((mat >> 1) * M + rr) * kcl * 2 + phys * 16) : zero_addr;
-              ldsm4(addr, b0, b1, b2, b3);
+            // B fragments from the fp32 tile, split on the fly: x = hi + lo (two bf16)
+            float2 xa = make_float2(0.f, 0.f), xb = make_float2(0.f, 0.f);
+            if (gq < M) {
+              const float* xr = X + gq * xs + s * 256 + c16 * 8 + 2 * tq;
+              xa = *reinterpret_cast<const float2*>(xr);
+              xb = *reinterpret_cast<const float2*>(xr + 8);
             }
+            const uint32_t b0 = pack_bf16(xa.x, xa.y), b1 = pack_bf16(xb.x, xb.y);
+            const uint32_t b2 = pack_bf16(xa.x - bf16lo(b0), xa.y - bf16hi(b0));
+            const uint32_t b3 = pack_bf16(xb.x - bf16lo(b1), xb.y - bf16hi(b1));
 #pragma unroll
             for (int gi = 0; gi < 2; ++gi) {
               if (gi * 16 < nr) {
@@ -529,7 +516,6 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, Fetch fetch, const
       }
     } else {
       // partial sums of the 8 warps (each had its own K slices) meet in shared memory
-      const int gq = lane >> 2, tq = lane & 3;
 #pragma unroll
       for (int gi = 0; gi < 2; ++gi) {
         float* rp = red + ((warp * 2 + gi) * 16) * 8;
@@ -543,11 +529,10 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, Fetch fetch, const
 #pragma unroll
         for (int w = 0; w < 8; ++w) v += red[w * 256 + tid];
         const int row = tid >> 3, m = tid & 7;
+        v = v * ctl->inv[m < M ? m : 0] + resid;
         const float partner = __shfl_down_sync(0xffffffffu, v, 8);
-        if ((row & 1) == 0 && m < M && row < nr) {
-          const float sc = ctl->inv[m];
-          epilogue_pair<WT>(g.epi, e, m, n0 + row, g.N, v * sc, partner * sc);
-        }
+        if ((row & 1) == 0 && m < M && row < nr)
+          epilogue_pair<WT>(g.epi == EPI_RESID ? EPI_STORE : g.epi, e, m, n0 + row, g.N, v, partner);
       }
       named_sync(1, CONSUMER_THREADS);
     }

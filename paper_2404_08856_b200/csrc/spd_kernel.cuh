@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
   extern __shared__ __align__(1024) char smem[];
   Ctrl* ctl = reinterpret_cast<Ctrl*>(smem);
   float* red = reinterpret_cast<float*>(smem + CTRL_BYTES + ZERO_BYTES);
-  char* X = smem + FIXED_SMEM;
+  float* X = reinterpret_cast<float*>(smem + FIXED_SMEM);
   char* stages = smem + FIXED_SMEM + x_bytes(M);
   const uint32_t zero_addr = smem_u32(smem + CTRL_BYTES);
   const ModelDev& md = *a.md;
@@ -105,6 +105,7 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
       mbar_init(&ctl->full[i], 1);
       mbar_init(&ctl->empty[i], CONSUMER_THREADS / 32);
     }
+    mbar_init(&ctl->xbar, 1);
     mbar_fence_init();
   }
   if (tid < ZERO_BYTES / 4) reinterpret_cast<uint32_t*>(smem + CTRL_BYTES)[tid] = 0u;
@@ -130,7 +131,7 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
   } else {
     // ---------------- compute warps
     Ring ring{0, 0u, a.nstage};
-    unsigned bar_target = 0;
+    unsigned bar_target = 0, xphase = 0;
     if (tid == 0) { ctl->trace = cta == 0 ? a.trace : nullptr; ctl->trace_n = 0; }
     named_sync(1, CONSUMER_THREADS);
     auto stamp = [&](int id = 3) { trace_stamp(ctl, id); };
@@ -139,9 +140,10 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
       Gemm g{a.gw, a.gN, a.gK, PRO_PLAIN, EPI_STORE, 0};
       EpiArgs e{};
       e.out = a.gy; e.ldo = a.gN;
-      const float* gx = a.gx; const int K = a.gK;
-      consume_gemm<M, WT>(g, e, [&](int m, int k) { return ldcg4(gx + (size_t)m * K + k); }, nullptr, 0.f, nullptr,
-                          cta, G, ring, ctl, X, red, zero_addr, stages, err);
+      XSrc<M> src;
+#pragma unroll
+      for (int m = 0; m < M; ++m) src.row[m] = a.gx + (size_t)m * a.gK;
+      consume_gemm<M, WT>(g, e, src, nullptr, 0.f, nullptr, cta, G, ring, ctl, X, xphase, red, zero_addr, stages, err);
     } else {
       // positions and token ids of the M rows
       int pos0, pending = 0;
@@ -173,13 +175,15 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
           if (tid == 0) atomicCAS(const_cast<int*>(err), DEV_OK, DEV_BAD_TOKEN);
           ids[m] = 0;
         }
-      const WT* table = static_cast<const WT*>(md.embed);
-      const float* rows = a.rows;
-      const int d = md.d;
-      auto fetch_x = [&](int m, int k) { return ldcg4(md.x + (size_t)m * d + k); };
-      auto fetch_in = [&](int m, int k) {
-        return from_ids ? cvt4(table + (size_t)ids[m] * d + k) : ldcg4(rows + (size_t)m * d + k);
-      };
+      const int d = md.d, f = md.f;
+      XSrc<M> src_in, src_x, src_attn, src_act;
+#pragma unroll
+      for (int m = 0; m < M; ++m) {
+        src_in.row[m] = from_ids ? md.embed + (size_t)ids[m] * d : a.rows + (size_t)m * d;
+        src_x.row[m] = md.x + (size_t)m * d;
+        src_attn.row[m] = md.attn + (size_t)m * d;
+        src_act.row[m] = md.act + (size_t)m * f;
+      }
 
       for (int l = 0; l < md.L; ++l) {
         const LayerDev& ly = md.layers[l];
@@ -188,39 +192,33 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
         e.qbuf = md.qbuf; e.d = d; e.dh = md.dh; e.pos0 = pos0; e.cs = md.rope_cos; e.sn = md.rope_sin;
         e.kc = static_cast<WT*>(md.kcache) + (size_t)l * md.max_seq * d;
         e.vc = static_cast<WT*>(md.vcache) + (size_t)l * md.max_seq * d;
-        if (l == 0)
-          consume_gemm<M, WT>(get_gemm(md, 0), e, fetch_in, ly.attn_norm, md.eps, cta == 0 ? md.x : nullptr, cta, G,
-                              ring, ctl, X, red, zero_addr, stages, err);
-        else
-          consume_gemm<M, WT>(get_gemm(md, l * 4), e, fetch_x, ly.attn_norm, md.eps, nullptr, cta, G, ring, ctl,
-                              X, red, zero_addr, stages, err);
+        consume_gemm<M, WT>(get_gemm(md, l * 4), e, l == 0 ? src_in : src_x, ly.attn_norm, md.eps,
+                            (l == 0 && cta == 0) ? md.x : nullptr, cta, G, ring, ctl, X, xphase, red, zero_addr,
+                            stages, err);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
-        attn_phase<M, WT>(md, l, pos0, cta, G, X, x_bytes(M), ctl);
+        attn_phase<M, WT>(md, l, pos0, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         // output projection + residual
         e.out = md.x; e.ldo = d;
-        consume_gemm<M, WT>(get_gemm(md, l * 4 + 1), e,
-                            [&](int m, int k) { return ldcg4(md.attn + (size_t)m * d + k); }, nullptr, 0.f, nullptr,
-                            cta, G, ring, ctl, X, red, zero_addr, stages, err);
+        consume_gemm<M, WT>(get_gemm(md, l * 4 + 1), e, src_attn, nullptr, 0.f, nullptr, cta, G, ring, ctl, X, xphase,
+                            red, zero_addr, stages, err);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         // gate/up + SwiGLU
         e.out = md.act; e.ldo = md.f;
-        consume_gemm<M, WT>(get_gemm(md, l * 4 + 2), e, fetch_x, ly.ffn_norm, md.eps, nullptr, cta, G, ring, ctl,
-                            X, red, zero_addr, stages, err);
+        consume_gemm<M, WT>(get_gemm(md, l * 4 + 2), e, src_x, ly.ffn_norm, md.eps, nullptr, cta, G, ring, ctl, X,
+                            xphase, red, zero_addr, stages, err);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         // down projection + residual
         e.out = md.x; e.ldo = d;
-        const int f = md.f;
-        consume_gemm<M, WT>(get_gemm(md, l * 4 + 3), e,
-                            [&](int m, int k) { return ldcg4(md.act + (size_t)m * f + k); }, nullptr, 0.f, nullptr,
-                            cta, G, ring, ctl, X, red, zero_addr, stages, err);
+        consume_gemm<M, WT>(get_gemm(md, l * 4 + 3), e, src_act, nullptr, 0.f, nullptr, cta, G, ring, ctl, X, xphase,
+                            red, zero_addr, stages, err);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
       }
       if (want_head) {
         EpiArgs e{};
         e.out = a.logits; e.ldo = md.V;
-        consume_gemm<M, WT>(get_gemm(md, md.L * 4), e, fetch_x, md.final_norm, md.eps, nullptr, cta, G, ring, ctl,
-                            X, red, zero_addr, stages, err);
+        consume_gemm<M, WT>(get_gemm(md, md.L * 4), e, src_x, md.final_norm, md.eps, nullptr, cta, G, ring, ctl, X,
+                            xphase, red, zero_addr, stages, err);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         // row statistics over vocabulary slices, then CTA 0 applies the sampling rule
         int r0, nrows;
