@@ -241,25 +241,44 @@ __device__ void load_x(float* X, int kcl, int klen, const XSrc<M>& src, int k0, 
     const int m = i / padq, c = i - m * padq;
     reinterpret_cast<float4*>(X + m * xs + klen)[c] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
+  constexpr int PER = KC_MAX / 4 / CONSUMER_THREADS;
+  const int kl4 = klen >> 2;
+  float4 gain[PER];
+  if (NORM) {   // the gains travel while the rows are still in flight
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+      const int k4 = tid + i * CONSUMER_THREADS;
+      gain[i] = k4 < kl4 ? __ldg(reinterpret_cast<const float4*>(norm_w) + k4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
   mbar_wait(&ctl->xbar, xphase, err, DEV_TIMEOUT_FULL);
   xphase ^= 1u;
   if (NORM) {
-    const int kl4 = klen >> 2;
+    float ss[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) ss[m] = 0.f;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+      const int k4 = tid + i * CONSUMER_THREADS;
+      if (k4 < kl4) {
+        const float4 g = gain[i];
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+          float4* xp = reinterpret_cast<float4*>(X + m * xs) + k4;
+          float4 x = *xp;
+          if (copy_out) __stcg(reinterpret_cast<float4*>(copy_out + (size_t)m * Ktotal + (k4 << 2)), x);
+          ss[m] += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+          x.x *= g.x; x.y *= g.y; x.z *= g.z; x.w *= g.w;
+          *xp = x;
+        }
+      }
+    }
 #pragma unroll
     for (int m = 0; m < M; ++m) {
-      float ss = 0.f;
-      float4* xr = reinterpret_cast<float4*>(X + m * xs);
-      for (int k4 = tid; k4 < kl4; k4 += CONSUMER_THREADS) {
-        float4 x = xr[k4];
-        if (copy_out) __stcg(reinterpret_cast<float4*>(copy_out + (size_t)m * Ktotal + (k4 << 2)), x);
-        ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
-        const float4 g = *reinterpret_cast<const float4*>(norm_w + (k4 << 2));
-        x.x *= g.x; x.y *= g.y; x.z *= g.z; x.w *= g.w;
-        xr[k4] = x;
-      }
+      float v = ss[m];
 #pragma unroll
-      for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-      if (lane == 0) ctl->red[warp][m] = ss;
+      for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0) ctl->red[warp][m] = v;
     }
     named_sync(1, CONSUMER_THREADS);
     if (tid < M) {
@@ -743,6 +762,196 @@ __device__ void attn_phase(const ModelDev& md, int layer, int pos0, int cta, int
 #pragma unroll
       for (int w = 0; w < 8; ++w) s += red[w * M * dh + i];
       stcg(part_out + i, s);
+    }
+    if (tid < M) {
+      float* ml = md.aml + ((size_t)(h * nsplit + sp) * MAX_M + tid) * 2;
+      stcg(ml, ctl->rowmax[tid]);
+      stcg(ml + 1, ctl->rowsum[tid]);
+    }
+    __threadfence();
+    named_sync(1, CONSUMER_THREADS);
+    if (tid == 0) {
+      const unsigned old = atomicAdd(md.head_cnt + h, 1u);
+      ctl->flag = (old == (unsigned)nsplit - 1u);
+      __threadfence();
+    }
+    named_sync(1, CONSUMER_THREADS);
+    if (ctl->flag) {
+      for (int i = tid; i < M * dh; i += CONSUMER_THREADS) {
+        const int m = i / dh, c = i - m * dh;
+        float gmax = -INFINITY;
+        for (int s2 = 0; s2 < nsplit; ++s2)
+          gmax = fmaxf(gmax, ldcg(md.aml + ((size_t)(h * nsplit + s2) * MAX_M + m) * 2));
+        float num = 0.f, den = 0.f;
+        for (int s2 = 0; s2 < nsplit; ++s2) {
+          const float* ml = md.aml + ((size_t)(h * nsplit + s2) * MAX_M + m) * 2;
+          const float mx = ldcg(ml);
+          const float w = (mx == -INFINITY) ? 0.f : expf(mx - gmax);
+          den = fmaf(w, ldcg(ml + 1), den);
+          num = fmaf(w, ldcg(md.apart + ((size_t)(h * nsplit + s2) * MAX_M) * dh + i), num);
+        }
+        stcg(md.attn + (size_t)m * d + h * dh + c, num / den);
+      }
+      if (tid == 0) md.head_cnt[h] = 0u;
+    }
+    named_sync(1, CONSUMER_THREADS);
+  }
+}
+
+__device__ __forceinline__ void ldsm4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+
+// split two fp32 pairs into bf16 hi and lo B-fragment registers
+__device__ __forceinline__ void split_frag(float2 xa, float2 xb, uint32_t& h0, uint32_t& h1, uint32_t& l0, uint32_t& l1) {
+  h0 = pack_bf16(xa.x, xa.y);
+  h1 = pack_bf16(xb.x, xb.y);
+  l0 = pack_bf16(xa.x - bf16lo(h0), xa.y - bf16hi(h0));
+  l1 = pack_bf16(xb.x - bf16lo(h1), xb.y - bf16hi(h1));
+}
+
+// bf16 KV cache: the same unit / split / merge scheme as attn_phase, with both products on
+// the tensor cores.  Scores: D[16 positions x 8 queries] = K tile (A, ldmatrix) x q^T (B,
+// fp32 q split into bf16 hi + lo).  Output: D[16 dims x 8 queries] = V^T (A, transposing
+// ldmatrix) x P^T (B, fp32 probabilities split the same way); warp w owns dims 16w..16w+15,
+// so no cross-warp reduction is needed.  Tile rows are 16-byte-chunk swizzled by position.
+template <int M>
+__device__ void attn_phase_mma(const ModelDev& md, int layer, int pos0, int cta, int G, char* xs, int xbytes,
+                               Ctrl* ctl) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int H = md.H, dh = md.dh, d = md.d, nsplit = md.nsplit;
+  const int len = pos0 + M;
+  const int Lc = (len + nsplit - 1) / nsplit;
+  const int rowb = dh * 2, cpr = rowb >> 4;
+  const int gq = lane >> 2, tq = lane & 3, mat = lane >> 3, rr = lane & 7;
+  const int qst = dh + 8;                                    // padded fp32 row of q
+  // scratch: q [M][dh+8] fp32 | K tile [SC][rowb] | V tile [SC][rowb] | S [M][SC+8] fp32
+  int SC = ((xbytes - M * qst * 4 - M * 8 * 4) / (2 * rowb + M * 4)) & ~15;
+  {  // equal sub-chunks instead of full ones plus a sliver
+    const int nsub = (Lc + SC - 1) / SC;
+    SC = min(SC, (((Lc + nsub - 1) / nsub) + 15) & ~15);
+  }
+  const int sst = SC + 8;
+  float* qs = reinterpret_cast<float*>(xs);
+  char* Kt = xs + M * qst * 4;
+  char* Vt = Kt + (size_t)SC * rowb;
+  float* S = reinterpret_cast<float*>(Vt + (size_t)SC * rowb);
+  const char* Kl = static_cast<const char*>(md.kcache) + (size_t)layer * md.max_seq * d * 2;
+  const char* Vl = static_cast<const char*>(md.vcache) + (size_t)layer * md.max_seq * d * 2;
+  const int nkd = dh >> 4;                                   // 16-wide slices of the head dim
+
+  for (int unit = cta; unit < H * nsplit; unit += G) {
+    const int h = unit / nsplit, sp = unit - h * nsplit;
+    const int p0 = sp * Lc, p1 = min(len, p0 + Lc);
+    // q rows (fp32) and the first sub-chunk of K/V are requested together
+    for (int i = tid; i < M * (dh >> 2); i += CONSUMER_THREADS) {
+      const int m = i / (dh >> 2), c = i - m * (dh >> 2);
+      cp_async16(qs + m * qst + c * 4, md.qbuf + (size_t)m * d + h * dh + c * 4);
+    }
+    if (tid < M) { ctl->rowmax[tid] = -INFINITY; ctl->rowsum[tid] = 0.f; }
+    float oacc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int c0 = p0; c0 < p1; c0 += SC) {
+      const int n = min(SC, p1 - c0), n16 = (n + 15) & ~15;
+      for (int i = tid; i < n16 * cpr; i += CONSUMER_THREADS) {
+        const int r = i / cpr, cc = i - r * cpr;
+        const int dst = r * rowb + ((cc ^ (r & 7)) << 4);
+        if (r < n) {
+          const size_t g = ((size_t)(c0 + r) * d + h * dh) * 2 + (size_t)cc * 16;
+          cp_async16(Kt + dst, Kl + g);
+          cp_async16(Vt + dst, Vl + g);
+        } else {   // rows past the end must not hold NaN patterns: P is 0 there
+          *reinterpret_cast<uint4*>(Vt + dst) = make_uint4(0, 0, 0, 0);
+        }
+      }
+      cp_async_wait_all();
+      named_sync(1, CONSUMER_THREADS);
+      // ---- scores: warp takes 16-position groups
+      for (int gp = warp; gp * 16 < n; gp += 8) {
+        float dsc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int kd = 0; kd < nkd; ++kd) {
+          float2 xa = make_float2(0.f, 0.f), xb = make_float2(0.f, 0.f);
+          if (gq < M) {
+            const float* qr = qs + gq * qst + kd * 16 + 2 * tq;
+            xa = *reinterpret_cast<const float2*>(qr);
+            xb = *reinterpret_cast<const float2*>(qr + 8);
+          }
+          uint32_t b0, b1, b2, b3;
+          split_frag(xa, xb, b0, b1, b2, b3);
+          const int r = gp * 16 + (mat & 1) * 8 + rr;
+          const int ch = (kd * 2 + (mat >> 1)) ^ (r & 7);
+          uint32_t a0, a1, a2, a3;
+          ldsm4(smem_u32(Kt + r * rowb + ch * 16), a0, a1, a2, a3);
+          mma_bf16(dsc, a0, a1, a2, a3, b0, b1);
+          mma_bf16(dsc, a0, a1, a2, a3, b2, b3);
+        }
+        // dsc[0,1]: position gp*16+gq, queries 2tq, 2tq+1; dsc[2,3]: position +8
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int r = gp * 16 + gq + (j >> 1) * 8, q = 2 * tq + (j & 1);
+          const bool vis = r < n && (c0 + r) <= pos0 + q;
+          if (q < M) S[q * sst + r] = vis ? dsc[j] * md.scale : -INFINITY;
+        }
+      }
+      named_sync(1, CONSUMER_THREADS);
+      // ---- online softmax: warp m owns row m
+      if (warp < M) {
+        float* row = S + warp * sst;
+        float mx = -INFINITY;
+        for (int i = lane; i < n16; i += 32) mx = fmaxf(mx, row[i]);
+#pragma unroll
+        for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        const float old = ctl->rowmax[warp];
+        const float nm = fmaxf(old, mx);
+        float sum = 0.f;
+        for (int i = lane; i < n16; i += 32) {
+          const float ex = (nm == -INFINITY) ? 0.f : expf(row[i] - nm);
+          row[i] = ex;
+          sum += ex;
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (lane == 0) {
+          const float rescale = (old == -INFINITY) ? 0.f : expf(old - nm);
+          ctl->red[0][warp] = rescale;
+          ctl->rowsum[warp] = ctl->rowsum[warp] * rescale + sum;
+          ctl->rowmax[warp] = nm;
+        }
+      }
+      named_sync(1, CONSUMER_THREADS);
+      // ---- output: warp w owns dims 16w..16w+15 (warps beyond dh/16 idle)
+      if (warp < nkd) {
+        const float r0s = 2 * tq < M ? ctl->red[0][2 * tq] : 0.f, r1s = 2 * tq + 1 < M ? ctl->red[0][2 * tq + 1] : 0.f;
+        oacc[0] *= r0s; oacc[1] *= r1s; oacc[2] *= r0s; oacc[3] *= r1s;
+        for (int kp = 0; kp * 16 < n; ++kp) {
+          float2 xa = make_float2(0.f, 0.f), xb = make_float2(0.f, 0.f);
+          if (gq < M) {
+            const float* pr = S + gq * sst + kp * 16 + 2 * tq;
+            xa = *reinterpret_cast<const float2*>(pr);
+            xb = *reinterpret_cast<const float2*>(pr + 8);
+          }
+          uint32_t b0, b1, b2, b3;
+          split_frag(xa, xb, b0, b1, b2, b3);
+          // A = V^T: matrices {pos 0-7 x dims 0-7, pos 0-7 x dims 8-15, pos 8-15 x dims 0-7, pos 8-15 x dims 8-15}
+          const int r = kp * 16 + (mat >> 1) * 8 + rr;
+          const int ch = (warp * 2 + (mat & 1)) ^ (r & 7);
+          uint32_t a0, a1, a2, a3;
+          ldsm4_trans(smem_u32(Vt + r * rowb + ch * 16), a0, a1, a2, a3);
+          mma_bf16(oacc, a0, a1, a2, a3, b0, b1);
+          mma_bf16(oacc, a0, a1, a2, a3, b2, b3);
+        }
+      }
+      named_sync(1, CONSUMER_THREADS);   // tiles and S are free again
+    }
+    // oacc[0,1]: dim 16w+gq, queries 2tq, 2tq+1; oacc[2,3]: dim +8
+    float* part_out = md.apart + ((size_t)(h * nsplit + sp) * MAX_M) * dh;
+    if (warp < nkd) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int q = 2 * tq + (j & 1), c = warp * 16 + gq + (j >> 1) * 8;
+        if (q < M) stcg(part_out + q * dh + c, oacc[j]);
+      }
     }
     if (tid < M) {
       float* ml = md.aml + ((size_t)(h * nsplit + sp) * MAX_M + tid) * 2;

@@ -196,7 +196,8 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
                             (l == 0 && cta == 0) ? md.x : nullptr, cta, G, ring, ctl, X, xphase, red, zero_addr,
                             stages, err);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
-        attn_phase<M, WT>(md, l, pos0, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
+        if constexpr (sizeof(WT) == 2) attn_phase_mma<M>(md, l, pos0, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
+        else attn_phase<M, WT>(md, l, pos0, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         // output projection + residual
         e.out = md.x; e.ldo = d;
