@@ -193,6 +193,37 @@ spd_status spd_reject_sample(const float* p, const float* q, const int32_t* ids,
 spd_status spd_skinny_gemm(const float* x, const void* w, int dtype, int M, int N, int K,
                            float* y, void* stream);
 
+/* The same product as spd_skinny_gemm for callers that must not allocate device memory.
+ * (The paper has no counterpart for this entry point; it exists for integration reasons.)
+ *
+ * Who needs it: code that runs where cudaMalloc / cudaFree are off limits -- inside a
+ * host program whose device memory is owned entirely by another allocator (a serving
+ * engine or framework that hands out fixed arenas and forbids side allocations), inside
+ * a latency-critical loop where the implicit device synchronisation of cudaMalloc/cudaFree
+ * is unacceptable, or in a process whose memory budget was fixed at start-up.
+ * spd_skinny_gemm keeps a growing device buffer for the repacked weights and allocates
+ * it on demand; this variant instead uses a fixed scratch array compiled into the library
+ * (SPD_NOALLOC_MAX_PACKED_BYTES plus a 512-byte header).  Every GPU that loads the library
+ * holds that array until the process exits, whether or not this function is ever called.
+ *
+ *   - x, w, y, dtype, M, N, K, stream: exactly as spd_skinny_gemm (the caller still owns
+ *     inputs and outputs).
+ *   - Limit: the repacked weights, ceil(N/4)*4 * ceil(K*esz/512)*512 bytes with esz = 2
+ *     (bf16) or 4 (fp32), must not exceed SPD_NOALLOC_MAX_PACKED_BYTES; otherwise the call
+ *     does nothing, prints one line to stderr and returns SPD_EOVERFLOW.
+ *   - It calls no cudaMalloc, cudaFree or other allocating routine.
+ *   - The first call on each device (with that device current) looks up the device address
+ *     of the scratch array and the device properties; make that first call before starting
+ *     any stream capture.
+ *   - All calls share the one array.  Its contents persist between calls; the words that
+ *     must start at zero are cleared on the stream at the start of every call.  Two calls
+ *     whose GPU work overlaps (different streams, or different host threads) race on it:
+ *     serialise them.
+ * Asynchronous on stream. */
+#define SPD_NOALLOC_MAX_PACKED_BYTES (16u << 20)
+spd_status spd_skinny_gemm_noalloc(const float* x, const void* w, int dtype, int M, int N,
+                                   int K, float* y, void* stream);
+
 /* Bytes that one verify step must move (weights + KV read + KV written) at the current
  * sequence length, the figure the roofline is computed from. */
 spd_status spd_verify_bytes(spd_ctx* ctx, int gamma, double* bytes);

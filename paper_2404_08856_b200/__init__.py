@@ -20,7 +20,8 @@ STATUS_NAMES = ["SPD_OK", "SPD_EINVAL", "SPD_ESTATE", "SPD_ENOMEM", "SPD_EOVERFL
 
 EXPORTS = ["spd_create", "spd_destroy", "spd_last_error", "spd_prefill", "spd_draft", "spd_verify",
            "spd_generate", "spd_get_logits", "spd_get_draft_logits", "spd_rollback", "spd_get_state",
-           "spd_reject_sample", "spd_skinny_gemm", "spd_verify_bytes", "spd_trace"]
+           "spd_reject_sample", "spd_skinny_gemm", "spd_verify_bytes", "spd_trace",
+           "spd_skinny_gemm_noalloc"]
 
 
 class SpdError(RuntimeError):
@@ -230,3 +231,17 @@ def skinny_gemm(x, w, y, dtype: int, stream: int = 0):
     st = lib().spd_skinny_gemm(_ptr(x), _ptr(w), dtype, M, N, K, _ptr(y), C.c_void_p(stream))
     if st != SPD_OK:
         raise SpdError(st, "spd_skinny_gemm")
+
+
+NOALLOC_MAX_PACKED_BYTES = 16 << 20
+
+
+def skinny_gemm_noalloc(x, w, y, dtype: int, stream: int = 0):
+    """y[M,N] = x[M,K] w[N,K]^T on device tensors through the entry point that never
+    allocates device memory (fixed scratch inside the library; see spd_skinny_gemm_noalloc).
+    Raises SpdError(SPD_EOVERFLOW) when the repacked weights exceed the fixed scratch."""
+    M, K = int(x.shape[0]), int(x.shape[1])
+    N = int(w.shape[0])
+    st = lib().spd_skinny_gemm_noalloc(_ptr(x), _ptr(w), dtype, M, N, K, _ptr(y), C.c_void_p(stream))
+    if st != SPD_OK:
+        raise SpdError(st, "spd_skinny_gemm_noalloc")

@@ -427,6 +427,13 @@ spd_status feed_rows(spd_ctx* ctx, ModelHost& mh, const float* rows_dev, const i
 
 }  // namespace
 
+// ------------------------------------------------------------------------------ fixed scratch
+// Scratch of spd_skinny_gemm_noalloc: lives in the library image, so no allocation call is
+// ever made for it.  Layout: [0,256) grid-barrier word, [256,512) kernel status block,
+// [512, ...) the streaming-layout copy of the weight matrix.
+constexpr size_t NOALLOC_HEADER = 512;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_HEADER + SPD_NOALLOC_MAX_PACKED_BYTES];
+
 // ------------------------------------------------------------------------------ C ABI
 
 extern "C" {
@@ -853,6 +860,47 @@ spd_status spd_skinny_gemm(const float* x, const void* w, int dtype, int M, int 
   a.st = st;
   a.gx = x; a.gw = packed; a.gy = y; a.gN = N; a.gK = K;
   return launch_forward(ctx, M, dtype, a, cs, n_sm, smem_optin, bar);
+}
+
+spd_status spd_skinny_gemm_noalloc(const float* x, const void* w, int dtype, int M, int N, int K, float* y,
+                                   void* stream) {
+  if (!x || !w || !y || M < 1 || M > MAX_M || N < 1 || K < 8 || K % 8 || (dtype != 0 && dtype != 1)) return SPD_EINVAL;
+  const size_t esz = dtype == 1 ? 2 : 4;
+  const size_t need = packed_bytes(N, K, esz);
+  if (need > SPD_NOALLOC_MAX_PACKED_BYTES) {
+    fprintf(stderr, "spd_skinny_gemm_noalloc: N=%d K=%d needs %zu bytes of scratch, the fixed scratch holds %zu\n", N,
+            K, need, (size_t)SPD_NOALLOC_MAX_PACKED_BYTES);
+    return SPD_EOVERFLOW;
+  }
+  // Per-device set-up on the first call with that device current: the array's name is only a
+  // host-side handle, the device address comes from the runtime.
+  constexpr int MAX_DEV = 64;
+  static unsigned char* base[MAX_DEV];
+  static int n_sm[MAX_DEV], smem_optin[MAX_DEV];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEV) return SPD_ECUDA;
+  if (!base[dev]) {
+    cudaDeviceProp prop{};
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess || prop.major != 10) return SPD_ECUDA;
+    unsigned char* ptr = nullptr;
+    if (cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return SPD_ECUDA;
+    n_sm[dev] = prop.multiProcessorCount;
+    smem_optin[dev] = (int)prop.sharedMemPerBlockOptin;
+    base[dev] = ptr;
+  }
+  spd_ctx* ctx = nullptr;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  unsigned char* sc = base[dev];
+  // the array keeps whatever the last call left: the barrier word and the status block must
+  // start at zero (launch_forward clears the barrier word, the status block is cleared here)
+  if (cudaMemsetAsync(sc + 256, 0, 256, cs) != cudaSuccess) return SPD_ECUDA;
+  spd_status s = pack_tiles(ctx, sc + NOALLOC_HEADER, w, N, K, esz, n_sm[dev], cs);
+  if (s) return s;
+  StepArgs a{};
+  a.mode = MODE_GEMM;
+  a.st = reinterpret_cast<DevState*>(sc + 256);
+  a.gx = x; a.gw = sc + NOALLOC_HEADER; a.gy = y; a.gN = N; a.gK = K;
+  return launch_forward(ctx, M, dtype, a, cs, n_sm[dev], smem_optin[dev], reinterpret_cast<unsigned*>(sc));
 }
 
 spd_status spd_verify_bytes(spd_ctx* ctx, int gamma, double* bytes) {
