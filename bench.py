@@ -177,7 +177,7 @@ def run_gpu(args, rank, world):
         build.build()
     if dist:
         dist.barrier()
-    wl = synth.llava7b_workload(gamma=GAMMA)
+    wl = synth.llava7b_workload(gamma=GAMMA, n_layers=args.layers, draft_layers=args.draft_layers)
     t0 = time.time()
     tw = synth.Weights(wl.target, wl.seeds["weights"], "target")
     dw = synth.Weights(wl.draft, wl.seeds["weights"], "draft")
@@ -252,7 +252,8 @@ def run_gpu(args, rank, world):
     line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps, "warmup": warm,
             "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32 accumulate on bf16 weights and bf16 KV cache", "data": "synthetic (seeded, random-init)",
-            "config": workload_config(), "clocks": clocks,
+            "config": dict(workload_config(), **({"truncated_layers": args.layers} if args.layers else {})),
+            "clocks": clocks,
             "e2e": {"value": e2e, "unit": "tokens/s", "h2d_bytes_per_step": GAMMA * 4, "d2h_bytes_per_step": (GAMMA + 2) * 4,
                     "ms_per_step": ms_e2e / steps},
             "gpu_launches": (GAMMA + 1) * steps,
@@ -267,7 +268,7 @@ def run_gpu(args, rank, world):
                     "tokens/s is below target-only decoding by construction; the verify step's cost does not "
                     "depend on acceptance",
             "setup_s": {"weights": t_gen, "prefill": t_prefill}}
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and not args.layers:
         tv, td, cores = oracle_block_seconds(2)
         line["cpu_baseline"] = {"value": 1.0 / (tv + GAMMA * td), "unit": "tokens/s", "cores": cores,
                                 "kind": "oracle", "sample": ORACLE_SAMPLE, "verify_s": tv, "draft_step_s": td}
@@ -314,6 +315,9 @@ def main():
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=None,
+                    help="truncate the target to this many layers (profiling captures only; not a bench value)")
+    ap.add_argument("--draft-layers", type=int, default=None)
     ap.add_argument("--micro", default=None, choices=["gemm"], help="time one kernel alone instead of the path")
     ap.add_argument("--M", type=int, default=6)
     ap.add_argument("--N", type=int, default=32768)
