@@ -93,7 +93,9 @@ typedef struct {
   int accepted;        /* draft tokens accepted in total */
   int tokens;          /* tokens written to out_ids */
   float tau;           /* block efficiency: tokens emitted per target call (Sec. 4) */
-  float ms_total, ms_draft, ms_verify; /* device time (CUDA events) */
+  float ms_total;      /* CUDA events around the whole loop */
+  float ms_draft, ms_verify; /* sums of kernel times by the device clock (%globaltimer) */
+  int graph_replays;   /* blocks issued by replaying the captured CUDA graph (0: plain launches) */
 } spd_stats;
 
 /* Validates cfg, copies and repacks the weights, allocates KV caches and workspaces,

@@ -53,7 +53,8 @@ class WeightsC(C.Structure):
 
 class StatsC(C.Structure):
     _fields_ = [("blocks", C.c_int), ("accepted", C.c_int), ("tokens", C.c_int), ("tau", C.c_float),
-                ("ms_total", C.c_float), ("ms_draft", C.c_float), ("ms_verify", C.c_float)]
+                ("ms_total", C.c_float), ("ms_draft", C.c_float), ("ms_verify", C.c_float),
+                ("graph_replays", C.c_int)]
 
 
 _lib = None
@@ -182,7 +183,8 @@ class Spd:
                                            else np.ascontiguousarray(uniforms, dtype=np.float32))
         self._check(lib().spd_generate(self._ctx, n_new, gamma, _ptr(u), _ptr(out), C.byref(st)))
         return out, {"blocks": st.blocks, "accepted": st.accepted, "tokens": st.tokens, "tau": st.tau,
-                     "ms_total": st.ms_total, "ms_draft": st.ms_draft, "ms_verify": st.ms_verify}
+                     "ms_total": st.ms_total, "ms_draft": st.ms_draft, "ms_verify": st.ms_verify,
+                     "graph_replays": st.graph_replays}
 
     def get_logits(self, rows: int) -> np.ndarray:
         out = np.zeros((rows, self.vocab), dtype=np.float32)

@@ -53,6 +53,11 @@ struct spd_ctx {
   int len_ub = 0;               // upper bound of n_text known to the host
   int n_prompt = 0, m_image = 0;
   int last_verify_rows = 0, last_draft_rows = 0;
+  cudaStream_t gs = nullptr;             // internal stream: block graphs are captured and replayed here
+  cudaGraphExec_t block_exec = nullptr;  // one speculative block (gamma draft steps + verify)
+  int block_gamma = -1;
+  const float* block_upool = nullptr;
+  bool graphs_ok = true;
   unsigned long long* trace = nullptr;   // device buffer of phase timestamps (verify steps)
   int trace_cap = 0;
   cudaEvent_t ev[4]{};
@@ -369,9 +374,10 @@ spd_status check_dev_err(spd_ctx* ctx, int e) {
   return fail(ctx, SPD_ETIMEOUT, "device-side wait ran out (code " + std::to_string(e) + ")");
 }
 
-spd_status sync_state(spd_ctx* ctx) {
-  CU(cudaMemcpyAsync(ctx->st_host, ctx->st, sizeof(DevState), cudaMemcpyDeviceToHost, ctx->stream));
-  CU(cudaStreamSynchronize(ctx->stream));
+spd_status sync_state(spd_ctx* ctx, cudaStream_t stream = nullptr, bool use_given = false) {
+  cudaStream_t cs = use_given ? stream : ctx->stream;
+  CU(cudaMemcpyAsync(ctx->st_host, ctx->st, sizeof(DevState), cudaMemcpyDeviceToHost, cs));
+  CU(cudaStreamSynchronize(cs));
   ctx->len_ub = ctx->st_host->n_text;
   const int e = ctx->st_host->err;
   if (e != DEV_OK) {
@@ -443,6 +449,9 @@ const char* spd_last_error(const spd_ctx* ctx) { return ctx ? ctx->err.c_str() :
 void spd_destroy(spd_ctx* ctx) {
   if (!ctx) return;
   cudaStreamSynchronize(ctx->stream);
+  if (ctx->gs) cudaStreamSynchronize(ctx->gs);
+  if (ctx->block_exec) cudaGraphExecDestroy(ctx->block_exec);
+  if (ctx->gs) cudaStreamDestroy(ctx->gs);
   for (void* p : ctx->allocs) cudaFree(p);
   if (ctx->st_host) cudaFreeHost(ctx->st_host);
   for (auto& e : ctx->ev)
@@ -511,6 +520,8 @@ spd_status spd_create(const spd_weights* target_w, const spd_weights* draft_w, c
   if (cudaMallocHost(&ctx->st_host, sizeof(DevState)) != cudaSuccess) return bail(fail(ctx, SPD_ENOMEM, "pinned allocation failed"));
   for (auto& e : ctx->ev)
     if (cudaEventCreate(&e) != cudaSuccess) return bail(fail(ctx, SPD_ECUDA, "event creation failed"));
+  if (cudaStreamCreateWithFlags(&ctx->gs, cudaStreamNonBlocking) != cudaSuccess)
+    return bail(fail(ctx, SPD_ECUDA, "stream creation failed"));
   // every kernel variant that can be launched must fit one CTA per SM
   for (int M = 1; M <= MAX_M; ++M)
     for (int dt : {cfg->target.dtype, cfg->draft.dtype}) {
@@ -706,36 +717,62 @@ spd_status spd_generate(spd_ctx* ctx, int n_new, int gamma, const float* uniform
       ctx->upool_cap = need;
     }
     CU(cudaMemcpyAsync(ctx->upool, uniforms, need * sizeof(float), cudaMemcpyDefault, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));   // the blocks run on the internal stream
   }
   ModelHost &tm = ctx->target, &dm = ctx->draft;
-  float ms_d = 0.f, ms_v = 0.f;
-  CU(cudaEventRecord(ctx->ev[0], ctx->stream));
-  int blocks = 0;
-  while (ctx->st_host->n_emitted < n_new) {
-    CU(cudaEventRecord(ctx->ev[1], ctx->stream));
+  double ms_d = 0.0, ms_v = 0.0;
+  // One block = gamma draft launches + one verify launch.  Everything a block needs (lengths,
+  // tokens, block counter, uniforms) lives on the device, so the same CUDA graph is replayed for
+  // every block; it is captured once per (gamma, uniform pool) on an internal stream.
+  auto enqueue_block = [&](cudaStream_t cs) -> spd_status {
+    spd_status r;
     for (int j = 0; j < gamma; ++j) {
       StepArgs a = base_args(ctx, dm);
       a.mode = MODE_DRAFT; a.gamma = gamma; a.j = j;
       a.uniforms = uniforms ? ctx->upool : nullptr; a.u_stride = us; a.u_by_block = 1;
       a.q_out = ctx->qbuf; a.logits = dm.logits;
-      if ((s = launch_forward(ctx, 2, dm.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx)))) return s;
+      if ((r = launch_forward(ctx, 2, dm.cfg.dtype, a, cs, ctx->n_sm, ctx->smem_optin, next_bar(ctx)))) return r;
     }
-    CU(cudaEventRecord(ctx->ev[2], ctx->stream));
     StepArgs a = base_args(ctx, tm);
     a.mode = MODE_VERIFY; a.gamma = gamma;
     a.uniforms = uniforms ? ctx->upool : nullptr; a.u_stride = us; a.u_by_block = 1;
     a.q_in = ctx->qbuf; a.out_ids = ctx->out_dev;
-    if ((s = launch_forward(ctx, gamma + 1, tm.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx)))) return s;
-    CU(cudaEventRecord(ctx->ev[3], ctx->stream));
-    if ((s = sync_state(ctx))) return s;
-    float t1 = 0.f, t2 = 0.f;
-    cudaEventElapsedTime(&t1, ctx->ev[1], ctx->ev[2]);
-    cudaEventElapsedTime(&t2, ctx->ev[2], ctx->ev[3]);
-    ms_d += t1; ms_v += t2;
+    return launch_forward(ctx, gamma + 1, tm.cfg.dtype, a, cs, ctx->n_sm, ctx->smem_optin, next_bar(ctx));
+  };
+  const float* pool_key = uniforms ? ctx->upool : nullptr;
+  if (ctx->graphs_ok && (!ctx->block_exec || ctx->block_gamma != gamma || ctx->block_upool != pool_key)) {
+    if (ctx->block_exec) { cudaGraphExecDestroy(ctx->block_exec); ctx->block_exec = nullptr; }
+    cudaGraph_t graph = nullptr;
+    bool ok = cudaStreamBeginCapture(ctx->gs, cudaStreamCaptureModeRelaxed) == cudaSuccess;
+    if (ok) {
+      const spd_status r = enqueue_block(ctx->gs);
+      const cudaError_t ce = cudaStreamEndCapture(ctx->gs, &graph);
+      ok = r == SPD_OK && ce == cudaSuccess && graph != nullptr;
+    }
+    if (ok) ok = cudaGraphInstantiate(&ctx->block_exec, graph, 0) == cudaSuccess;
+    if (graph) cudaGraphDestroy(graph);
+    if (!ok) {   // capture not available here: fall back to plain launches for good
+      cudaGetLastError();
+      ctx->block_exec = nullptr;
+      ctx->graphs_ok = false;
+    } else {
+      ctx->block_gamma = gamma;
+      ctx->block_upool = pool_key;
+    }
+  }
+  CU(cudaEventRecord(ctx->ev[0], ctx->gs));
+  int blocks = 0;
+  while (ctx->st_host->n_emitted < n_new) {
+    if (ctx->block_exec) CU(cudaGraphLaunch(ctx->block_exec, ctx->gs));
+    else if ((s = enqueue_block(ctx->gs))) return s;
+    if ((s = sync_state(ctx, ctx->gs, true))) return s;
+    ms_d += gamma ? (double)(ctx->st_host->t_draft1 - ctx->st_host->t_draft0) * 1e-6 : 0.0;
+    ms_v += (double)(ctx->st_host->t_verify1 - ctx->st_host->t_verify0) * 1e-6;
     ++blocks;
     if (blocks > n_new + 1) return fail(ctx, SPD_ECUDA, "block loop made no progress");
   }
-  CU(cudaEventRecord(ctx->ev[3], ctx->stream));
+  CU(cudaEventRecord(ctx->ev[3], ctx->gs));
+  CU(cudaStreamSynchronize(ctx->gs));
   CU(cudaMemcpyAsync(out_ids, ctx->out_dev, n_new * sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream));
   CU(cudaStreamSynchronize(ctx->stream));
   ctx->drafted_gamma = -1;
@@ -748,7 +785,8 @@ spd_status spd_generate(spd_ctx* ctx, int n_new, int gamma, const float* uniform
     const int emitted = ctx->st_host->n_emitted - 1;
     stats->accepted = emitted - blocks;
     stats->tau = blocks ? (float)emitted / blocks : 0.f;
-    stats->ms_total = tot; stats->ms_draft = ms_d; stats->ms_verify = ms_v;
+    stats->ms_total = tot; stats->ms_draft = (float)ms_d; stats->ms_verify = (float)ms_v;
+    stats->graph_replays = ctx->block_exec ? blocks : 0;
   }
   return SPD_OK;
 }

@@ -77,6 +77,8 @@ struct DevState {
   int d_ids[MAX_M];
   int out_cap;
   int pad[3];
+  // %globaltimer (ns) at the start / end of the last draft steps and verify step
+  unsigned long long t_draft0, t_draft1, t_verify0, t_verify1;
 };
 
 struct StepArgs {

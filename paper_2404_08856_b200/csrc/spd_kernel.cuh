@@ -136,6 +136,10 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
     named_sync(1, CONSUMER_THREADS);
     auto stamp = [&](int id = 3) { trace_stamp(ctl, id); };
     stamp(0);
+    if (cta == 0 && tid == 0) {
+      if (a.mode == MODE_VERIFY) st->t_verify0 = globaltimer();
+      else if (a.mode == MODE_DRAFT && a.j == 0) st->t_draft0 = globaltimer();
+    }
     if (gemm_only) {
       Gemm g{a.gw, a.gN, a.gK, PRO_PLAIN, EPI_STORE, 0};
       EpiArgs e{};
@@ -239,6 +243,10 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
           }
         }
         stamp();
+      }
+      if (cta == 0 && tid == 0) {
+        if (a.mode == MODE_VERIFY) st->t_verify1 = globaltimer();
+        else if (a.mode == MODE_DRAFT) st->t_draft1 = globaltimer();
       }
     }
   }

@@ -379,3 +379,19 @@ def test_state_and_overflow_errors():
     bad = synth.ModelCfg(2, 100, 3, 64, 64, dtype="fp32")   # d_model not divisible by heads
     with pytest.raises(spd.SpdError):
         H.make_gpu(synth.Workload("bad", bad, bad, 0, 4, 1, 4), tw, tw, 48)
+
+
+# ------------------------------------------------------------------ full size
+
+@pytest.mark.gpu
+def test_llava7b_full_size_greedy_blocks_match_oracle():
+    """The benchmark's own configuration: all 32 layers of the LLaVA-7B-shaped target and the
+    12-layer draft, 576 image rows + 64 prompt ids, gamma 5, greedy acceptance.  Prefill
+    logits, two drafted blocks and two verify steps against the oracle (about a minute of CPU).
+    Sampling decisions at this depth are covered on the 2-layer truncation: with 32000 nearly
+    equiprobable tokens a draw flips on logit differences far below the 5e-2 allowance."""
+    wl = synth.llava7b_workload(gamma=5)
+    r = lockstep(wl, True, 1.0, 2, 5e-2)
+    assert r["blocks"] >= 1
+    assert r["max_logit_err"] < 2e-2 and r["max_draft_logit_err"] < 2e-2
+    print("full-size max logit error", r["max_logit_err"], "draft", r["max_draft_logit_err"])
