@@ -10,6 +10,7 @@
 
 #include "../../include/spd.h"
 #include "spd_kernel.cuh"
+#include "spd_prefill.cuh"
 
 using namespace spd;
 
@@ -27,6 +28,10 @@ struct ModelHost {
   void* adapter = nullptr;  // draft only [d][adapter_in]
   size_t wbytes = 0;        // bytes of matrices streamed per forward (layers + LM head)
   size_t esz = 2;
+  // bf16 models: plain row-major copies for the tensor-core prefill (natural row order)
+  struct RowMajor { __nv_bfloat16 *wqkv, *wo, *wgu, *wd; const float *attn_norm, *ffn_norm; };
+  std::vector<RowMajor> rm;
+  __nv_bfloat16* adapter_rm = nullptr;
 };
 
 }  // namespace
@@ -53,6 +58,13 @@ struct spd_ctx {
   int len_ub = 0;               // upper bound of n_text known to the host
   int n_prompt = 0, m_image = 0;
   int last_verify_rows = 0, last_draft_rows = 0;
+  // scratch of the tensor-core prefill, grown on demand
+  struct {
+    size_t cap_rows = 0;
+    __nv_bfloat16 *h_hi = nullptr, *h_lo = nullptr, *q_hi = nullptr, *q_lo = nullptr, *vT = nullptr;
+    __nv_bfloat16 *p_hi = nullptr, *p_lo = nullptr;
+    float *wide = nullptr, *S = nullptr;
+  } pf;
   cudaStream_t gs = nullptr;             // internal stream: block graphs are captured and replayed here
   cudaGraphExec_t block_exec = nullptr;  // one speculative block (gamma draft steps + verify)
   int block_gamma = -1;
@@ -262,6 +274,28 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
     CU(cudaMemcpyAsync(fnw, w->ffn_norm[l], d * sizeof(float), cudaMemcpyDefault, ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
     layers[l] = LayerDev{wqkv, wo, wgu, wd, an, fnw};
+    if (esz == 2) {   // natural-order copies for the prefill GEMMs
+      ModelHost::RowMajor r{};
+      if ((s = dalloc(ctx, &r.wqkv, (size_t)3 * d * d))) return s;
+      if ((s = dalloc(ctx, &r.wo, (size_t)d * d))) return s;
+      if ((s = dalloc(ctx, &r.wgu, (size_t)2 * f * d))) return s;
+      if ((s = dalloc(ctx, &r.wd, (size_t)d * f))) return s;
+      CU(cudaMemcpyAsync(r.wqkv, w->wq[l], (size_t)d * d * 2, cudaMemcpyDefault, ctx->stream));
+      CU(cudaMemcpyAsync(r.wqkv + (size_t)d * d, w->wk[l], (size_t)d * d * 2, cudaMemcpyDefault, ctx->stream));
+      CU(cudaMemcpyAsync(r.wqkv + (size_t)2 * d * d, w->wv[l], (size_t)d * d * 2, cudaMemcpyDefault, ctx->stream));
+      CU(cudaMemcpyAsync(r.wo, w->wo[l], (size_t)d * d * 2, cudaMemcpyDefault, ctx->stream));
+      CU(cudaMemcpyAsync(r.wgu, w->w_gate[l], (size_t)f * d * 2, cudaMemcpyDefault, ctx->stream));
+      CU(cudaMemcpyAsync(r.wgu + (size_t)f * d, w->w_up[l], (size_t)f * d * 2, cudaMemcpyDefault, ctx->stream));
+      CU(cudaMemcpyAsync(r.wd, w->w_down[l], (size_t)d * f * 2, cudaMemcpyDefault, ctx->stream));
+      CU(cudaStreamSynchronize(ctx->stream));
+      r.attn_norm = an; r.ffn_norm = fnw;
+      mh.rm.push_back(r);
+    }
+  }
+  if (esz == 2 && adapter_in > 0) {
+    if ((s = dalloc(ctx, &mh.adapter_rm, (size_t)d * adapter_in))) return s;
+    CU(cudaMemcpyAsync(mh.adapter_rm, w->adapter, (size_t)d * adapter_in * 2, cudaMemcpyDefault, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
   }
   if ((s = dalloc(ctx, &mh.layers_dev, (size_t)L))) return s;
   CU(cudaMemcpyAsync(mh.layers_dev, layers.data(), L * sizeof(LayerDev), cudaMemcpyHostToDevice, ctx->stream));
@@ -431,6 +465,153 @@ spd_status feed_rows(spd_ctx* ctx, ModelHost& mh, const float* rows_dev, const i
   return SPD_OK;
 }
 
+
+// ---- tensor-core prefill (bf16 models)
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q{};
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 operand view [batch][rows][inner] with byte strides; box = 64 inner x 128 rows x 1.
+spd_status make_map(spd_ctx* ctx, CUtensorMap* m, const void* ptr, int inner, int rows, int batch, size_t row_stride,
+                    size_t batch_stride) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return fail(ctx, SPD_ECUDA, "cuTensorMapEncodeTiled not available");
+  const cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)batch};
+  const cuuint64_t strides[2] = {(cuuint64_t)row_stride, (cuuint64_t)batch_stride};
+  const cuuint32_t box[3] = {(cuuint32_t)TC_BK, (cuuint32_t)TC_BM, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(ctx, SPD_ECUDA, "cuTensorMapEncodeTiled failed (" + std::to_string((int)r) + ")");
+  return SPD_OK;
+}
+
+struct Operand { const void* ptr; int inner, rows, batch; size_t row_stride, batch_stride; };
+
+spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const Operand& b, TcArgs args) {
+  CUtensorMap ma, ml, mb;
+  spd_status s;
+  if ((s = make_map(ctx, &ma, a_hi.ptr, a_hi.inner, a_hi.rows, a_hi.batch, a_hi.row_stride, a_hi.batch_stride))) return s;
+  if ((s = make_map(ctx, &ml, a_lo.ptr, a_lo.inner, a_lo.rows, a_lo.batch, a_lo.row_stride, a_lo.batch_stride))) return s;
+  if ((s = make_map(ctx, &mb, b.ptr, b.inner, b.rows, b.batch, b.row_stride, b.batch_stride))) return s;
+  static bool attr_set = false;
+  if (!attr_set) {
+    CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
+    attr_set = true;
+  }
+  args.split = 1;
+  args.err = &ctx->st->err;
+  dim3 grid((args.N + TC_BN - 1) / TC_BN, (args.M + TC_BM - 1) / TC_BM, a_hi.batch);
+  tc_gemm_kernel<<<grid, 128, TC_SMEM_BYTES, ctx->stream>>>(ma, ml, mb, args);
+  CU(cudaGetLastError());
+  return SPD_OK;
+}
+
+__global__ void gather_rows_kernel(const int* ids, const float* table, float* out, int n, int d) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < (size_t)n * (d >> 2);
+       i += (size_t)gridDim.x * blockDim.x) {
+    const int r = (int)(i / (d >> 2)), c = (int)(i - (size_t)r * (d >> 2));
+    reinterpret_cast<float4*>(out + (size_t)r * d)[c] = reinterpret_cast<const float4*>(table + (size_t)ids[r] * d)[c];
+  }
+}
+
+spd_status prefill_scratch(spd_ctx* ctx, int R) {
+  if ((size_t)R <= ctx->pf.cap_rows) return SPD_OK;
+  const spd_model_cfg &t = ctx->cfg.target, &d = ctx->cfg.draft;
+  const size_t dm = t.d_model > d.d_model ? t.d_model : d.d_model;
+  const size_t fm = t.d_ffn > d.d_ffn ? t.d_ffn : d.d_ffn;
+  const size_t hm = t.n_heads > d.n_heads ? t.n_heads : d.n_heads;
+  const size_t ad = ctx->cfg.draft_adapter_in;
+  size_t kin = dm > fm ? dm : fm;
+  if (ad > kin) kin = ad;
+  const size_t wide = 3 * dm > 2 * fm ? 3 * dm : 2 * fm;
+  const size_t rp = ((size_t)R + 63) / 64 * 64;
+  spd_status s;   // earlier buffers stay in the context's allocation list until spd_destroy
+  if ((s = dalloc(ctx, &ctx->pf.h_hi, rp * kin))) return s;
+  if ((s = dalloc(ctx, &ctx->pf.h_lo, rp * kin))) return s;
+  if ((s = dalloc(ctx, &ctx->pf.q_hi, rp * dm))) return s;
+  if ((s = dalloc(ctx, &ctx->pf.q_lo, rp * dm))) return s;
+  if ((s = dalloc(ctx, &ctx->pf.vT, dm * rp))) return s;
+  if ((s = dalloc(ctx, &ctx->pf.wide, rp * wide))) return s;
+  if ((s = dalloc(ctx, &ctx->pf.S, hm * rp * rp))) return s;
+  if ((s = dalloc(ctx, &ctx->pf.p_hi, hm * rp * rp))) return s;
+  if ((s = dalloc(ctx, &ctx->pf.p_lo, hm * rp * rp))) return s;
+  ctx->pf.cap_rows = rp;
+  return SPD_OK;
+}
+
+// Dense forward of rows X [R][d] (fp32, device; positions 0..R-1) through every layer of a
+// bf16 model: fills the KV cache rows 0..R-1 and leaves the final residual stream in X.
+spd_status prefill_tc(spd_ctx* ctx, ModelHost& mh, float* X, int R) {
+  const int d = mh.cfg.d_model, f = mh.cfg.d_ffn, H = mh.cfg.n_heads, dh = d / H, L = mh.cfg.n_layers;
+  const int rp = (R + 63) / 64 * 64;
+  spd_status s;
+  if ((s = prefill_scratch(ctx, R))) return s;
+  auto& pf = ctx->pf;
+  cudaStream_t cs = ctx->stream;
+  CU(cudaMemsetAsync(pf.vT, 0, (size_t)d * rp * 2, cs));
+  const size_t max_seq = ctx->cfg.max_seq;
+  for (int l = 0; l < L; ++l) {
+    const ModelHost::RowMajor& w = mh.rm[l];
+    __nv_bfloat16* kc = static_cast<__nv_bfloat16*>(mh.md.kcache) + (size_t)l * max_seq * d;
+    __nv_bfloat16* vc = static_cast<__nv_bfloat16*>(mh.md.vcache) + (size_t)l * max_seq * d;
+    TcArgs a{};
+    // attention block
+    rms_split_kernel<<<R, 256, 0, cs>>>(X, w.attn_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
+    a = TcArgs{}; a.M = R; a.N = 3 * d; a.K = d; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = pf.wide; a.ldo = 3 * d;
+    if ((s = tc_gemm(ctx, {pf.h_hi, d, R, 1, (size_t)d * 2, (size_t)R * d * 2}, {pf.h_lo, d, R, 1, (size_t)d * 2, (size_t)R * d * 2},
+                     {w.wqkv, d, 3 * d, 1, (size_t)d * 2, (size_t)3 * d * d * 2}, a))) return s;
+    rope_kv_kernel<<<592, 256, 0, cs>>>(pf.wide, R, d, dh, 0, mh.md.rope_cos, mh.md.rope_sin, pf.q_hi, pf.q_lo, kc, vc,
+                                        pf.vT, rp);
+    a = TcArgs{}; a.M = R; a.N = R; a.K = dh; a.mode = TC_OUT_F32; a.alpha = mh.md.scale; a.out_f32 = pf.S; a.ldo = rp;
+    a.out_batch = (long long)R * rp;
+    if ((s = tc_gemm(ctx, {pf.q_hi, dh, R, H, (size_t)d * 2, (size_t)dh * 2}, {pf.q_lo, dh, R, H, (size_t)d * 2, (size_t)dh * 2},
+                     {kc, dh, R, H, (size_t)d * 2, (size_t)dh * 2}, a))) return s;
+    softmax_causal_split_kernel<<<H * R, 256, 0, cs>>>(pf.S, R, rp, pf.p_hi, pf.p_lo);
+    a = TcArgs{}; a.M = R; a.N = dh; a.K = rp; a.mode = TC_OUT_SPLIT; a.alpha = 1.f; a.out_hi = pf.h_hi; a.out_lo = pf.h_lo;
+    a.ldo = d; a.out_batch = dh;
+    if ((s = tc_gemm(ctx, {pf.p_hi, rp, R, H, (size_t)rp * 2, (size_t)R * rp * 2}, {pf.p_lo, rp, R, H, (size_t)rp * 2, (size_t)R * rp * 2},
+                     {pf.vT, rp, dh, H, (size_t)rp * 2, (size_t)dh * rp * 2}, a))) return s;
+    a = TcArgs{}; a.M = R; a.N = d; a.K = d; a.mode = TC_OUT_F32_ADD; a.alpha = 1.f; a.out_f32 = X; a.ldo = d;
+    if ((s = tc_gemm(ctx, {pf.h_hi, d, R, 1, (size_t)d * 2, (size_t)R * d * 2}, {pf.h_lo, d, R, 1, (size_t)d * 2, (size_t)R * d * 2},
+                     {w.wo, d, d, 1, (size_t)d * 2, (size_t)d * d * 2}, a))) return s;
+    // feed-forward block
+    rms_split_kernel<<<R, 256, 0, cs>>>(X, w.ffn_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
+    a = TcArgs{}; a.M = R; a.N = 2 * f; a.K = d; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = pf.wide; a.ldo = 2 * f;
+    if ((s = tc_gemm(ctx, {pf.h_hi, d, R, 1, (size_t)d * 2, (size_t)R * d * 2}, {pf.h_lo, d, R, 1, (size_t)d * 2, (size_t)R * d * 2},
+                     {w.wgu, d, 2 * f, 1, (size_t)d * 2, (size_t)2 * f * d * 2}, a))) return s;
+    swiglu_split_kernel<<<592, 256, 0, cs>>>(pf.wide, R, f, pf.h_hi, pf.h_lo);
+    a = TcArgs{}; a.M = R; a.N = d; a.K = f; a.mode = TC_OUT_F32_ADD; a.alpha = 1.f; a.out_f32 = X; a.ldo = d;
+    if ((s = tc_gemm(ctx, {pf.h_hi, f, R, 1, (size_t)f * 2, (size_t)R * f * 2}, {pf.h_lo, f, R, 1, (size_t)f * 2, (size_t)R * f * 2},
+                     {w.wd, f, d, 1, (size_t)f * 2, (size_t)d * f * 2}, a))) return s;
+    CU(cudaGetLastError());
+  }
+  return SPD_OK;
+}
+
+bool use_tc_prefill(const ModelHost& mh) {
+  static int forced = -1;   // SPD_PREFILL=rows keeps the 8-row kernel (comparison runs)
+  if (forced < 0) {
+    const char* e = getenv("SPD_PREFILL");
+    forced = (e && !strcmp(e, "rows")) ? 1 : 0;
+  }
+  return !forced && mh.cfg.dtype == 1;
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------------------ fixed scratch
@@ -561,8 +742,43 @@ spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m, const flo
   CU(cudaMemcpyAsync(&ctx->st->out_cap, &ctx->out_cap, sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
   CU(cudaStreamSynchronize(ctx->stream));
   spd_status s;
-  // ---- draft: [adapter(features) ; embed(prompt)] or embed(prompt) alone (Sec. 3)
   ModelHost& dm = ctx->draft;
+  ModelHost& tm = ctx->target;
+  bool moved_logits = false;
+  if (use_tc_prefill(dm) && use_tc_prefill(tm)) {
+    // ---- dense tensor-core pass over all rows of each model
+    const int dd = dm.cfg.d_model, dt = tm.cfg.d_model;
+    const int Rd = (ad > 0 ? m : 0) + n, Rt = m + n;
+    if ((s = prefill_scratch(ctx, Rt > Rd ? Rt : Rd))) return s;
+    float* X = ctx->rows;
+    dm.pos_base = 0;
+    if (ad > 0) {   // draft rows [H W_a^T ; embed(prompt)]
+      CU(cudaMemcpyAsync(ctx->pf.wide, draft_image_feats, (size_t)m * ad * sizeof(float), cudaMemcpyDefault, ctx->stream));
+      split_rows_kernel<<<592, 256, 0, ctx->stream>>>(ctx->pf.wide, ctx->pf.h_hi, ctx->pf.h_lo, (size_t)m * ad);
+      TcArgs a{}; a.M = m; a.N = dd; a.K = ad; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = X; a.ldo = dd;
+      if ((s = tc_gemm(ctx, {ctx->pf.h_hi, ad, m, 1, (size_t)ad * 2, (size_t)m * ad * 2},
+                       {ctx->pf.h_lo, ad, m, 1, (size_t)ad * 2, (size_t)m * ad * 2},
+                       {dm.adapter_rm, ad, dd, 1, (size_t)ad * 2, (size_t)dd * ad * 2}, a))) return s;
+      dm.pos_base = m;
+    }
+    gather_rows_kernel<<<592, 256, 0, ctx->stream>>>(ctx->ids_dev, dm.md.embed, X + (size_t)dm.pos_base * dd, n, dd);
+    if ((s = prefill_tc(ctx, dm, X, Rd))) return s;
+    // ---- target rows [V_1..V_m ; embed(prompt)] (Eq. 1); last row -> first generated token
+    tm.pos_base = m;
+    if (m > 0)
+      CU(cudaMemcpyAsync(X, image_embeds, (size_t)m * dt * sizeof(float), cudaMemcpyDefault, ctx->stream));
+    gather_rows_kernel<<<592, 256, 0, ctx->stream>>>(ctx->ids_dev, tm.md.embed, X + (size_t)m * dt, n, dt);
+    if ((s = prefill_tc(ctx, tm, X, Rt))) return s;
+    CU(cudaMemcpyAsync(tm.md.x, X + (size_t)(Rt - 1) * dt, dt * sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));
+    StepArgs a = base_args(ctx, tm);
+    a.mode = MODE_ROWS; a.skip_layers = 1; a.want_sample = 1;
+    a.rows = tm.md.x; a.rows_pos0 = Rt - 1;
+    a.init_n_text = n; a.init_prev = last_id;
+    a.uniforms = ctx->ubuf + 8; a.out_ids = ctx->out_dev;
+    if ((s = launch_forward(ctx, 1, tm.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx)))) return s;
+    moved_logits = true;
+  } else {
+  // ---- draft: [adapter(features) ; embed(prompt)] or embed(prompt) alone (Sec. 3)
   dm.pos_base = 0;
   if (ad > 0) {
     const int dd = dm.cfg.d_model;
@@ -586,19 +802,19 @@ spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m, const flo
   }
   if ((s = feed_rows(ctx, dm, nullptr, ctx->ids_dev, 0, n, dm.pos_base, false, 0, 0))) return s;
   // ---- target: [V_1..V_m ; embed(prompt)] (Eq. 1); last row -> first generated token
-  ModelHost& tm = ctx->target;
   tm.pos_base = m;
   if (m > 0) {
     CU(cudaMemcpyAsync(ctx->rows, image_embeds, (size_t)m * tm.cfg.d_model * sizeof(float), cudaMemcpyDefault, ctx->stream));
     if ((s = feed_rows(ctx, tm, ctx->rows, nullptr, 0, m, 0, false, 0, 0))) return s;
   }
   if ((s = feed_rows(ctx, tm, nullptr, ctx->ids_dev, 0, n, m, true, n, last_id))) return s;
+  }
   ctx->prefilled = true;
   ctx->drafted_gamma = -1;
   ctx->n_prompt = n; ctx->m_image = m;
   ctx->last_verify_rows = 1; ctx->last_draft_rows = 0;
   // the sampled row was row (chunk rows - 1) of the last chunk: move it to row 0
-  {
+  if (!moved_logits) {
     const int lastM = (n % MAX_M) ? (n % MAX_M) : MAX_M;
     if (lastM > 1)
       CU(cudaMemcpyAsync(tm.logits, tm.logits + (size_t)(lastM - 1) * V, V * sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));

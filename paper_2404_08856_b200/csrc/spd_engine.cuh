@@ -91,6 +91,7 @@ struct StepArgs {
   const float* rows;      // fp32 [M, d] input rows (already embeddings), or NULL: ids
   const int* row_ids;     // MODE_ROWS with rows == NULL: token ids [M]
   int rows_pos0, want_sample, init_n_text, init_prev;
+  int skip_layers;        // MODE_ROWS: rows are the final residual stream (md.x); run the LM head only
   // uniforms
   const float* uniforms;
   int u_stride, u_by_block;

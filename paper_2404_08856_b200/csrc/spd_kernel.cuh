@@ -113,7 +113,10 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
 
   const bool gemm_only = a.mode == MODE_GEMM;
   const bool want_head = gemm_only ? false : (a.mode != MODE_ROWS || a.want_sample);
-  const int n_gemm = gemm_only ? 1 : md.L * 4 + (want_head ? 1 : 0);
+  const bool head_only = !gemm_only && a.mode == MODE_ROWS && a.skip_layers;
+  const int n_layers_run = head_only ? 0 : (gemm_only ? 0 : md.L);
+  const int g_first = head_only ? md.L * 4 : 0;
+  const int n_gemm = gemm_only ? 1 : n_layers_run * 4 + (want_head ? 1 : 0);
 
   if (tid >= CONSUMER_THREADS) {
     // ---------------- producer warp: stream every weight tile of this CTA, in order
@@ -124,7 +127,7 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
       produce_gemm<WT>(g, cta, G, ring, ctl, stages, pol, err);
     } else {
       for (int i = 0; i < n_gemm; ++i) {
-        const Gemm g = get_gemm(md, i);
+        const Gemm g = get_gemm(md, g_first + i);
         produce_gemm<WT>(g, cta, G, ring, ctl, stages, pol, err);
       }
     }
@@ -189,7 +192,7 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
         src_act.row[m] = md.act + (size_t)m * f;
       }
 
-      for (int l = 0; l < md.L; ++l) {
+      for (int l = 0; l < n_layers_run; ++l) {
         const LayerDev& ly = md.layers[l];
         EpiArgs e{};
         // QKV + RoPE + KV append

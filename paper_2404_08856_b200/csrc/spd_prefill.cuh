@@ -1,0 +1,281 @@
+// Prefill (Eq. 1: the target reads [V_1..V_m ; embed(X_1..X_n)] in one pass): dense GEMMs on
+// the 5th-generation tensor cores.  C[M,N] = A[M,K] B[N,K]^T with both operands K-major bf16:
+// tiles arrive by TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a ring of
+// shared-memory stages, one thread issues tcgen05.mma (128x128x16 per instruction) with the
+// accumulator in tensor memory, and the epilogue reads it back with tcgen05.ld.
+//
+// Precision: B operands are exact bf16 data (weights, cached K and V).  The A operand
+// (activations, probabilities) is fp32 upstream and is fed as TWO bf16 matrices hi + lo
+// (x = hi + lo up to 2^-17 |x|), i.e. the K loop runs twice.  Prefill results therefore
+// match an fp32 reference to ~1e-5 relative, like the M <= 8 path, at twice the tensor work.
+#pragma once
+#include <cuda.h>
+
+#include "spd_device.cuh"
+
+namespace spd {
+
+constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64, TC_STAGES = 6;
+constexpr int TC_A_BYTES = TC_BM * TC_BK * 2, TC_B_BYTES = TC_BN * TC_BK * 2;
+constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;                  // 32 KB
+constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 + 256;   // + alignment slack + barriers
+constexpr int TC_TMEM_COLS = 128;
+
+enum : int { TC_OUT_F32 = 0, TC_OUT_F32_ADD = 1, TC_OUT_SPLIT = 2 };
+
+struct TcArgs {
+  int M, N, K;              // A rows, B rows (= output columns), inner dimension
+  int split;                // 1: A is given as hi and lo maps
+  int mode;                 // TC_OUT_*
+  float alpha;              // result scale
+  float* out_f32;
+  __nv_bfloat16 *out_hi, *out_lo;
+  long long ldo, out_batch; // output row stride and per-batch offset, in elements
+  int* err;                 // sticky error word (DEV_TIMEOUT_*)
+};
+
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
+      : "memory");
+}
+
+// K-major operand tile in shared memory, rows of 128 bytes, 128-byte swizzle: 8-row groups are
+// 1024 bytes apart (stride byte offset), leading byte offset 1 (unused for swizzled K-major).
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// kind::f16: D = fp32, A = B = bf16, both K-major, M = 128, N = 128.
+constexpr uint32_t TC_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TC_BN >> 3) << 17) |
+                              ((uint32_t)(TC_BM >> 4) << 24);
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(TC_IDESC), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// grid = (N tiles, M tiles, batch); 128 threads: thread 0 feeds TMA, thread 32 issues the MMAs,
+// all four warps read the accumulator back (warp w owns TMEM lanes 32w..32w+31 = tile rows).
+__global__ void __launch_bounds__(128, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
+               const __grid_constant__ CUtensorMap map_b, const TcArgs a) {
+  extern __shared__ uint8_t tc_smem_raw[];
+  uint8_t* stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full = reinterpret_cast<uint64_t*>(stages + TC_STAGES * TC_STAGE_BYTES);
+  uint64_t* empty = full + TC_STAGES;
+  uint64_t* accum = empty + TC_STAGES;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
+  volatile int* err = a.err;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tile_n = blockIdx.x, tile_m = blockIdx.y, z = blockIdx.z;
+
+  if (tid == 0) {
+    for (int i = 0; i < TC_STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    mbar_init(accum, 1);
+    mbar_fence_init();
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(TC_TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int k_blocks = (a.K + TC_BK - 1) / TC_BK;
+  const int total = k_blocks * (a.split ? 2 : 1);
+  if (tid == 0) {
+    // ---- TMA producer
+    for (int it = 0; it < total; ++it) {
+      const int s = it % TC_STAGES;
+      const unsigned ph = (it / TC_STAGES) & 1;
+      if (!mbar_wait(&empty[s], ph ^ 1u, err, DEV_TIMEOUT_EMPTY)) break;
+      mbar_arrive_expect_tx(&full[s], TC_STAGE_BYTES);
+      const int kb = it % k_blocks;
+      const CUtensorMap* ma = (it >= k_blocks) ? &map_a_lo : &map_a_hi;
+      tma_load_3d(stages + s * TC_STAGE_BYTES, ma, kb * TC_BK, tile_m * TC_BM, z, &full[s]);
+      tma_load_3d(stages + s * TC_STAGE_BYTES + TC_A_BYTES, &map_b, kb * TC_BK, tile_n * TC_BN, z, &full[s]);
+    }
+  } else if (tid == 32) {
+    // ---- MMA issuer
+    bool ok = true;
+    for (int it = 0; it < total && ok; ++it) {
+      const int s = it % TC_STAGES;
+      const unsigned ph = (it / TC_STAGES) & 1;
+      ok = mbar_wait(&full[s], ph, err, DEV_TIMEOUT_FULL);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint64_t ad = umma_desc(smem_u32(stages + s * TC_STAGE_BYTES));
+      const uint64_t bd = umma_desc(smem_u32(stages + s * TC_STAGE_BYTES + TC_A_BYTES));
+#pragma unroll
+      for (int k = 0; k < TC_BK / 16; ++k)   // 32 bytes further along K inside the swizzle atom
+        umma_bf16(tmem_base, ad + 2 * k, bd + 2 * k, (it > 0 || k > 0) ? 1u : 0u);
+      umma_commit(&empty[s]);   // the stage is free once these MMAs have read it
+    }
+    umma_commit(accum);         // arrives when every MMA above has completed
+  }
+  __syncwarp();
+  // ---- epilogue
+  const bool done = mbar_wait(accum, 0u, err, DEV_TIMEOUT_FULL);
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const int row = tile_m * TC_BM + warp * 32 + lane;
+  if (done) {
+#pragma unroll 1
+    for (int c0 = 0; c0 < TC_BN; c0 += 32) {
+      uint32_t v[32];
+      tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+      const int col0 = tile_n * TC_BN + c0;
+      if (row < a.M && col0 < a.N) {
+        const long long off = (long long)z * a.out_batch + (long long)row * a.ldo + col0;
+        const int nv = min(32, a.N - col0);
+        if (a.mode == TC_OUT_SPLIT) {
+          for (int j = 0; j < nv; j += 2) {
+            const float x0 = __uint_as_float(v[j]) * a.alpha, x1 = (j + 1 < nv) ? __uint_as_float(v[j + 1]) * a.alpha : 0.f;
+            const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
+            a.out_hi[off + j] = h0;
+            a.out_lo[off + j] = __float2bfloat16_rn(x0 - __bfloat162float(h0));
+            if (j + 1 < nv) {
+              a.out_hi[off + j + 1] = h1;
+              a.out_lo[off + j + 1] = __float2bfloat16_rn(x1 - __bfloat162float(h1));
+            }
+          }
+        } else if (a.mode == TC_OUT_F32_ADD) {
+          for (int j = 0; j < nv; ++j) a.out_f32[off + j] += __uint_as_float(v[j]) * a.alpha;
+        } else {
+          for (int j = 0; j < nv; ++j) a.out_f32[off + j] = __uint_as_float(v[j]) * a.alpha;
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) {
+    if (!done) for (int i = 0; i < 200; ++i) __nanosleep(1000);   // let copies in flight land
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------ elementwise
+
+__device__ __forceinline__ void store_split(__nv_bfloat16* hi, __nv_bfloat16* lo, size_t i, float x) {
+  const __nv_bfloat16 h = __float2bfloat16_rn(x);
+  hi[i] = h;
+  lo[i] = __float2bfloat16_rn(x - __bfloat162float(h));
+}
+
+// fp32 [R][K] -> hi/lo bf16 [R][K]
+__global__ void split_rows_kernel(const float* x, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t n) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    store_split(hi, lo, i, x[i]);
+}
+
+// RMSNorm of each row (one block per row), output split into hi/lo bf16.
+__global__ void __launch_bounds__(256) rms_split_kernel(const float* x, const float* gain, float eps, int d,
+                                                        __nv_bfloat16* hi, __nv_bfloat16* lo) {
+  __shared__ float red[8];
+  const float* row = x + (size_t)blockIdx.x * d;
+  float ss = 0.f;
+  for (int k = threadIdx.x; k < d; k += 256) ss += row[k] * row[k];
+#pragma unroll
+  for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) tot += red[w];
+  const float inv = 1.0f / sqrtf(tot / (float)d + eps);
+  for (int k = threadIdx.x; k < d; k += 256)
+    store_split(hi, lo, (size_t)blockIdx.x * d + k, (row[k] * inv) * gain[k]);
+}
+
+// qkv fp32 [R][3d] (natural row order) -> rotary on q and k (pairs (i, i + dh/2)), q split into
+// hi/lo [R][d], k and v appended to the cache rows pos0.., v also transposed to vT [H][dh][rpad].
+__global__ void rope_kv_kernel(const float* qkv, int R, int d, int dh, int pos0, const float* cs, const float* sn,
+                               __nv_bfloat16* q_hi, __nv_bfloat16* q_lo, __nv_bfloat16* kc, __nv_bfloat16* vc,
+                               __nv_bfloat16* vT, int rpad) {
+  const int half = dh >> 1, pairs = d >> 1;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < (size_t)R * pairs;
+       i += (size_t)gridDim.x * blockDim.x) {
+    const int r = (int)(i / pairs), p = (int)(i - (size_t)r * pairs);
+    const int h = p / half, j = p - h * half;
+    const int c0 = h * dh + j, c1 = c0 + half;
+    const float* row = qkv + (size_t)r * 3 * d;
+    const float c = cs[(size_t)(pos0 + r) * half + j], s = sn[(size_t)(pos0 + r) * half + j];
+    const float qa = row[c0], qb = row[c1], ka = row[d + c0], kb = row[d + c1];
+    store_split(q_hi, q_lo, (size_t)r * d + c0, qa * c - qb * s);
+    store_split(q_hi, q_lo, (size_t)r * d + c1, qb * c + qa * s);
+    kc[(size_t)(pos0 + r) * d + c0] = __float2bfloat16_rn(ka * c - kb * s);
+    kc[(size_t)(pos0 + r) * d + c1] = __float2bfloat16_rn(kb * c + ka * s);
+    const __nv_bfloat16 v0 = __float2bfloat16_rn(row[2 * d + c0]), v1 = __float2bfloat16_rn(row[2 * d + c1]);
+    vc[(size_t)(pos0 + r) * d + c0] = v0;
+    vc[(size_t)(pos0 + r) * d + c1] = v1;
+    vT[((size_t)h * dh + j) * rpad + r] = v0;
+    vT[((size_t)h * dh + j + half) * rpad + r] = v1;
+  }
+}
+
+// Causal softmax of each score row (one block per (head, row)): row r sees columns 0..r.
+// Output probabilities split into hi/lo bf16 [H][R][rpad], zero beyond the diagonal.
+__global__ void __launch_bounds__(256) softmax_causal_split_kernel(const float* S, int R, int rpad,
+                                                                   __nv_bfloat16* hi, __nv_bfloat16* lo) {
+  __shared__ float red[8];
+  const size_t base = (size_t)blockIdx.x * rpad;
+  const int r = blockIdx.x % R, n = r + 1;
+  const float* row = S + base;
+  float mx = -INFINITY;
+  for (int k = threadIdx.x; k < n; k += 256) mx = fmaxf(mx, row[k]);
+#pragma unroll
+  for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  mx = red[0];
+#pragma unroll
+  for (int w = 1; w < 8; ++w) mx = fmaxf(mx, red[w]);
+  __syncthreads();
+  float sum = 0.f;
+  for (int k = threadIdx.x; k < n; k += 256) sum += expf(row[k] - mx);
+#pragma unroll
+  for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) tot += red[w];
+  for (int k = threadIdx.x; k < rpad; k += 256)
+    store_split(hi, lo, base + k, k < n ? expf(row[k] - mx) / tot : 0.f);
+}
+
+// gu fp32 [R][2f] = [gate | up] -> silu(gate) * up, split into hi/lo [R][f]
+__global__ void swiglu_split_kernel(const float* gu, int R, int f, __nv_bfloat16* hi, __nv_bfloat16* lo) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < (size_t)R * f; i += (size_t)gridDim.x * blockDim.x) {
+    const size_t r = i / f, c = i - r * f;
+    const float g = gu[r * 2 * f + c], u = gu[r * 2 * f + f + c];
+    store_split(hi, lo, i, (g / (1.0f + expf(-g))) * u);
+  }
+}
+
+}  // namespace spd

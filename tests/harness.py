@@ -97,3 +97,17 @@ class SafeUniforms:
 def top2_gap(row):
     part = np.partition(row, -2)[-2:]
     return float(part[1] - part[0])
+
+
+def token_within_cdf_band(w, u, token, delta):
+    """True if `token` is what the inverse-CDF draw returns for SOME weight vector within a
+    relative perturbation `delta` of w: the threshold u*Z lies within delta*Z of the token's
+    CDF interval.  Used where logits differ by a known bound eps between the two sides: a
+    logit error eps changes every probability by at most a factor e^(2 eps), hence any prefix
+    sum of the CDF by at most about 2 eps."""
+    W = S.fixed_point(w).astype(np.float64)
+    cum = np.cumsum(W)
+    Z = cum[-1]
+    t = Z * float(u)
+    lo = cum[token - 1] if token else 0.0
+    return lo - delta * Z <= t <= cum[token] + delta * Z
