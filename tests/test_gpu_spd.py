@@ -412,3 +412,14 @@ def test_llava7b_full_size_greedy_blocks_match_oracle():
     assert r["blocks"] >= 1
     assert r["max_logit_err"] < 4e-2 and r["max_draft_logit_err"] < 2e-2
     print("full-size max logit error", r["max_logit_err"], "draft", r["max_draft_logit_err"])
+
+
+@pytest.mark.gpu
+def test_llava7b_shaped_two_layer_with_draft_adapter():
+    """The draft with an image adapter at LLaVA-7B shapes: 576 features of width 1024 projected
+    by one linear layer to the draft's width and prepended to its input (bf16, tensor-core
+    prefill path)."""
+    wl = synth.llava7b_workload(gamma=5, n_layers=2, draft_layers=2, adapter=True)
+    r = lockstep(wl, False, 1.0, 2, 5e-2)
+    print("adapter report", r)
+    assert r["blocks"] >= 1 and r["max_draft_logit_err"] < 1e-2
