@@ -205,6 +205,13 @@ __device__ void produce_gemm(const Gemm& g, int cta, int G, Ring& ring, Ctrl* ct
   }
 }
 
+// KV splits actually used for a context of `len` rows: short contexts are not cut up (a head
+// is then finished by one CTA and needs no merge), long ones use up to md.nsplit CTAs per head.
+__device__ __forceinline__ int eff_nsplit(const ModelDev& md, int len) {
+  const int want = (len + 175) / 176;
+  return want < 1 ? 1 : (want < md.nsplit ? want : md.nsplit);
+}
+
 // ------------------------------------------------------------------------------ X tile
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
@@ -567,8 +574,7 @@ __device__ __forceinline__ void grid_barrier(unsigned* counter, unsigned& target
   named_sync(1, CONSUMER_THREADS);
   if (threadIdx.x == 0) {
     target += G;
-    __threadfence();
-    atomicAdd(counter, 1u);
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(counter) : "memory");
     unsigned it = 0;
     while (ld_acquire(counter) < target) {
       if (++it > SPIN_LIMIT_GRID || ((it & 255u) == 0 && *err != DEV_OK)) {
@@ -628,8 +634,9 @@ template <int M, typename CT>
 __device__ void attn_phase(const ModelDev& md, int layer, int pos0, int cta, int G, char* xs, int xbytes, Ctrl* ctl) {
   constexpr int E = CTraits<CT>::E;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int H = md.H, dh = md.dh, d = md.d, nsplit = md.nsplit;
+  const int H = md.H, dh = md.dh, d = md.d;
   const int len = pos0 + M;
+  const int nsplit = eff_nsplit(md, len);
   const int Lc = (len + nsplit - 1) / nsplit;
   const int LPP = dh / E, PPI = 32 / LPP;
   const int sub = lane / LPP, li = lane - sub * LPP;
@@ -759,6 +766,17 @@ __device__ void attn_phase(const ModelDev& md, int layer, int pos0, int cta, int
         for (int e = 0; e < E; ++e) red[(warp * M + m) * dh + li * E + e] = acc[m][e];
     }
     named_sync(1, CONSUMER_THREADS);
+    if (nsplit == 1) {   // the whole context was here: normalise and finish the head
+      for (int i = tid; i < M * dh; i += CONSUMER_THREADS) {
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) s += red[w * M * dh + i];
+        const int m = i / dh, c = i - m * dh;
+        stcg(md.attn + (size_t)m * d + h * dh + c, s / ctl->rowsum[m]);
+      }
+      named_sync(1, CONSUMER_THREADS);
+      continue;
+    }
     float* part_out = md.apart + ((size_t)(h * nsplit + sp) * MAX_M) * dh;
     for (int i = tid; i < M * dh; i += CONSUMER_THREADS) {
       float s = 0.f;
@@ -824,8 +842,9 @@ template <int M>
 __device__ void attn_phase_mma(const ModelDev& md, int layer, int pos0, int cta, int G, char* xs, int xbytes,
                                Ctrl* ctl) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int H = md.H, dh = md.dh, d = md.d, nsplit = md.nsplit;
+  const int H = md.H, dh = md.dh, d = md.d;
   const int len = pos0 + M;
+  const int nsplit = eff_nsplit(md, len);
   const int Lc = (len + nsplit - 1) / nsplit;
   const int rowb = dh * 2, cpr = rowb >> 4;
   const int gq = lane >> 2, tq = lane & 3, mat = lane >> 3, rr = lane & 7;
@@ -948,6 +967,17 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int pos0, int cta,
       named_sync(1, CONSUMER_THREADS);   // tiles and S are free again
     }
     // oacc[0,1]: dim 16w+gq, queries 2tq, 2tq+1; oacc[2,3]: dim +8
+    if (nsplit == 1) {   // the whole context was here: normalise and finish the head
+      if (warp < nkd) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int q = 2 * tq + (j & 1), c = warp * 16 + gq + (j >> 1) * 8;
+          if (q < M) stcg(md.attn + (size_t)q * d + h * dh + c, oacc[j] / ctl->rowsum[q]);
+        }
+      }
+      named_sync(1, CONSUMER_THREADS);
+      continue;
+    }
     float* part_out = md.apart + ((size_t)(h * nsplit + sp) * MAX_M) * dh;
     if (warp < nkd) {
 #pragma unroll

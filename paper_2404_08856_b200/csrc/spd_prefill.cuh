@@ -15,7 +15,7 @@
 
 namespace spd {
 
-constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64, TC_STAGES = 6;
+constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64, TC_STAGES = 3;   // 3 stages: two CTAs per SM
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2, TC_B_BYTES = TC_BN * TC_BK * 2;
 constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;                  // 32 KB
 constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 + 256;   // + alignment slack + barriers
@@ -77,7 +77,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
 
 // grid = (N tiles, M tiles, batch); 128 threads: thread 0 feeds TMA, thread 32 issues the MMAs,
 // all four warps read the accumulator back (warp w owns TMEM lanes 32w..32w+31 = tile rows).
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(128, 2)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
                const __grid_constant__ CUtensorMap map_b, const TcArgs a) {
   extern __shared__ uint8_t tc_smem_raw[];
