@@ -207,7 +207,7 @@ def run_gpu(args, rank, world):
     dw = synth.Weights(wl.draft, wl.seeds["weights"], "draft")
     t_gen = time.time() - t0
     steps, warm = args.steps, max(args.warmup, 3)
-    max_seq = wl.n_image + wl.n_prompt + (GAMMA + 1) * (2 * (steps + warm) + 8) + 64
+    max_seq = wl.n_image + wl.n_prompt + max((GAMMA + 1) * (2 * (steps + warm) + 8), 128 + 4 * GAMMA) + 64
     ctx = spd.Spd(wl.target, wl.draft, tw.stored, dw.stored, max_seq, GAMMA, 1.0, True)
     del tw, dw
     img, ids = synth.image_embeds(wl), synth.prompt_ids(wl)
@@ -271,6 +271,39 @@ def run_gpu(args, rank, world):
     ctx.rollback(n_text0, prev0, pend0)
     ms_e2e, tokens_e2e = timed(block_host, steps)
 
+    # Injected acceptance: random-init models accept ~nothing, so to see the block loop at
+    # paper-like acceptance the draft still runs (for its cost) but the ids handed to the verify
+    # step are the target's own greedy continuation with probability alpha per token (seeded).
+    # Greedy speculative output equals the target's own output (Sec. 4 "Decoding"), so the
+    # continuation is known from one target-only run.
+    injected = []
+    if not args.no_injected:
+        n_inj = 96
+        ctx.rollback(n_text0, prev0, pend0)
+        ar, _ = ctx.generate(n_inj + GAMMA + 2, 0)            # ar[0] is the pending token
+        V = wl.target.vocab
+        for alpha in (0.5, 0.7, 0.9):
+            rng = np.random.default_rng(int(alpha * 100))
+            ctx.rollback(n_text0, prev0, pend0)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            done, blocks = 1, 0                                # tokens known so far (the pending one)
+            while done < n_inj:
+                ctx.draft_async(GAMMA)
+                ids_inj = np.empty(GAMMA, dtype=np.int32)
+                ok = True
+                for j in range(GAMMA):
+                    ok = ok and (rng.random() < alpha)
+                    tok = int(ar[done + j])
+                    ids_inj[j] = tok if ok else (tok + 1) % V
+                a_acc, nxt = ctx.verify(GAMMA, None, draft_ids=ids_inj)
+                done += a_acc + 1
+                blocks += 1
+            torch.cuda.synchronize()
+            dt = time.perf_counter() - t0
+            injected.append({"alpha": alpha, "tau": (done - 1) / blocks, "tokens_per_s": (done - 1) / dt,
+                             "blocks": blocks})
+
     # prefill again (scratch and tensor maps exist now): dense pass over 640 rows of both models
     pe = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
     pe[0].record(stream)
@@ -304,6 +337,7 @@ def run_gpu(args, rank, world):
                          "draft_step_ms_device_clock": st["ms_draft"] / max(st["blocks"], 1) / GAMMA},
             "target_only_tokens_per_s": st_ar["tokens"] / (st_ar["ms_total"] * 1e-3),
             "target_only_ms_per_token": st_ar["ms_total"] / st_ar["tokens"],
+            "injected_acceptance": injected,
             "note": "random-init target and draft agree on ~1/vocab of greedy tokens, so tau ~ 1 and speculative "
                     "tokens/s is below target-only decoding by construction; the verify step's cost does not "
                     "depend on acceptance",
@@ -361,6 +395,7 @@ def main():
     ap.add_argument("--layers", type=int, default=None,
                     help="truncate the target to this many layers (profiling captures only; not a bench value)")
     ap.add_argument("--draft-layers", type=int, default=None)
+    ap.add_argument("--no-injected", action="store_true", help="skip the injected-acceptance rows")
     ap.add_argument("--micro", default=None, choices=["gemm"], help="time one kernel alone instead of the path")
     ap.add_argument("--M", type=int, default=6)
     ap.add_argument("--N", type=int, default=32768)

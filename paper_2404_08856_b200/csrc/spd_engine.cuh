@@ -15,11 +15,15 @@
 // within the block | output projection + residual | RMSNorm -> gate/up projection +
 // SwiGLU | down projection + residual.  "|" is a grid barrier.
 //
-// Skinny GEMM Y[M,N] = X[M,K] W[N,K]^T: a tile is 32 weight rows; each of 8 compute warps
-// owns 4 rows, its lanes split K in 16-byte pieces (one ring stage = 32 rows x 512 B).
-// X lives in shared memory as fp32, laid out so that a lane's 16-byte reads are
-// conflict-free; products accumulate in fp32 with packed two-wide FMAs; the 4*M sums per
-// warp are reduced across lanes by a halving butterfly.
+// Skinny GEMM Y[M,N] = X[M,K] W[N,K]^T.  Weight rows are dealt to the CTAs in quads (balanced to
+// within 4 rows), a CTA's rows are cut into tiles of <= 32 rows and a ring stage is 512 bytes of
+// every row of a tile.  The M activation rows sit in shared memory as fp32.
+//  * bf16 weights: mma.sync m16n8k16 with the weights as the A operand (ldmatrix from the stage,
+//    16-byte chunks swizzled) and the activations as the B operand, split on the fly into two
+//    bf16 values (x = hi + lo), fp32 accumulation; the 8 warps split K inside a stage and their
+//    partial sums meet once per tile in shared memory.
+//  * fp32 weights: warp w owns rows 4w..4w+3 of the tile, lanes split K in 16-byte pieces,
+//    packed two-wide fp32 FMAs, butterfly reduction over the lanes.
 #pragma once
 #include "spd_device.cuh"
 #include "spd_sample.cuh"
