@@ -610,6 +610,53 @@ template <> struct CTraits<float> {
   }
 };
 
+// Merge of a head's KV splits (run by the CTA that finished the head's last split): the
+// per-split maxima and sums are fetched once into shared memory and turned into weights
+// w_s = exp(max_s - max) / sum_s' w_s' sum_s'; the partial outputs are then combined with all
+// loads of a thread in flight together.
+template <int M>
+__device__ void merge_head(const ModelDev& md, int h, int nsplit, float* scratch) {
+  const int tid = threadIdx.x, dh = md.dh, d = md.d;
+  float* mxs = scratch;                   // [nsplit][M] max, then weight
+  float* sms = scratch + nsplit * M;      // [nsplit][M] sum
+  for (int i = tid; i < nsplit * M; i += CONSUMER_THREADS) {
+    const int s2 = i / M, m = i - s2 * M;
+    const float* ml = md.aml + ((size_t)(h * nsplit + s2) * MAX_M + m) * 2;
+    mxs[i] = ldcg(ml);
+    sms[i] = ldcg(ml + 1);
+  }
+  named_sync(1, CONSUMER_THREADS);
+  if (tid < M) {
+    float gmax = -INFINITY;
+    for (int s2 = 0; s2 < nsplit; ++s2) gmax = fmaxf(gmax, mxs[s2 * M + tid]);
+    float den = 0.f;
+    for (int s2 = 0; s2 < nsplit; ++s2) {
+      const float mx = mxs[s2 * M + tid];
+      const float w = (mx == -INFINITY) ? 0.f : expf(mx - gmax);
+      den = fmaf(w, sms[s2 * M + tid], den);
+      mxs[s2 * M + tid] = w;
+    }
+    const float inv = 1.0f / den;
+    for (int s2 = 0; s2 < nsplit; ++s2) mxs[s2 * M + tid] *= inv;
+  }
+  named_sync(1, CONSUMER_THREADS);
+  for (int i = tid; i < M * dh; i += CONSUMER_THREADS) {
+    const int m = i / dh, c = i - m * dh;
+    float num = 0.f;
+    for (int s0 = 0; s0 < nsplit; s0 += 4) {
+      float pv[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        pv[u] = (s0 + u < nsplit) ? ldcg(md.apart + ((size_t)(h * nsplit + s0 + u) * MAX_M) * dh + i) : 0.f;
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (s0 + u < nsplit) num = fmaf(mxs[(s0 + u) * M + m], pv[u], num);
+    }
+    stcg(md.attn + (size_t)m * d + h * dh + c, num);
+  }
+  if (tid == 0) md.head_cnt[h] = 0u;
+}
+
 __device__ __forceinline__ void cp_async16(void* dst_smem, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
 }
@@ -801,24 +848,7 @@ __device__ void attn_phase(const ModelDev& md, int layer, int pos0, int cta, int
       __threadfence();
     }
     named_sync(1, CONSUMER_THREADS);
-    if (ctl->flag) {
-      for (int i = tid; i < M * dh; i += CONSUMER_THREADS) {
-        const int m = i / dh, c = i - m * dh;
-        float gmax = -INFINITY;
-        for (int s2 = 0; s2 < nsplit; ++s2)
-          gmax = fmaxf(gmax, ldcg(md.aml + ((size_t)(h * nsplit + s2) * MAX_M + m) * 2));
-        float num = 0.f, den = 0.f;
-        for (int s2 = 0; s2 < nsplit; ++s2) {
-          const float* ml = md.aml + ((size_t)(h * nsplit + s2) * MAX_M + m) * 2;
-          const float mx = ldcg(ml);
-          const float w = (mx == -INFINITY) ? 0.f : expf(mx - gmax);
-          den = fmaf(w, ldcg(ml + 1), den);
-          num = fmaf(w, ldcg(md.apart + ((size_t)(h * nsplit + s2) * MAX_M) * dh + i), num);
-        }
-        stcg(md.attn + (size_t)m * d + h * dh + c, num / den);
-      }
-      if (tid == 0) md.head_cnt[h] = 0u;
-    }
+    if (ctl->flag) merge_head<M>(md, h, nsplit, reinterpret_cast<float*>(Kt));
     named_sync(1, CONSUMER_THREADS);
   }
 }
@@ -1003,24 +1033,7 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int pos0, int cta,
       __threadfence();
     }
     named_sync(1, CONSUMER_THREADS);
-    if (ctl->flag) {
-      for (int i = tid; i < M * dh; i += CONSUMER_THREADS) {
-        const int m = i / dh, c = i - m * dh;
-        float gmax = -INFINITY;
-        for (int s2 = 0; s2 < nsplit; ++s2)
-          gmax = fmaxf(gmax, ldcg(md.aml + ((size_t)(h * nsplit + s2) * MAX_M + m) * 2));
-        float num = 0.f, den = 0.f;
-        for (int s2 = 0; s2 < nsplit; ++s2) {
-          const float* ml = md.aml + ((size_t)(h * nsplit + s2) * MAX_M + m) * 2;
-          const float mx = ldcg(ml);
-          const float w = (mx == -INFINITY) ? 0.f : expf(mx - gmax);
-          den = fmaf(w, ldcg(ml + 1), den);
-          num = fmaf(w, ldcg(md.apart + ((size_t)(h * nsplit + s2) * MAX_M) * dh + i), num);
-        }
-        stcg(md.attn + (size_t)m * d + h * dh + c, num / den);
-      }
-      if (tid == 0) md.head_cnt[h] = 0u;
-    }
+    if (ctl->flag) merge_head<M>(md, h, nsplit, reinterpret_cast<float*>(Kt));
     named_sync(1, CONSUMER_THREADS);
   }
 }
