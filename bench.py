@@ -34,7 +34,7 @@ sys.path.insert(0, os.path.join(ROOT, "tests"))
 
 import synth  # noqa: E402
 
-GAMMA = 5
+GAMMA = 5   # block size of the benchmark's workload; --gamma overrides it for sweeps
 METRIC = "spec_decode_tokens_per_s_llava7b_shape_bs1"
 
 
@@ -128,7 +128,7 @@ def run_reference(args, rank):
 def workload_config():
     return {"workload": "LLaVA-7B-shaped target (32 layers, d 4096, 32 heads, ffn 11008, vocab 32000, bf16) + "
                         "115M text-only draft (12 layers, d 768, tied, bf16); 576 image rows + 64 prompt ids; "
-                        "gamma 5; batch 1; greedy acceptance",
+                        f"gamma {GAMMA}; batch 1; greedy acceptance",
             "gamma": GAMMA, "kv_rows_at_start": 640, "l2": "inputs larger than L2 (13.2 GB of weights per step)",
             "parallelism": "replicas"}
 
@@ -328,7 +328,7 @@ def run_gpu(args, rank, world):
                     "ms_per_step": ms_e2e / steps},
             "gpu_launches": (GAMMA + 1) * steps,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "kernel": "forward_kernel<6,bf16> (verify step)",
+                         "traffic": None, "kernel": f"forward_kernel<{GAMMA + 1},bf16> (verify step)",
                          "bytes_per_launch": bytes_step, "ms_per_launch": verify_ms, "peak_kind": peak_kind,
                          "frac_of_8TBs": achieved / 8000.0},
             "verify_ms": verify_ms, "draft_step_ms": draft_ms, "tau": st["tau"],
@@ -400,7 +400,11 @@ def main():
     ap.add_argument("--M", type=int, default=6)
     ap.add_argument("--N", type=int, default=32768)
     ap.add_argument("--K", type=int, default=4096)
+    ap.add_argument("--gamma", type=int, default=None, help="block size (default 5; 3 and 7 for sweeps)")
     args = ap.parse_args()
+    if args.gamma is not None:
+        global GAMMA
+        GAMMA = args.gamma
     if args.micro:
         return run_micro(args)
     rank = int(os.environ.get("RANK", 0))

@@ -782,13 +782,11 @@ spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m, const flo
   dm.pos_base = 0;
   if (ad > 0) {
     const int dd = dm.cfg.d_model;
-    float* feats = ctx->rows;                 // [m][ad] staged behind the output rows
     float* outrows = ctx->rows;
     // stage features at the end of the rows buffer so that outputs can start at 0
     float* fstage = ctx->rows + (size_t)ctx->cfg.max_seq * (ctx->target.cfg.d_model > dd ? ctx->target.cfg.d_model : dd) - (size_t)m * ad;
     if ((size_t)m * ad + (size_t)m * dd > (size_t)ctx->cfg.max_seq * (ctx->target.cfg.d_model > dd ? ctx->target.cfg.d_model : dd))
       return fail(ctx, SPD_EOVERFLOW, "image features do not fit the staging buffer");
-    (void)feats;
     CU(cudaMemcpyAsync(fstage, draft_image_feats, (size_t)m * ad * sizeof(float), cudaMemcpyDefault, ctx->stream));
     for (int r = 0; r < m; r += MAX_M) {
       const int M = (m - r) < MAX_M ? (m - r) : MAX_M;
