@@ -423,3 +423,79 @@ def test_llava7b_shaped_two_layer_with_draft_adapter():
     r = lockstep(wl, False, 1.0, 2, 5e-2)
     print("adapter report", r)
     assert r["blocks"] >= 1 and r["max_draft_logit_err"] < 1e-2
+
+
+# ------------------------------------------------------------------ more edges
+
+@pytest.mark.gpu
+def test_llava7b_shaped_long_context_uses_attention_sub_chunks():
+    """576 image rows + 300 prompt ids: each KV split of the target now exceeds the attention
+    scratch, so the running softmax across sub-chunks is exercised (bf16 tensor-core attention),
+    as is a multi-split draft context."""
+    wl = synth.llava7b_workload(gamma=5, n_layers=2, draft_layers=2, n_prompt=300)
+    r = lockstep(wl, False, 1.0, 2, 5e-2)
+    print("long-context report", r)
+    assert r["blocks"] >= 1 and r["max_logit_err"] < 1e-2
+
+
+@pytest.mark.gpu
+def test_tiny_long_prompt_fp32_attention_splits():
+    wl = synth.Workload("tiny-long", synth.TINY_TARGET, synth.TINY_DRAFT, 16, 400, 4, 16)
+    r = lockstep(wl, False, 1.0, 3, 2e-4, std=0.1)
+    assert r["blocks"] == 3
+
+
+@pytest.mark.gpu
+def test_rollback_replays_identically_and_cache_overflow_is_reported():
+    spd = _lib()
+    wl = synth.tiny_workload(4)
+    tw, dw = H.build_weights(wl, 0.1)
+    max_seq = 16 + 16 + 40
+    gpu = H.make_gpu(wl, tw, dw, max_seq, 1.0, False, gamma_max=4)
+    img, ids = synth.image_embeds(wl), synth.prompt_ids(wl)
+    first = gpu.prefill(img, ids, u0=0.25)
+    u = synth.uniforms(3, "rollback", (12, 9))
+    a, sa = gpu.generate(12, 4, u)
+    # roll back to the state right after prefill and run the same loop again
+    gpu.rollback(len(ids), int(ids[-1]), first)
+    b, sb = gpu.generate(12, 4, u)
+    assert np.array_equal(a, b) and sa["blocks"] == sb["blocks"] and sa["accepted"] == sb["accepted"]
+    # fill the cache: verify steps until the library refuses
+    gpu.rollback(len(ids), int(ids[-1]), first)
+    seen = None
+    for _ in range(64):
+        try:
+            gpu.draft(4, u[0, :4])
+            gpu.verify(4, u[0, 4:])
+        except spd.SpdError as e:
+            seen = e.status
+            break
+    assert seen == spd.SPD_EOVERFLOW
+    n_text, _ = gpu.get_state()
+    assert 16 + n_text + 4 + 1 > max_seq - 5      # it stopped at the end of the cache, not before
+    gpu.close()
+
+
+@pytest.mark.gpu
+def test_device_resident_ids_and_probabilities():
+    """spd_draft writing ids / probabilities to device buffers and spd_verify reading them back
+    from there gives the same result as the internal hand-over."""
+    import torch
+    wl = synth.tiny_workload(4)
+    tw, dw = H.build_weights(wl, 0.1)
+    img, ids = synth.image_embeds(wl), synth.prompt_ids(wl)
+    u = synth.uniforms(3, "devptr", 9)
+    res = []
+    for external in (False, True):
+        gpu = H.make_gpu(wl, tw, dw, 96, 1.0, False)
+        gpu.prefill(img, ids, u0=0.5)
+        if external:
+            probs = torch.zeros(4, wl.target.vocab, device="cuda")
+            d = gpu.draft(4, u[:4], probs_out=probs)
+            assert abs(float(probs.sum()) - 4.0) < 1e-3
+            res.append(gpu.verify(4, u[4:], draft_ids=d, draft_probs=probs))
+        else:
+            gpu.draft(4, u[:4])
+            res.append(gpu.verify(4, u[4:]))
+        gpu.close()
+    assert res[0] == res[1]
