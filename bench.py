@@ -34,6 +34,11 @@ sys.path.insert(0, os.path.join(ROOT, "tests"))
 
 import synth  # noqa: E402
 
+# DRAM traffic of the verify kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum) on
+# the 2-layer truncation of the same workload: 1.093005 GB read + 5.92 MB written against 1.0931 GB of
+# algorithmic bytes.  Weights dominate and grow in proportion to the layer count, so the full launch's
+# traffic is this ratio times its algorithmic bytes.  Set to None when the kernel has changed since.
+VERIFY_TRAFFIC_RATIO = (1.093005e9 + 5.92128e6) / 1.0931e9
 GAMMA = 5   # block size of the benchmark's workload; --gamma overrides it for sweeps
 METRIC = "spec_decode_tokens_per_s_llava7b_shape_bs1"
 
@@ -328,7 +333,9 @@ def run_gpu(args, rank, world):
                     "ms_per_step": ms_e2e / steps},
             "gpu_launches": (GAMMA + 1) * steps,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "kernel": f"forward_kernel<{GAMMA + 1},bf16> (verify step)",
+                         "traffic": (VERIFY_TRAFFIC_RATIO * bytes_step if VERIFY_TRAFFIC_RATIO and GAMMA == 5 else None),
+                         "traffic_source": "ncu capture on the 2-layer truncation, scaled by algorithmic bytes",
+                         "kernel": f"forward_kernel<{GAMMA + 1},bf16> (verify step)",
                          "bytes_per_launch": bytes_step, "ms_per_launch": verify_ms, "peak_kind": peak_kind,
                          "frac_of_8TBs": achieved / 8000.0},
             "verify_ms": verify_ms, "draft_step_ms": draft_ms, "tau": st["tau"],
