@@ -326,6 +326,8 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
   md.kcache = kc; md.vcache = vc;
   if ((s = dalloc(ctx, &md.x, (size_t)MAX_M * d))) return s;
   if ((s = dalloc(ctx, &md.qbuf, (size_t)MAX_M * d))) return s;
+  if ((s = dalloc(ctx, &md.xg, (size_t)MAX_M * d))) return s;
+  if ((s = dalloc(ctx, &md.ssq, (size_t)ctx->n_sm * 8))) return s;
   if ((s = dalloc(ctx, &md.attn, (size_t)MAX_M * d))) return s;
   if ((s = dalloc(ctx, &md.act, (size_t)MAX_M * f))) return s;
   if ((s = dalloc(ctx, &md.apart, (size_t)H * md.nsplit * MAX_M * dh))) return s;
@@ -434,7 +436,7 @@ spd_status copy_out(spd_ctx* ctx, void* dst, const void* src_dev, size_t bytes, 
 
 StepArgs base_args(spd_ctx* ctx, ModelHost& mh) {
   StepArgs a{};
-  a.md = mh.md_dev;
+  a.md = mh.md;
   a.st = ctx->st;
   a.greedy = ctx->cfg.greedy;
   a.temperature = ctx->cfg.temperature;
@@ -666,6 +668,7 @@ spd_status spd_create(const spd_weights* target_w, const spd_weights* draft_w, c
   if (prop.major != 10) return bail(fail(ctx, SPD_ECUDA, "this library is built for sm_100a only"));
   if (!prop.cooperativeLaunch) return bail(fail(ctx, SPD_ECUDA, "cooperative launch not supported"));
   ctx->n_sm = prop.multiProcessorCount;
+  if (ctx->n_sm > 256) return bail(fail(ctx, SPD_ECUDA, "more than 256 SMs: the per-CTA partial sums are read 8 per lane"));
   ctx->smem_optin = (int)prop.sharedMemPerBlockOptin;
   if (cfg->temperature <= 0.f) ctx->cfg.temperature = 1.0f;
   const size_t esz_t = cfg->target.dtype ? 2 : 4, esz_d = cfg->draft.dtype ? 2 : 4;

@@ -39,7 +39,10 @@ constexpr int ENGINE_THREADS = CONSUMER_THREADS + 32;
 constexpr int CTRL_BYTES = 1024;
 constexpr int ZERO_BYTES = 512;         // a row of zeros for out-of-range ldmatrix lanes
 constexpr int RED_BYTES = 8192;         // cross-warp partial sums of one tile
-constexpr int FIXED_SMEM = CTRL_BYTES + ZERO_BYTES + RED_BYTES;
+constexpr int LAYER_SMEM_MAX = 64;       // per-layer pointer records kept in shared memory (more: read from global)
+constexpr int LAYER_BYTES = LAYER_SMEM_MAX * 48;
+constexpr int PRE_BYTES = 2048;          // epilogue operands fetched asynchronously during a tile's K loop
+constexpr int FIXED_SMEM = CTRL_BYTES + ZERO_BYTES + RED_BYTES + LAYER_BYTES + PRE_BYTES;
 // activation region: M rows of KC_MAX fp32 (or two bf16 planes), at least 64 KB so that the
 // attention phase can stage its K/V tiles there
 constexpr int X_PAD = 8;                // floats of padding per activation row (bank spread)
@@ -55,6 +58,7 @@ struct LayerDev {
   const void *wqkv, *wo, *wgu, *wd;   // repacked: see spd_api.cu
   const float *attn_norm, *ffn_norm;
 };
+static_assert(sizeof(LayerDev) == 48, "LAYER_BYTES assumes 48-byte records");
 
 struct ModelDev {
   int L, d, H, dh, f, V, max_seq, nsplit;
@@ -65,6 +69,8 @@ struct ModelDev {
   const float *rope_cos, *rope_sin;   // [max_seq][dh/2]
   void *kcache, *vcache;              // [L][max_seq][d]
   float *x, *qbuf, *attn, *act;       // [8][d], [8][d], [8][d], [8][f]
+  float *xg;                          // [8][d]: residual stream times the gain of the next RMSNorm
+  float *ssq;                         // [grid][8]: per-CTA partial sums of x^2 of the residual stream rows
   float *apart, *aml;                 // attention partials [H][nsplit][8][dh], [H][nsplit][8][2]
   unsigned* head_cnt;                 // [H]
   float* stat_part;                   // [grid][8][4]: row max, row sum, argmax value, argmax index
@@ -86,7 +92,7 @@ struct DevState {
 };
 
 struct StepArgs {
-  const ModelDev* md;
+  ModelDev md;            // by value: read through the constant bank
   DevState* st;
   unsigned* bar;          // grid-barrier counter, zero at launch
   int mode, gamma, j, pos_base, nstage, greedy;
@@ -135,12 +141,12 @@ struct Gemm {
   int N, K, pro, epi, layer;
 };
 
-__device__ __forceinline__ Gemm get_gemm(const ModelDev& md, int idx) {
+__device__ __forceinline__ Gemm get_gemm(const ModelDev& md, const LayerDev* layers, int idx) {
   Gemm g;
   const int l = idx >> 2, which = idx & 3;
   g.layer = l;
   if (l >= md.L) { g.W = md.lm_head; g.N = md.V; g.K = md.d; g.pro = PRO_NORM; g.epi = EPI_STORE; return g; }
-  const LayerDev& ly = md.layers[l];
+  const LayerDev& ly = layers[l];
   switch (which) {
     case 0: g.W = ly.wqkv; g.N = 3 * md.d; g.K = md.d; g.pro = PRO_NORM; g.epi = EPI_QKV; break;
     case 1: g.W = ly.wo; g.N = md.d; g.K = md.d; g.pro = PRO_PLAIN; g.epi = EPI_RESID; break;
@@ -236,7 +242,8 @@ struct XSrc {
 // the contraction).  `copy_out`: also publish the raw rows to global memory.
 template <int M, bool NORM>
 __device__ void load_x(float* X, int kcl, int klen, const XSrc<M>& src, int k0, const float* norm_w, float eps,
-                       int Ktotal, Ctrl* ctl, unsigned& xphase, float* copy_out, volatile int* err) {
+                       int Ktotal, Ctrl* ctl, unsigned& xphase, float* copy_out, volatile int* err,
+                       const float* ssq_in = nullptr, int G = 0) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int xs = kcl + X_PAD;
   if (tid == 0) {
@@ -263,6 +270,14 @@ __device__ void load_x(float* X, int kcl, int klen, const XSrc<M>& src, int k0, 
     for (int i = 0; i < PER; ++i) {
       const int k4 = tid + i * CONSUMER_THREADS;
       gain[i] = k4 < kl4 ? __ldg(reinterpret_cast<const float4*>(norm_w) + k4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
+  float part[8];
+  if (!NORM && ssq_in && warp < M) {   // requested after the rows' copies were issued
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int c = lane + 32 * i;
+      part[i] = c < G ? ldcg(ssq_in + c * 8 + warp) : 0.f;
     }
   }
   mbar_wait(&ctl->xbar, xphase, err, DEV_TIMEOUT_FULL);
@@ -300,6 +315,17 @@ __device__ void load_x(float* X, int kcl, int klen, const XSrc<M>& src, int k0, 
 #pragma unroll
       for (int w = 0; w < 8; ++w) s += ctl->red[w][tid];
       ctl->inv[tid] = 1.0f / sqrtf(s / (float)Ktotal + eps);
+    }
+  } else if (ssq_in) {
+    // the rows already carry the gain; the sums of squares wait as per-CTA partials (left by the last
+    // residual epilogue): warp m adds them up for row m in a fixed order
+    if (warp < M) {
+      float v = 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v += part[i];
+#pragma unroll
+      for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0) ctl->inv[warp] = 1.0f / sqrtf(v / (float)Ktotal + eps);
     }
   } else if (tid < M) {
     ctl->inv[tid] = 1.0f;
@@ -343,6 +369,10 @@ constexpr int dup_mask(int cnt, int bit) {
 struct EpiArgs {
   float* out;     // STORE: [M][ldo]; RESID: x [M][ldo]; SWIGLU: act [M][ldo]
   int ldo;
+  // RESID on bf16 models: the epilogue also prepares the next RMSNorm (NULL: off)
+  const float* next_gain;   // gain of the norm that reads the updated residual stream next
+  float* xg;                // [M][ldo] = x * next_gain
+  float* ssq;               // [grid][8] partial sums of x^2
   // QKV
   float* qbuf; void* kc; void* vc;  // cache bases already offset to the layer
   const float *cs, *sn;
@@ -392,6 +422,13 @@ __device__ __forceinline__ void epilogue_pair(int epi, const EpiArgs& e, int m, 
 
 // ------------------------------------------------------------------------------ consumers
 
+__device__ __forceinline__ void cp_async16(void* dst_smem, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+
 // fp32 weights: warp w owns rows 4w..4w+3 of the tile, lanes split K, packed fp32 FMAs.
 template <int M>
 __device__ __forceinline__ void compute_step_f32(const char* stage, const float* X, int xs, int s, int warp,
@@ -434,8 +471,8 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
 // This CTA's share of one projection.  src gives the M activation rows (fp32).
 template <int M, typename WT>
 __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, const XSrc<M>& src, const float* norm_w, float eps,
-                             float* copy_out, int cta, int G, Ring& ring, Ctrl* ctl, float* X, unsigned& xphase,
-                             float* red, uint32_t zero_addr, const char* stages, volatile int* err) {
+                             float* copy_out, const float* ssq_in, int cta, int G, Ring& ring, Ctrl* ctl, float* X,
+                             unsigned& xphase, float* red, float* pre_s, uint32_t zero_addr, const char* stages, volatile int* err) {
   constexpr int EPL = WTraits<WT>::EPL, KSTEP = 32 * EPL;
   constexpr bool BF = sizeof(WT) == 2;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -450,17 +487,22 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, const XSrc<M>& src
                __ldcg(reinterpret_cast<const float4*>(src.row[m] + k)));
       }
     }
+    if (e.ssq && tid < 8) stcg(e.ssq + cta * 8 + tid, 0.f);
     return;
   }
   int nchunk, kcl;
   chunking(g.K, KSTEP, nchunk, kcl);
   const int xs = kcl + X_PAD;
   if (nchunk == 1) {
-    if (g.pro == PRO_NORM) load_x<M, true>(X, kcl, g.K, src, 0, norm_w, eps, g.K, ctl, xphase, copy_out, err);
-    else load_x<M, false>(X, kcl, g.K, src, 0, nullptr, 0.f, g.K, ctl, xphase, nullptr, err);
+    const bool prenorm = g.pro == PRO_NORM && ssq_in != nullptr;
+    if (g.pro == PRO_NORM && !prenorm)
+      load_x<M, true>(X, kcl, g.K, src, 0, norm_w, eps, g.K, ctl, xphase, copy_out, err);
+    else
+      load_x<M, false>(X, kcl, g.K, src, 0, nullptr, eps, g.K, ctl, xphase, nullptr, err, prenorm ? ssq_in : nullptr, G);
   }
   trace_stamp(ctl, 1);
   const int gq = lane >> 2, tq = lane & 3;
+  float ssq_acc = 0.f;    // threads 0..7: this CTA's sum of x^2 of activation row tid (bf16 RESID with xg)
   for (int t = 0; t * 32 < rows; ++t) {
     const int nr = min(32, rows - t * 32);
     const int n0 = q0 * 4 + t * 32;
@@ -474,11 +516,14 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, const XSrc<M>& src
     for (int i = 0; i < 2; ++i)
 #pragma unroll
       for (int j = 0; j < 4; ++j) dacc[i][j] = 0.f;
-    // the residual this thread will add in the epilogue is requested now (bf16 path)
-    float resid = 0.f;
+    // bf16 RESID: the residual values (and the next norm's gains) of this tile travel to shared
+    // memory asynchronously while the K loop runs: pre_s[m*32 + row] and pre_s[256 + row].  No
+    // register waits for them until the epilogue.
     if (BF && g.epi == EPI_RESID) {
       const int row = tid >> 3, m = tid & 7;
-      if (m < M && row < nr && n0 + row < g.N) resid = ldcg(e.out + (size_t)m * e.ldo + n0 + row);
+      if (m < M && (row & 3) == 0 && row < nr) cp_async16(pre_s + m * 32 + row, e.out + (size_t)m * e.ldo + n0 + row);
+      if (e.xg && tid < 8 && tid * 4 < nr) cp_async16(pre_s + 256 + tid * 4, e.next_gain + n0 + tid * 4);
+      asm volatile("cp.async.commit_group;" ::: "memory");
     }
     for (int c = 0; c < nchunk; ++c) {
       const int k0 = c * kcl, klen = min(kcl, g.K - k0);
@@ -555,9 +600,15 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, const XSrc<M>& src
         *reinterpret_cast<float2*>(rp + gq * 8 + tq * 2) = make_float2(dacc[gi][0], dacc[gi][1]);
         *reinterpret_cast<float2*>(rp + (gq + 8) * 8 + tq * 2) = make_float2(dacc[gi][2], dacc[gi][3]);
       }
+      if (g.epi == EPI_RESID) asm volatile("cp.async.wait_group 0;" ::: "memory");
       named_sync(1, CONSUMER_THREADS);
       {
         // thread -> (row of the tile, activation row): tid = row*8 + m
+        float resid = 0.f, gnext = 0.f;
+        if (g.epi == EPI_RESID) {
+          resid = pre_s[(tid & 7) * 32 + (tid >> 3)];
+          gnext = pre_s[256 + (tid >> 3)];
+        }
         float v = 0.f;
 #pragma unroll
         for (int w = 0; w < 8; ++w) v += red[w * 256 + tid];
@@ -566,10 +617,25 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, const XSrc<M>& src
         const float partner = __shfl_down_sync(0xffffffffu, v, 8);
         if ((row & 1) == 0 && m < M && row < nr)
           epilogue_pair<WT>(g.epi == EPI_RESID ? EPI_STORE : g.epi, e, m, n0 + row, g.N, v, partner);
+        if (g.epi == EPI_RESID && e.xg) {
+          // v is the updated residual stream at (m, n0 + row): hand the next RMSNorm its input
+          // times the gain, and this warp's share of sum(x^2) per activation row
+          const bool valid = m < M && row < nr && n0 + row < g.N;
+          if (valid) stcg(e.xg + (size_t)m * e.ldo + n0 + row, v * gnext);
+          float sq = valid ? v * v : 0.f;
+          sq += __shfl_xor_sync(0xffffffffu, sq, 8);
+          sq += __shfl_xor_sync(0xffffffffu, sq, 16);
+          if (lane < 8) ctl->red[warp][lane] = sq;
+        }
       }
       named_sync(1, CONSUMER_THREADS);
+      if (g.epi == EPI_RESID && e.xg && tid < 8) {
+#pragma unroll
+        for (int w = 0; w < 8; ++w) ssq_acc += ctl->red[w][tid];
+      }
     }
   }
+  if (BF && g.epi == EPI_RESID && e.ssq && tid < 8) stcg(e.ssq + cta * 8 + tid, ssq_acc);
 }
 
 // ------------------------------------------------------------------------------ grid barrier
@@ -657,12 +723,6 @@ __device__ void merge_head(const ModelDev& md, int h, int nsplit, float* scratch
   if (tid == 0) md.head_cnt[h] = 0u;
 }
 
-__device__ __forceinline__ void cp_async16(void* dst_smem, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() {
-  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
-}
 
 template <typename CT>
 __device__ __forceinline__ void frag_from_smem(const char* p, float (&f)[CTraits<CT>::E]) {

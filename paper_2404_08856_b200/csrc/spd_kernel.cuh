@@ -88,14 +88,16 @@ __device__ void draft_sample(const StepArgs& a, const ModelDev& md, DevState* st
 }
 
 template <int M, typename WT>
-__global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepArgs a) {
+__global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid_constant__ StepArgs a) {
   extern __shared__ __align__(1024) char smem[];
   Ctrl* ctl = reinterpret_cast<Ctrl*>(smem);
   float* red = reinterpret_cast<float*>(smem + CTRL_BYTES + ZERO_BYTES);
+  LayerDev* lay_s = reinterpret_cast<LayerDev*>(smem + CTRL_BYTES + ZERO_BYTES + RED_BYTES);
+  float* pre_s = reinterpret_cast<float*>(smem + CTRL_BYTES + ZERO_BYTES + RED_BYTES + LAYER_BYTES);
   float* X = reinterpret_cast<float*>(smem + FIXED_SMEM);
   char* stages = smem + FIXED_SMEM + x_bytes(M);
   const uint32_t zero_addr = smem_u32(smem + CTRL_BYTES);
-  const ModelDev& md = *a.md;
+  const ModelDev& md = a.md;
   DevState* st = a.st;
   volatile int* err = &st->err;
   const int tid = threadIdx.x, cta = blockIdx.x, G = gridDim.x;
@@ -109,6 +111,12 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
     mbar_fence_init();
   }
   if (tid < ZERO_BYTES / 4) reinterpret_cast<uint32_t*>(smem + CTRL_BYTES)[tid] = 0u;
+  // per-layer pointer records: shared memory copy (a dependent global load per projection otherwise)
+  const bool lay_in_smem = md.L <= LAYER_SMEM_MAX;
+  if (lay_in_smem)
+    for (int i = tid; i < md.L * (int)(sizeof(LayerDev) / 8); i += ENGINE_THREADS)
+      reinterpret_cast<uint64_t*>(lay_s)[i] = reinterpret_cast<const uint64_t*>(md.layers)[i];
+  const LayerDev* layers = lay_in_smem ? lay_s : md.layers;
   __syncthreads();
 
   const bool gemm_only = a.mode == MODE_GEMM;
@@ -127,7 +135,7 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
       produce_gemm<WT>(g, cta, G, ring, ctl, stages, pol, err);
     } else {
       for (int i = 0; i < n_gemm; ++i) {
-        const Gemm g = get_gemm(md, g_first + i);
+        const Gemm g = get_gemm(md, layers, g_first + i);
         produce_gemm<WT>(g, cta, G, ring, ctl, stages, pol, err);
       }
     }
@@ -150,7 +158,7 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
       XSrc<M> src;
 #pragma unroll
       for (int m = 0; m < M; ++m) src.row[m] = a.gx + (size_t)m * a.gK;
-      consume_gemm<M, WT>(g, e, src, nullptr, 0.f, nullptr, cta, G, ring, ctl, X, xphase, red, zero_addr, stages, err);
+      consume_gemm<M, WT>(g, e, src, nullptr, 0.f, nullptr, nullptr, cta, G, ring, ctl, X, xphase, red, pre_s, zero_addr, stages, err);
     } else {
       // positions and token ids of the M rows
       int pos0, pending = 0;
@@ -183,50 +191,64 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const StepAr
           ids[m] = 0;
         }
       const int d = md.d, f = md.f;
+      // bf16 models: every residual epilogue leaves x * (gain of the next RMSNorm) in md.xg and
+      // per-CTA sums of x^2 in md.ssq, so the norm costs its reader nothing; only the first
+      // projection of a launch normalises its rows itself.  fp32 models normalise on load.
+      constexpr bool PRE = sizeof(WT) == 2;
       XSrc<M> src_in, src_x, src_attn, src_act;
 #pragma unroll
       for (int m = 0; m < M; ++m) {
         src_in.row[m] = from_ids ? md.embed + (size_t)ids[m] * d : a.rows + (size_t)m * d;
-        src_x.row[m] = md.x + (size_t)m * d;
+        src_x.row[m] = (PRE ? md.xg : md.x) + (size_t)m * d;
         src_attn.row[m] = md.attn + (size_t)m * d;
         src_act.row[m] = md.act + (size_t)m * f;
       }
+      const float* ssq_in = PRE ? md.ssq : nullptr;
 
       for (int l = 0; l < n_layers_run; ++l) {
-        const LayerDev& ly = md.layers[l];
+        const LayerDev& ly = layers[l];
         EpiArgs e{};
         // QKV + RoPE + KV append
         e.qbuf = md.qbuf; e.d = d; e.dh = md.dh; e.pos0 = pos0; e.cs = md.rope_cos; e.sn = md.rope_sin;
         e.kc = static_cast<WT*>(md.kcache) + (size_t)l * md.max_seq * d;
         e.vc = static_cast<WT*>(md.vcache) + (size_t)l * md.max_seq * d;
-        consume_gemm<M, WT>(get_gemm(md, l * 4), e, l == 0 ? src_in : src_x, ly.attn_norm, md.eps,
-                            (l == 0 && cta == 0) ? md.x : nullptr, cta, G, ring, ctl, X, xphase, red, zero_addr,
-                            stages, err);
+        consume_gemm<M, WT>(get_gemm(md, layers, l * 4), e, l == 0 ? src_in : src_x, ly.attn_norm, md.eps,
+                            (l == 0 && cta == 0) ? md.x : nullptr, l == 0 ? nullptr : ssq_in, cta, G, ring, ctl, X,
+                            xphase, red, pre_s, zero_addr, stages, err);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         if constexpr (sizeof(WT) == 2) attn_phase_mma<M>(md, l, pos0, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
         else attn_phase<M, WT>(md, l, pos0, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         // output projection + residual
         e.out = md.x; e.ldo = d;
-        consume_gemm<M, WT>(get_gemm(md, l * 4 + 1), e, src_attn, nullptr, 0.f, nullptr, cta, G, ring, ctl, X, xphase,
-                            red, zero_addr, stages, err);
+        if (PRE) { e.next_gain = ly.ffn_norm; e.xg = md.xg; e.ssq = md.ssq; }
+        consume_gemm<M, WT>(get_gemm(md, layers, l * 4 + 1), e, src_attn, nullptr, 0.f, nullptr, nullptr, cta, G, ring, ctl, X,
+                            xphase, red, pre_s, zero_addr, stages, err);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         // gate/up + SwiGLU
         e.out = md.act; e.ldo = md.f;
-        consume_gemm<M, WT>(get_gemm(md, l * 4 + 2), e, src_x, ly.ffn_norm, md.eps, nullptr, cta, G, ring, ctl, X,
-                            xphase, red, zero_addr, stages, err);
+        e.next_gain = nullptr; e.xg = nullptr; e.ssq = nullptr;
+        consume_gemm<M, WT>(get_gemm(md, layers, l * 4 + 2), e, src_x, ly.ffn_norm, md.eps, nullptr, ssq_in, cta, G, ring, ctl,
+                            X, xphase, red, pre_s, zero_addr, stages, err);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         // down projection + residual
         e.out = md.x; e.ldo = d;
-        consume_gemm<M, WT>(get_gemm(md, l * 4 + 3), e, src_act, nullptr, 0.f, nullptr, cta, G, ring, ctl, X, xphase,
-                            red, zero_addr, stages, err);
+        if (PRE) {
+          e.next_gain = l + 1 < md.L ? layers[l + 1].attn_norm : md.final_norm;
+          e.xg = md.xg; e.ssq = md.ssq;
+        }
+        consume_gemm<M, WT>(get_gemm(md, layers, l * 4 + 3), e, src_act, nullptr, 0.f, nullptr, nullptr, cta, G, ring, ctl, X,
+                            xphase, red, pre_s, zero_addr, stages, err);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
       }
       if (want_head) {
         EpiArgs e{};
         e.out = a.logits; e.ldo = md.V;
-        consume_gemm<M, WT>(get_gemm(md, md.L * 4), e, src_x, md.final_norm, md.eps, nullptr, cta, G, ring, ctl, X,
-                            xphase, red, zero_addr, stages, err);
+        // head-only launches get the residual stream itself as rows and normalise it on load
+        const bool pre_head = PRE && n_layers_run > 0;
+        consume_gemm<M, WT>(get_gemm(md, layers, md.L * 4), e, pre_head ? src_x : (head_only ? src_in : src_x), md.final_norm,
+                            md.eps, nullptr, pre_head ? ssq_in : nullptr, cta, G, ring, ctl, X, xphase, red, pre_s, zero_addr,
+                            stages, err);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         // row statistics over vocabulary slices, then CTA 0 applies the sampling rule
         int r0, nrows;
