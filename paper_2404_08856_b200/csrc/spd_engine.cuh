@@ -540,33 +540,44 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, const XSrc<M>& src
           // warp w takes the two 16-wide K slices 2w, 2w+1 of this 256-wide step
           const uint32_t st_addr = smem_u32(stage);
           const int mat = lane >> 3, rr = lane & 7;
+          // B fragments from the fp32 tile, split on the fly: x = hi + lo (two bf16)
+          uint32_t bq[2][4];
 #pragma unroll
           for (int kk = 0; kk < 2; ++kk) {
             const int c16 = (warp * 2 + kk) * 2;     // first 16-byte chunk of the slice (of 32)
-            // B fragments from the fp32 tile, split on the fly: x = hi + lo (two bf16)
             float2 xa = make_float2(0.f, 0.f), xb = make_float2(0.f, 0.f);
             if (gq < M) {
               const float* xr = X + gq * xs + s * 256 + c16 * 8 + 2 * tq;
               xa = *reinterpret_cast<const float2*>(xr);
               xb = *reinterpret_cast<const float2*>(xr + 8);
             }
-            const uint32_t b0 = pack_bf16(xa.x, xa.y), b1 = pack_bf16(xb.x, xb.y);
-            const uint32_t b2 = pack_bf16(xa.x - bf16lo(b0), xa.y - bf16hi(b0));
-            const uint32_t b3 = pack_bf16(xb.x - bf16lo(b1), xb.y - bf16hi(b1));
+            bq[kk][0] = pack_bf16(xa.x, xa.y);
+            bq[kk][1] = pack_bf16(xb.x, xb.y);
+            bq[kk][2] = pack_bf16(xa.x - bf16lo(bq[kk][0]), xa.y - bf16hi(bq[kk][0]));
+            bq[kk][3] = pack_bf16(xb.x - bf16lo(bq[kk][1]), xb.y - bf16hi(bq[kk][1]));
+          }
+          // A fragments of both slices and both 16-row groups first, then the eight MMAs
+          uint32_t af[2][2][4];
+#pragma unroll
+          for (int kk = 0; kk < 2; ++kk) {
+            const int c16 = (warp * 2 + kk) * 2;
 #pragma unroll
             for (int gi = 0; gi < 2; ++gi) {
-              if (gi * 16 < nr) {
-                // A: matrices {rows 0-7 k0-7, rows 8-15 k0-7, rows 0-7 k8-15, rows 8-15 k8-15}
-                const int r = gi * 16 + (mat & 1) * 8 + rr;
-                const int ch = (c16 + (mat >> 1)) ^ (r & 7);
-                const uint32_t addr = r < nr ? st_addr + (uint32_t)(r * 512 + ch * 16) : zero_addr;
-                uint32_t a0, a1, a2, a3;
-                ldsm4(addr, a0, a1, a2, a3);
-                mma_bf16(dacc[gi], a0, a1, a2, a3, b0, b1);
-                mma_bf16(dacc[gi], a0, a1, a2, a3, b2, b3);
-              }
+              // A: matrices {rows 0-7 k0-7, rows 8-15 k0-7, rows 0-7 k8-15, rows 8-15 k8-15}
+              const int r = gi * 16 + (mat & 1) * 8 + rr;
+              const int ch = (c16 + (mat >> 1)) ^ (r & 7);
+              const uint32_t addr = r < nr ? st_addr + (uint32_t)(r * 512 + ch * 16) : zero_addr;
+              if (gi * 16 < nr) ldsm4(addr, af[kk][gi][0], af[kk][gi][1], af[kk][gi][2], af[kk][gi][3]);
             }
           }
+#pragma unroll
+          for (int kk = 0; kk < 2; ++kk)
+#pragma unroll
+            for (int gi = 0; gi < 2; ++gi)
+              if (gi * 16 < nr) {
+                mma_bf16(dacc[gi], af[kk][gi][0], af[kk][gi][1], af[kk][gi][2], af[kk][gi][3], bq[kk][0], bq[kk][1]);
+                mma_bf16(dacc[gi], af[kk][gi][0], af[kk][gi][1], af[kk][gi][2], af[kk][gi][3], bq[kk][2], bq[kk][3]);
+              }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&ctl->empty[ring.stage]);
