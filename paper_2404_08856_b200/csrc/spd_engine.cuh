@@ -125,6 +125,7 @@ struct Ctrl {
   float inv[MAX_M];
   float rowmax[MAX_M], rowsum[MAX_M];
   int flag;
+  int tok[MAX_M];                   // token ids of the M rows
   int trace_n;                      // entries written so far (CTA 0 only)
   unsigned long long* trace;        // NULL: tracing off
 };
@@ -229,10 +230,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-// Source rows of an activation tile: row m starts at row[m] (fp32, 16-byte aligned).
-template <int M>
+// Source rows of an activation tile (fp32, 16-byte aligned): row m starts at
+// base + (idx ? idx[m] : m) * stride; idx points to shared memory (token ids -> embedding rows).
 struct XSrc {
-  const float* row[M];
+  const float* base;
+  size_t stride;
+  const int* idx;
+  __device__ __forceinline__ const float* row(int m) const { return base + (size_t)(idx ? idx[m] : m) * stride; }
 };
 
 // Activation rows [M][klen] -> shared memory, fp32, row stride kcl + X_PAD floats.  The rows
@@ -241,7 +245,7 @@ struct XSrc {
 // gain in and leaves 1/rms in ctl->inv[m] for the epilogue (a per-row scalar commutes with
 // the contraction).  `copy_out`: also publish the raw rows to global memory.
 template <int M, bool NORM>
-__device__ void load_x(float* X, int kcl, int klen, const XSrc<M>& src, int k0, const float* norm_w, float eps,
+__device__ void load_x(float* X, int kcl, int klen, const XSrc& src, int k0, const float* norm_w, float eps,
                        int Ktotal, Ctrl* ctl, unsigned& xphase, float* copy_out, volatile int* err,
                        const float* ssq_in = nullptr, int G = 0) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -252,7 +256,7 @@ __device__ void load_x(float* X, int kcl, int klen, const XSrc<M>& src, int k0, 
 #pragma unroll
     for (int m = 0; m < M; ++m)
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                   ::"r"(smem_u32(X + m * xs)), "l"(src.row[m] + k0), "r"((unsigned)(klen * 4)),
+                   ::"r"(smem_u32(X + m * xs)), "l"(src.row(m) + k0), "r"((unsigned)(klen * 4)),
                      "r"(smem_u32(&ctl->xbar))
                    : "memory");
   }
@@ -470,7 +474,7 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
 
 // This CTA's share of one projection.  src gives the M activation rows (fp32).
 template <int M, typename WT>
-__device__ void consume_gemm(const Gemm& g, const EpiArgs& e, const XSrc<M>& src, const float* norm_w, float eps,
+__device__ void consume_gemm(const Gemm& g, const EpiArgs& e, const XSrc& src, const float* norm_w, float eps,
                              float* copy_out, const float* ssq_in, int cta, int G, Ring& ring, Ctrl* ctl, float* X,
                              unsigned& xphase, float* red, float* pre_s, uint32_t zero_addr, const char* stages, volatile int* err) {
   constexpr int EPL = WTraits<WT>::EPL, KSTEP = 32 * EPL;
@@ -484,7 +488,7 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, const XSrc<M>& src
       for (int i = tid; i < M * (g.K >> 2); i += CONSUMER_THREADS) {
         const int m = i / (g.K >> 2), k = (i - m * (g.K >> 2)) << 2;
         __stcg(reinterpret_cast<float4*>(copy_out + (size_t)m * g.K + k),
-               __ldcg(reinterpret_cast<const float4*>(src.row[m] + k)));
+               __ldcg(reinterpret_cast<const float4*>(src.row(m) + k)));
       }
     }
     if (e.ssq && tid < 8) stcg(e.ssq + cta * 8 + tid, 0.f);

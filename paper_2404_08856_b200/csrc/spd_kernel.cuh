@@ -155,9 +155,7 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
       Gemm g{a.gw, a.gN, a.gK, PRO_PLAIN, EPI_STORE, 0};
       EpiArgs e{};
       e.out = a.gy; e.ldo = a.gN;
-      XSrc<M> src;
-#pragma unroll
-      for (int m = 0; m < M; ++m) src.row[m] = a.gx + (size_t)m * a.gK;
+      const XSrc src{a.gx, (size_t)a.gK, nullptr};
       consume_gemm<M, WT>(g, e, src, nullptr, 0.f, nullptr, nullptr, cta, G, ring, ctl, X, xphase, red, pre_s, zero_addr, stages, err);
     } else {
       // positions and token ids of the M rows
@@ -191,65 +189,72 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
           ids[m] = 0;
         }
       const int d = md.d, f = md.f;
+      // the ids live in shared memory from here on (embedding rows, sampling rule)
+      if (tid == 0) {
+#pragma unroll
+        for (int m = 0; m < M; ++m) ctl->tok[m] = ids[m];
+      }
+      named_sync(1, CONSUMER_THREADS);
       // bf16 models: every residual epilogue leaves x * (gain of the next RMSNorm) in md.xg and
       // per-CTA sums of x^2 in md.ssq, so the norm costs its reader nothing; only the first
       // projection of a launch normalises its rows itself.  fp32 models normalise on load.
       constexpr bool PRE = sizeof(WT) == 2;
-      XSrc<M> src_in, src_x, src_attn, src_act;
-#pragma unroll
-      for (int m = 0; m < M; ++m) {
-        src_in.row[m] = from_ids ? md.embed + (size_t)ids[m] * d : a.rows + (size_t)m * d;
-        src_x.row[m] = (PRE ? md.xg : md.x) + (size_t)m * d;
-        src_attn.row[m] = md.attn + (size_t)m * d;
-        src_act.row[m] = md.act + (size_t)m * f;
-      }
-      const float* ssq_in = PRE ? md.ssq : nullptr;
+      const XSrc src_in = from_ids ? XSrc{md.embed, (size_t)d, ctl->tok} : XSrc{a.rows, (size_t)d, nullptr};
+      const XSrc src_x{PRE ? md.xg : md.x, (size_t)d, nullptr};
 
-      for (int l = 0; l < n_layers_run; ++l) {
-        const LayerDev& ly = layers[l];
+      // One pass over the projections: index 4l + {0: QKV, 1: O, 2: gate/up, 3: down}, then the LM
+      // head.  A single call site keeps one copy of the projection code in the kernel.
+      for (int i = 0; i < n_gemm; ++i) {
+        const int idx = g_first + i, l = idx >> 2, which = idx & 3;
+        const bool head = l >= md.L;
+        const Gemm g = get_gemm(md, layers, idx);
         EpiArgs e{};
-        // QKV + RoPE + KV append
-        e.qbuf = md.qbuf; e.d = d; e.dh = md.dh; e.pos0 = pos0; e.cs = md.rope_cos; e.sn = md.rope_sin;
-        e.kc = static_cast<WT*>(md.kcache) + (size_t)l * md.max_seq * d;
-        e.vc = static_cast<WT*>(md.vcache) + (size_t)l * md.max_seq * d;
-        consume_gemm<M, WT>(get_gemm(md, layers, l * 4), e, l == 0 ? src_in : src_x, ly.attn_norm, md.eps,
-                            (l == 0 && cta == 0) ? md.x : nullptr, l == 0 ? nullptr : ssq_in, cta, G, ring, ctl, X,
-                            xphase, red, pre_s, zero_addr, stages, err);
-        stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
-        if constexpr (sizeof(WT) == 2) attn_phase_mma<M>(md, l, pos0, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
-        else attn_phase<M, WT>(md, l, pos0, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
-        stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
-        // output projection + residual
-        e.out = md.x; e.ldo = d;
-        if (PRE) { e.next_gain = ly.ffn_norm; e.xg = md.xg; e.ssq = md.ssq; }
-        consume_gemm<M, WT>(get_gemm(md, layers, l * 4 + 1), e, src_attn, nullptr, 0.f, nullptr, nullptr, cta, G, ring, ctl, X,
-                            xphase, red, pre_s, zero_addr, stages, err);
-        stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
-        // gate/up + SwiGLU
-        e.out = md.act; e.ldo = md.f;
-        e.next_gain = nullptr; e.xg = nullptr; e.ssq = nullptr;
-        consume_gemm<M, WT>(get_gemm(md, layers, l * 4 + 2), e, src_x, ly.ffn_norm, md.eps, nullptr, ssq_in, cta, G, ring, ctl,
-                            X, xphase, red, pre_s, zero_addr, stages, err);
-        stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
-        // down projection + residual
-        e.out = md.x; e.ldo = d;
-        if (PRE) {
-          e.next_gain = l + 1 < md.L ? layers[l + 1].attn_norm : md.final_norm;
-          e.xg = md.xg; e.ssq = md.ssq;
+        XSrc src = src_x;
+        const float* norm_w = nullptr;
+        const float* ssq_in = nullptr;
+        float* copy_out = nullptr;
+        if (head) {
+          e.out = a.logits; e.ldo = md.V;
+          norm_w = md.final_norm;
+          // head-only launches get the residual stream itself as rows and normalise it on load
+          if (PRE && n_layers_run > 0) ssq_in = md.ssq;
+          else if (head_only) src = src_in;
+        } else {
+          const LayerDev& ly = layers[l];
+          if (which == 0) {          // QKV + RoPE + KV append
+            e.qbuf = md.qbuf; e.d = d; e.dh = md.dh; e.pos0 = pos0; e.cs = md.rope_cos; e.sn = md.rope_sin;
+            e.kc = static_cast<WT*>(md.kcache) + (size_t)l * md.max_seq * d;
+            e.vc = static_cast<WT*>(md.vcache) + (size_t)l * md.max_seq * d;
+            norm_w = ly.attn_norm;
+            if (l == 0) { src = src_in; if (cta == 0) copy_out = md.x; }
+            else if (PRE) ssq_in = md.ssq;
+          } else if (which == 1) {   // output projection + residual
+            e.out = md.x; e.ldo = d;
+            src = XSrc{md.attn, (size_t)d, nullptr};
+            if (PRE) { e.next_gain = ly.ffn_norm; e.xg = md.xg; e.ssq = md.ssq; }
+          } else if (which == 2) {   // gate/up + SwiGLU
+            e.out = md.act; e.ldo = f;
+            norm_w = ly.ffn_norm;
+            if (PRE) ssq_in = md.ssq;
+          } else {                   // down projection + residual
+            e.out = md.x; e.ldo = d;
+            src = XSrc{md.act, (size_t)f, nullptr};
+            if (PRE) {
+              e.next_gain = l + 1 < md.L ? layers[l + 1].attn_norm : md.final_norm;
+              e.xg = md.xg; e.ssq = md.ssq;
+            }
+          }
         }
-        consume_gemm<M, WT>(get_gemm(md, layers, l * 4 + 3), e, src_act, nullptr, 0.f, nullptr, nullptr, cta, G, ring, ctl, X,
-                            xphase, red, pre_s, zero_addr, stages, err);
+        consume_gemm<M, WT>(g, e, src, norm_w, md.eps, copy_out, ssq_in, cta, G, ring, ctl, X, xphase, red, pre_s,
+                            zero_addr, stages, err);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
+        if (!head && which == 0) {
+          if constexpr (sizeof(WT) == 2) attn_phase_mma<M>(md, l, pos0, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
+          else attn_phase<M, WT>(md, l, pos0, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
+          stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
+        }
       }
       if (want_head) {
-        EpiArgs e{};
-        e.out = a.logits; e.ldo = md.V;
-        // head-only launches get the residual stream itself as rows and normalise it on load
-        const bool pre_head = PRE && n_layers_run > 0;
-        consume_gemm<M, WT>(get_gemm(md, layers, md.L * 4), e, pre_head ? src_x : (head_only ? src_in : src_x), md.final_norm,
-                            md.eps, nullptr, pre_head ? ssq_in : nullptr, cta, G, ring, ctl, X, xphase, red, pre_s, zero_addr,
-                            stages, err);
-        stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
         // row statistics over vocabulary slices, then CTA 0 applies the sampling rule
         int r0, nrows;
         if (a.mode == MODE_VERIFY) { r0 = 0; nrows = a.gamma + 1; }
@@ -259,12 +264,12 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
         if (cta == 0) {
           const float* u = a.uniforms ? a.uniforms + (a.u_by_block ? (size_t)st->block * a.u_stride : 0) : nullptr;
           if (a.mode == MODE_VERIFY) {
-            verify_sample<M>(a, md, st, ctl, G, 0, a.gamma, u ? u + (a.u_by_block ? a.gamma : 0) : nullptr, ids + 1,
+            verify_sample<M>(a, md, st, ctl, G, 0, a.gamma, u ? u + (a.u_by_block ? a.gamma : 0) : nullptr, ctl->tok + 1,
                              pending);
           } else if (a.mode == MODE_DRAFT) {
             draft_sample<M>(a, md, st, ctl, G, M - 1, u);
           } else {
-            verify_sample<M>(a, md, st, ctl, G, M - 1, 0, u, ids, 0);
+            verify_sample<M>(a, md, st, ctl, G, M - 1, 0, u, ctl->tok, 0);
           }
         }
         stamp();
