@@ -152,21 +152,60 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
       if (row < a.M && col0 < a.N) {
         const long long off = (long long)z * a.out_batch + (long long)row * a.ldo + col0;
         const int nv = min(32, a.N - col0);
+        // a thread owns 32 consecutive columns of its row: 16-byte stores where the row start
+        // and the width allow it (ldo and out_batch multiples of 8, all 32 columns present)
+        const bool vec = nv == 32 && (a.ldo & 7) == 0 && (a.out_batch & 7) == 0;
         if (a.mode == TC_OUT_SPLIT) {
-          for (int j = 0; j < nv; j += 2) {
-            const float x0 = __uint_as_float(v[j]) * a.alpha, x1 = (j + 1 < nv) ? __uint_as_float(v[j + 1]) * a.alpha : 0.f;
-            const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
-            a.out_hi[off + j] = h0;
-            a.out_lo[off + j] = __float2bfloat16_rn(x0 - __bfloat162float(h0));
-            if (j + 1 < nv) {
-              a.out_hi[off + j + 1] = h1;
-              a.out_lo[off + j + 1] = __float2bfloat16_rn(x1 - __bfloat162float(h1));
+          if (vec) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              uint32_t hw[4], lw[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const float x0 = __uint_as_float(v[j + 2 * q]) * a.alpha, x1 = __uint_as_float(v[j + 2 * q + 1]) * a.alpha;
+                const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+                const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - __low2float(h), x1 - __high2float(h));
+                hw[q] = *reinterpret_cast<const uint32_t*>(&h);
+                lw[q] = *reinterpret_cast<const uint32_t*>(&l);
+              }
+              *reinterpret_cast<uint4*>(a.out_hi + off + j) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+              *reinterpret_cast<uint4*>(a.out_lo + off + j) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+            }
+          } else {
+            for (int j = 0; j < nv; j += 2) {
+              const float x0 = __uint_as_float(v[j]) * a.alpha, x1 = (j + 1 < nv) ? __uint_as_float(v[j + 1]) * a.alpha : 0.f;
+              const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
+              a.out_hi[off + j] = h0;
+              a.out_lo[off + j] = __float2bfloat16_rn(x0 - __bfloat162float(h0));
+              if (j + 1 < nv) {
+                a.out_hi[off + j + 1] = h1;
+                a.out_lo[off + j + 1] = __float2bfloat16_rn(x1 - __bfloat162float(h1));
+              }
             }
           }
         } else if (a.mode == TC_OUT_F32_ADD) {
-          for (int j = 0; j < nv; ++j) a.out_f32[off + j] += __uint_as_float(v[j]) * a.alpha;
+          if (vec) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              float4* p4 = reinterpret_cast<float4*>(a.out_f32 + off + j);
+              float4 o = *p4;
+              o.x += __uint_as_float(v[j]) * a.alpha; o.y += __uint_as_float(v[j + 1]) * a.alpha;
+              o.z += __uint_as_float(v[j + 2]) * a.alpha; o.w += __uint_as_float(v[j + 3]) * a.alpha;
+              *p4 = o;
+            }
+          } else {
+            for (int j = 0; j < nv; ++j) a.out_f32[off + j] += __uint_as_float(v[j]) * a.alpha;
+          }
         } else {
-          for (int j = 0; j < nv; ++j) a.out_f32[off + j] = __uint_as_float(v[j]) * a.alpha;
+          if (vec) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+              *reinterpret_cast<float4*>(a.out_f32 + off + j) =
+                  make_float4(__uint_as_float(v[j]) * a.alpha, __uint_as_float(v[j + 1]) * a.alpha,
+                              __uint_as_float(v[j + 2]) * a.alpha, __uint_as_float(v[j + 3]) * a.alpha);
+          } else {
+            for (int j = 0; j < nv; ++j) a.out_f32[off + j] = __uint_as_float(v[j]) * a.alpha;
+          }
         }
       }
     }
