@@ -156,9 +156,18 @@ def test_reject_sample_distribution_small_vocab():
 
 # ------------------------------------------------------------------ whole path, lock-step
 
-def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None, max_seq=None):
+def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None, max_seq=None, gain_seed=None):
     spd = _lib()
     tw, dw = H.build_weights(wl, std)
+    if gain_seed is not None:
+        # non-trivial RMSNorm gains (the generated ones are all 1): a gain taken from the wrong
+        # norm or layer, or dropped, then shows up in the logits
+        g = np.random.default_rng(gain_seed)
+        for w, cfg in ((tw, wl.target), (dw, wl.draft)):
+            for l in range(cfg.n_layers):
+                w.stored["attn_norm"][l] = g.uniform(0.5, 1.5, cfg.d_model).astype(np.float32)
+                w.stored["ffn_norm"][l] = g.uniform(0.5, 1.5, cfg.d_model).astype(np.float32)
+            w.stored["final_norm"] = g.uniform(0.5, 1.5, cfg.d_model).astype(np.float32)
     max_seq = max_seq or (wl.n_image + wl.n_prompt + 8 * (n_blocks + 2) + 16)
     orc = H.make_oracle(wl, tw, dw, max_seq, temperature, greedy)
     gpu = H.make_gpu(wl, tw, dw, max_seq, temperature, greedy)
@@ -307,6 +316,20 @@ def test_llava7b_shaped_two_layer_lockstep(gamma):
     print("two-layer report", r)
     assert r["blocks"] >= 1
     assert r["max_logit_err"] < 1e-2   # far inside the 5e-2 allowance
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("shape", ["tiny", "llava7b-3L"])
+def test_lockstep_with_random_norm_gains(shape):
+    """Every RMSNorm gain differs (per layer, per norm, per column): covers the gains that the
+    residual epilogue multiplies in for the NEXT norm on bf16 models (attention norm of the next
+    layer, FFN norm of the same layer, final norm after the last layer) and the on-load path."""
+    if shape == "tiny":
+        r = lockstep(synth.tiny_workload(gamma=4), False, 1.0, 4, 2e-4, gain_seed=7)
+    else:
+        wl = synth.llava7b_workload(gamma=5, n_layers=3, draft_layers=3, n_image=64, n_prompt=24)
+        r = lockstep(wl, False, 1.0, 3, 3e-2, gain_seed=8)   # gains up to 1.5 scale the logits and their error
+    assert r["blocks"] >= 3
 
 
 @pytest.mark.gpu
