@@ -333,6 +333,18 @@ def test_lockstep_with_random_norm_gains(shape):
 
 
 @pytest.mark.gpu
+def test_small_bf16_models_where_most_ctas_own_no_rows():
+    """bf16 weights at the tiny shapes (d 256 / 128): most of the 148 CTAs get no row of a
+    projection, the ragged K = 688 and 344 need zero padding, heads are 64 wide; exercises the
+    empty-CTA branches (residual copy, zero partial sums) and the dense prefill at odd sizes."""
+    t = synth.ModelCfg(2, 256, 4, 688, 1024, False, dtype="bf16")
+    d = synth.ModelCfg(1, 128, 2, 344, 1024, False, dtype="bf16")
+    wl = synth.Workload("tiny-bf16", t, d, 16, 16, 4, 32)
+    r = lockstep(wl, False, 1.0, 4, 2e-2, std=0.08, gain_seed=9)
+    assert r["blocks"] >= 4
+
+
+@pytest.mark.gpu
 def test_llava7b_shaped_two_layer_greedy():
     wl = synth.llava7b_workload(gamma=5, n_layers=2, draft_layers=2)
     r = lockstep(wl, True, 1.0, 3, 5e-2)
