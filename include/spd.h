@@ -107,6 +107,19 @@ spd_status spd_create(const spd_weights* target_w, const spd_weights* draft_w,
 void spd_destroy(spd_ctx* ctx);
 const char* spd_last_error(const spd_ctx* ctx);
 
+/* A second, independent sequence on the same models.  The method is stated for one sequence
+ * (Sec. 2.1: one draft block, one target call, one accept/reject pass); serving several
+ * sequences needs one KV cache pair, one device state and one set of work buffers per
+ * sequence, while the repacked weights (13 GB for the 7B shape) exist once.  *out gets a
+ * context with the same cfg and stream as `parent` that shares every weight buffer with it
+ * and owns everything else; it starts un-prefilled.  Each sequence is then driven with the
+ * calls below, in any interleaving on the shared stream (each call still streams the weights
+ * once: sequences are not batched into one kernel), and rolled back on its own.  Destroy
+ * order is free: the weights are released with the last context that uses them.  Errors:
+ * SPD_EINVAL (NULL), SPD_ESTATE (parent already destroyed), SPD_ENOMEM / SPD_ECUDA with the
+ * message left on `parent`.  Not thread-safe against other calls on `parent`. */
+spd_status spd_fork(spd_ctx* parent, spd_ctx** out);
+
 /* Prefill (Eq. 1): the target reads [image_embeds ; embed(prompt_ids)] at positions
  * 0..m+n-1 and fills its KV cache; its last row gives the first generated token (argmax,
  * or a draw with *u0).  The draft reads embed(prompt_ids) only, or, with an adapter,

@@ -18,7 +18,7 @@ SPD_OK, SPD_EINVAL, SPD_ESTATE, SPD_ENOMEM, SPD_EOVERFLOW, SPD_ECUDA, SPD_ETIMEO
 STATUS_NAMES = ["SPD_OK", "SPD_EINVAL", "SPD_ESTATE", "SPD_ENOMEM", "SPD_EOVERFLOW", "SPD_ECUDA",
                 "SPD_ETIMEOUT", "SPD_ENOTIMPL"]
 
-EXPORTS = ["spd_create", "spd_destroy", "spd_last_error", "spd_prefill", "spd_draft", "spd_verify",
+EXPORTS = ["spd_create", "spd_destroy", "spd_fork", "spd_last_error", "spd_prefill", "spd_draft", "spd_verify",
            "spd_generate", "spd_get_logits", "spd_get_draft_logits", "spd_rollback", "spd_get_state",
            "spd_reject_sample", "spd_skinny_gemm", "spd_verify_bytes", "spd_trace",
            "spd_skinny_gemm_noalloc"]
@@ -133,6 +133,14 @@ class Spd:
     def _check(self, st: int):
         if st != SPD_OK:
             raise SpdError(st, lib().spd_last_error(self._ctx).decode())
+
+    def fork(self) -> "Spd":
+        """Another sequence on the same weights (see spd_fork): own KV caches and state."""
+        other = object.__new__(Spd)
+        other.vocab, other.greedy = self.vocab, self.greedy
+        other._ctx = C.c_void_p(0)
+        self._check(lib().spd_fork(self._ctx, C.byref(other._ctx)))
+        return other
 
     def close(self):
         if getattr(self, "_ctx", None) and self._ctx.value:

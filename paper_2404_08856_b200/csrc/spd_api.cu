@@ -21,7 +21,6 @@ namespace {
 struct ModelHost {
   spd_model_cfg cfg{};
   ModelDev md{};            // host copy of the device descriptor
-  ModelDev* md_dev = nullptr;
   LayerDev* layers_dev = nullptr;
   int pos_base = 0;         // rows in front of the text (image rows / adapter rows)
   float* logits = nullptr;  // [8][V]
@@ -73,6 +72,10 @@ struct spd_ctx {
   unsigned long long* trace = nullptr;   // device buffer of phase timestamps (verify steps)
   int trace_cap = 0;
   cudaEvent_t ev[4]{};
+  // spd_fork: a fork shares its origin's weights; the origin is kept alive until the last fork is gone
+  spd_ctx* origin = nullptr;
+  int n_forks = 0;
+  bool zombie = false;       // destroyed by the caller while forks were alive
 };
 
 namespace {
@@ -198,6 +201,34 @@ spd_status check_model(spd_ctx* ctx, const spd_model_cfg& c, const char* who) {
   return SPD_OK;
 }
 
+// Everything of a model that belongs to ONE sequence: KV cache, activation rows, attention
+// partials, statistics, logits.  (Weights, embedding table, layer records and rotary tables are
+// shared between a context and its forks.)
+spd_status alloc_sequence_state(spd_ctx* ctx, ModelHost& mh) {
+  const spd_model_cfg& c = mh.cfg;
+  const int d = c.d_model, f = c.d_ffn, V = c.vocab, L = c.n_layers, H = c.n_heads, dh = d / H;
+  const int max_seq = ctx->cfg.max_seq;
+  const size_t esz = mh.esz;
+  ModelDev& md = mh.md;
+  spd_status s;
+  char *kc, *vc;
+  if ((s = dalloc(ctx, &kc, (size_t)L * max_seq * d * esz))) return s;
+  if ((s = dalloc(ctx, &vc, (size_t)L * max_seq * d * esz))) return s;
+  md.kcache = kc; md.vcache = vc;
+  if ((s = dalloc(ctx, &md.x, (size_t)MAX_M * d))) return s;
+  if ((s = dalloc(ctx, &md.qbuf, (size_t)MAX_M * d))) return s;
+  if ((s = dalloc(ctx, &md.xg, (size_t)MAX_M * d))) return s;
+  if ((s = dalloc(ctx, &md.ssq, (size_t)ctx->n_sm * 8))) return s;
+  if ((s = dalloc(ctx, &md.attn, (size_t)MAX_M * d))) return s;
+  if ((s = dalloc(ctx, &md.act, (size_t)MAX_M * f))) return s;
+  if ((s = dalloc(ctx, &md.apart, (size_t)H * md.nsplit * MAX_M * dh))) return s;
+  if ((s = dalloc(ctx, &md.aml, (size_t)H * md.nsplit * MAX_M * 2))) return s;
+  if ((s = dalloc(ctx, &md.head_cnt, (size_t)H))) return s;
+  if ((s = dalloc(ctx, &md.stat_part, (size_t)ctx->n_sm * MAX_M * 4))) return s;
+  if ((s = dalloc(ctx, &mh.logits, (size_t)MAX_M * V))) return s;
+  return SPD_OK;
+}
+
 spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, const spd_weights* w, int adapter_in,
                        void* staging, char* rm) {
   mh.cfg = c;
@@ -320,23 +351,7 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
     CU(cudaStreamSynchronize(ctx->stream));
     md.rope_cos = dc; md.rope_sin = ds;
   }
-  char *kc, *vc;
-  if ((s = dalloc(ctx, &kc, (size_t)L * max_seq * d * esz))) return s;
-  if ((s = dalloc(ctx, &vc, (size_t)L * max_seq * d * esz))) return s;
-  md.kcache = kc; md.vcache = vc;
-  if ((s = dalloc(ctx, &md.x, (size_t)MAX_M * d))) return s;
-  if ((s = dalloc(ctx, &md.qbuf, (size_t)MAX_M * d))) return s;
-  if ((s = dalloc(ctx, &md.xg, (size_t)MAX_M * d))) return s;
-  if ((s = dalloc(ctx, &md.ssq, (size_t)ctx->n_sm * 8))) return s;
-  if ((s = dalloc(ctx, &md.attn, (size_t)MAX_M * d))) return s;
-  if ((s = dalloc(ctx, &md.act, (size_t)MAX_M * f))) return s;
-  if ((s = dalloc(ctx, &md.apart, (size_t)H * md.nsplit * MAX_M * dh))) return s;
-  if ((s = dalloc(ctx, &md.aml, (size_t)H * md.nsplit * MAX_M * 2))) return s;
-  if ((s = dalloc(ctx, &md.head_cnt, (size_t)H))) return s;
-  if ((s = dalloc(ctx, &md.stat_part, (size_t)ctx->n_sm * MAX_M * 4))) return s;
-  if ((s = dalloc(ctx, &mh.logits, (size_t)MAX_M * V))) return s;
-  if ((s = dalloc(ctx, &mh.md_dev, (size_t)1))) return s;
-  CU(cudaMemcpyAsync(mh.md_dev, &md, sizeof(ModelDev), cudaMemcpyHostToDevice, ctx->stream));
+  if ((s = alloc_sequence_state(ctx, mh))) return s;
   CU(cudaStreamSynchronize(ctx->stream));
   mh.wbytes = ((size_t)L * (4ull * d * d + 3ull * d * f) + (size_t)V * d) * esz;
   return SPD_OK;
@@ -605,6 +620,29 @@ spd_status prefill_tc(spd_ctx* ctx, ModelHost& mh, float* X, int R) {
   return SPD_OK;
 }
 
+// Buffers of a context that are not part of a model: device state, barrier pool, uniforms,
+// draft distributions, prefill staging, output ids, pinned state copy, events, graph stream.
+spd_status alloc_ctx_buffers(spd_ctx* ctx) {
+  const spd_cfg* cfg = &ctx->cfg;
+  const int V = cfg->target.vocab;
+  const int dmax = cfg->target.d_model > cfg->draft.d_model ? cfg->target.d_model : cfg->draft.d_model;
+  spd_status s;
+  if ((s = dalloc(ctx, &ctx->st, 1))) return s;
+  if ((s = dalloc(ctx, &ctx->bars, (size_t)32 * BAR_POOL))) return s;
+  if ((s = dalloc(ctx, &ctx->ubuf, 16))) return s;
+  if ((s = dalloc(ctx, &ctx->qbuf, (size_t)(cfg->gamma_max > 0 ? cfg->gamma_max : 1) * V))) return s;
+  if ((s = dalloc(ctx, &ctx->rows, (size_t)cfg->max_seq * dmax))) return s;
+  if ((s = dalloc(ctx, &ctx->ids_dev, (size_t)cfg->max_seq))) return s;
+  ctx->out_cap = cfg->max_seq + MAX_M;
+  if ((s = dalloc(ctx, &ctx->out_dev, (size_t)ctx->out_cap))) return s;
+  if (cudaMallocHost(&ctx->st_host, sizeof(DevState)) != cudaSuccess) return fail(ctx, SPD_ENOMEM, "pinned allocation failed");
+  for (auto& e : ctx->ev)
+    if (cudaEventCreate(&e) != cudaSuccess) return fail(ctx, SPD_ECUDA, "event creation failed");
+  if (cudaStreamCreateWithFlags(&ctx->gs, cudaStreamNonBlocking) != cudaSuccess)
+    return fail(ctx, SPD_ECUDA, "stream creation failed");
+  return SPD_OK;
+}
+
 bool use_tc_prefill(const ModelHost& mh) {
   static int forced = -1;   // SPD_PREFILL=rows keeps the 8-row kernel (comparison runs)
   if (forced < 0) {
@@ -629,8 +667,7 @@ extern "C" {
 
 const char* spd_last_error(const spd_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
 
-void spd_destroy(spd_ctx* ctx) {
-  if (!ctx) return;
+static void destroy_now(spd_ctx* ctx) {
   cudaStreamSynchronize(ctx->stream);
   if (ctx->gs) cudaStreamSynchronize(ctx->gs);
   if (ctx->block_exec) cudaGraphExecDestroy(ctx->block_exec);
@@ -640,6 +677,46 @@ void spd_destroy(spd_ctx* ctx) {
   for (auto& e : ctx->ev)
     if (e) cudaEventDestroy(e);
   delete ctx;
+}
+
+void spd_destroy(spd_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->n_forks > 0) {   // forks still read this context's weights: free it with the last of them
+    cudaStreamSynchronize(ctx->stream);
+    ctx->zombie = true;
+    return;
+  }
+  spd_ctx* origin = ctx->origin;
+  destroy_now(ctx);
+  if (origin && --origin->n_forks == 0 && origin->zombie) destroy_now(origin);
+}
+
+spd_status spd_fork(spd_ctx* parent, spd_ctx** out) {
+  if (out) *out = nullptr;
+  if (!parent || !out) return SPD_EINVAL;
+  if (parent->zombie) return fail(parent, SPD_ESTATE, "spd_fork on a destroyed context");
+  spd_ctx* origin = parent->origin ? parent->origin : parent;   // forks of forks hang off the owner of the weights
+  spd_ctx* ctx = new (std::nothrow) spd_ctx();
+  if (!ctx) return SPD_ENOMEM;
+  ctx->cfg = parent->cfg;
+  ctx->stream = parent->stream;
+  ctx->device = parent->device; ctx->n_sm = parent->n_sm; ctx->smem_optin = parent->smem_optin;
+  ctx->target = origin->target;     // copies the descriptors: weight pointers are shared ...
+  ctx->draft = origin->draft;
+  ctx->target.pos_base = 0; ctx->draft.pos_base = 0;
+  spd_status s = alloc_sequence_state(ctx, ctx->target);   // ... the per-sequence buffers are new
+  if (!s) s = alloc_sequence_state(ctx, ctx->draft);
+  if (!s) s = alloc_ctx_buffers(ctx);
+  if (!s && cudaStreamSynchronize(ctx->stream) != cudaSuccess) s = fail(ctx, SPD_ECUDA, "sync failed");
+  if (s) {
+    parent->err = "spd_fork: " + ctx->err;
+    destroy_now(ctx);
+    return s;
+  }
+  ctx->origin = origin;
+  origin->n_forks++;
+  *out = ctx;
+  return SPD_OK;
 }
 
 spd_status spd_create(const spd_weights* target_w, const spd_weights* draft_w, const spd_cfg* cfg, spd_ctx** out) {
@@ -691,21 +768,7 @@ spd_status spd_create(const spd_weights* target_w, const spd_weights* draft_w, c
   cudaFree(staging);
   cudaFree(rowmajor);
   if (s) return bail(s);
-  const int V = cfg->target.vocab;
-  const int dmax = cfg->target.d_model > cfg->draft.d_model ? cfg->target.d_model : cfg->draft.d_model;
-  if ((s = dalloc(ctx, &ctx->st, 1))) return bail(s);
-  if ((s = dalloc(ctx, &ctx->bars, (size_t)32 * BAR_POOL))) return bail(s);
-  if ((s = dalloc(ctx, &ctx->ubuf, 16))) return bail(s);
-  if ((s = dalloc(ctx, &ctx->qbuf, (size_t)(cfg->gamma_max > 0 ? cfg->gamma_max : 1) * V))) return bail(s);
-  if ((s = dalloc(ctx, &ctx->rows, (size_t)cfg->max_seq * dmax))) return bail(s);
-  if ((s = dalloc(ctx, &ctx->ids_dev, (size_t)cfg->max_seq))) return bail(s);
-  ctx->out_cap = cfg->max_seq + MAX_M;
-  if ((s = dalloc(ctx, &ctx->out_dev, (size_t)ctx->out_cap))) return bail(s);
-  if (cudaMallocHost(&ctx->st_host, sizeof(DevState)) != cudaSuccess) return bail(fail(ctx, SPD_ENOMEM, "pinned allocation failed"));
-  for (auto& e : ctx->ev)
-    if (cudaEventCreate(&e) != cudaSuccess) return bail(fail(ctx, SPD_ECUDA, "event creation failed"));
-  if (cudaStreamCreateWithFlags(&ctx->gs, cudaStreamNonBlocking) != cudaSuccess)
-    return bail(fail(ctx, SPD_ECUDA, "stream creation failed"));
+  if ((s = alloc_ctx_buffers(ctx))) return bail(s);
   // every kernel variant that can be launched must fit one CTA per SM
   for (int M = 1; M <= MAX_M; ++M)
     for (int dt : {cfg->target.dtype, cfg->draft.dtype}) {

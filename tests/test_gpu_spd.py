@@ -534,3 +534,66 @@ def test_device_resident_ids_and_probabilities():
             res.append(gpu.verify(4, u[4:]))
         gpu.close()
     assert res[0] == res[1]
+
+
+def _prompt_variant(wl, k):
+    """k-th prompt / image of a multi-sequence case: same shapes, different seeded draws."""
+    w2 = synth.Workload(wl.name, wl.target, wl.draft, wl.n_image, wl.n_prompt + 3 * k, wl.gamma, wl.n_new,
+                        adapter_in=wl.adapter_in, seeds={"weights": 1, "inputs": 20 + k, "uniforms": 3})
+    return synth.image_embeds(w2), synth.prompt_ids(w2)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_forked_sequences_share_weights_and_keep_their_own_state(dtype):
+    """Three sequences on one set of weights (spd_fork), driven block by block in an interleaved
+    order with per-sequence rollback: each must produce what the oracle produces for that
+    sequence alone (greedy speculative decoding == target-only greedy decoding, Sec. 4), so
+    neither KV caches nor device state leak between sequences."""
+    t = synth.ModelCfg(2, 256, 4, 688, 1024, False, dtype=dtype)
+    d = synth.ModelCfg(1, 128, 2, 344, 1024, False, dtype=dtype)
+    wl = synth.Workload("tiny-fork", t, d, 16, 16, 4, 32)
+    # std 0.2 saturates the softmaxes: fine in fp32, but with a bf16 KV cache one rounding flip
+    # then moves a whole attention row, so the bf16 case uses a gentler scale
+    tw, dw = H.build_weights(wl, 0.2 if dtype == "fp32" else 0.05)
+    max_seq = 160
+    seqs = [H.make_gpu(wl, tw, dw, max_seq, 1.0, True)]
+    seqs += [seqs[0].fork(), seqs[0].fork()]
+    inputs = [_prompt_variant(wl, k) for k in range(3)]
+    want = []
+    for img, ids in inputs:
+        o = H.make_oracle(wl, tw, dw, max_seq, 1.0, True)
+        o.prefill(img, ids)
+        want.append(np.asarray(o.generate_target_only(24)))
+    firsts = [g.prefill(img, ids) for g, (img, ids) in zip(seqs, inputs)]
+    got = [[f] for f in firsts]
+    # sequence 1 runs two blocks that are thrown away again (rollback to the state after prefill)
+    seqs[1].draft(4, None); seqs[1].verify(4, None)
+    seqs[1].draft(4, None); seqs[1].verify(4, None)
+    seqs[1].rollback(len(inputs[1][1]), int(inputs[1][1][-1]), firsts[1])
+    for blk in range(40):
+        order = [(blk + k) % 3 for k in range(3)]
+        for k in order:
+            if len(got[k]) >= 24:
+                continue
+            ids_k = seqs[k].draft(4, None)
+            a, nxt = seqs[k].verify(4, None)
+            got[k] += [int(x) for x in ids_k[:a]] + [int(nxt)]
+        if all(len(g) >= 24 for g in got):
+            break
+    # the origin may go first: the weights live as long as a fork does
+    seqs[0].close()
+    extra = seqs[2].draft(4, None)
+    assert len(extra) == 4
+    for k in range(3):
+        g = np.asarray(got[k][:24])
+        if not np.array_equal(g, want[k]):
+            j = int(np.argmax(g != want[k]))
+            o2 = H.make_oracle(wl, tw, dw, max_seq, 1.0, True)
+            o2.prefill(*inputs[k])
+            if j > 0:
+                o2.generate_target_only(j)
+            row = o2.prefill_logits if j == 0 else o2.last_logits[-1]
+            assert H.top2_gap(row) < 1e-2, f"sequence {k} differs at token {j}"
+    seqs[1].close()
+    seqs[2].close()
