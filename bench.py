@@ -363,6 +363,64 @@ def run_gpu(args, rank, world):
         dist.destroy_process_group()
 
 
+def run_batched(args):
+    """The batched KV-heavy workload on forked sequences: B sequences (default 16), each with
+    576 image rows + 1024 prompt ids in its bf16 KV cache, gamma = 5, temperature 1, one block per
+    sequence per step.  Sequences share the weights (spd_fork) but are NOT batched into one weight
+    pass: every draft and verify call streams the weights once.  Prints one JSON line; not the
+    default benchmark."""
+    import torch
+    import paper_2404_08856_b200 as spd
+    from paper_2404_08856_b200 import build
+    torch.cuda.set_device(0)
+    build.build()
+    B, n_prompt, steps = args.batch, 1024, args.steps
+    wl = synth.llava7b_workload(gamma=GAMMA, n_layers=args.layers, draft_layers=args.draft_layers, n_prompt=n_prompt)
+    tw = synth.Weights(wl.target, wl.seeds["weights"], "target")
+    dw = synth.Weights(wl.draft, wl.seeds["weights"], "draft")
+    max_seq = wl.n_image + n_prompt + (GAMMA + 1) * (steps + max(args.warmup, 1) + 2) + 64
+    seqs = [spd.Spd(wl.target, wl.draft, tw.stored, dw.stored, max_seq, GAMMA, 1.0, False)]
+    del tw, dw
+    seqs += [seqs[0].fork() for _ in range(B - 1)]
+    stream = torch.cuda.current_stream()
+    t0 = time.time()
+    for k, g in enumerate(seqs):
+        w2 = synth.Workload(wl.name, wl.target, wl.draft, wl.n_image, n_prompt, GAMMA, 0,
+                            seeds={"weights": 1, "inputs": 100 + k, "uniforms": 3})
+        g.prefill(synth.image_embeds(w2), synth.prompt_ids(w2), u0=0.5)
+    torch.cuda.synchronize()
+    t_prefill = time.time() - t0
+    u = torch.from_numpy(synth.uniforms(3, "batched", (steps + args.warmup + 1, B, 2 * GAMMA + 1))).cuda()
+
+    def step(i):
+        for k, g in enumerate(seqs):
+            g.draft_async(GAMMA, u[i, k, :GAMMA])
+            g.verify_async(GAMMA, u[i, k, GAMMA:])
+
+    for i in range(max(args.warmup, 1)):
+        step(i)
+    torch.cuda.synchronize()
+    n0 = [g.get_state()[0] for g in seqs]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        step(max(args.warmup, 1) + i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    tokens = sum(g.get_state()[0] - a for g, a in zip(seqs, n0))
+    bytes_step = seqs[0].verify_bytes(GAMMA)
+    line = {"workload": "batched KV-heavy verify on forked sequences (weights shared, not batched)", "batch": B,
+            "kv_rows_per_sequence": wl.n_image + n_prompt, "gamma": GAMMA, "temperature": 1.0, "steps": steps,
+            "ms_per_step": ms / steps, "tokens_per_s": tokens / (ms * 1e-3), "tau": tokens / (steps * B),
+            "verify_bytes_per_sequence": bytes_step, "prefill_s_total": t_prefill,
+            "truncated_layers": args.layers}
+    for g in seqs[1:]:
+        g.close()
+    seqs[0].close()
+    print(json.dumps(line), flush=True)
+
+
 def run_micro(args):
     """Times the weight-streaming GEMM alone (the projections of one verify step):
     y[M,N] = x[M,K] w[N,K]^T, bf16 weights larger than L2, CUDA events, prints one JSON line."""
@@ -404,6 +462,9 @@ def main():
     ap.add_argument("--draft-layers", type=int, default=None)
     ap.add_argument("--no-injected", action="store_true", help="skip the injected-acceptance rows")
     ap.add_argument("--micro", default=None, choices=["gemm"], help="time one kernel alone instead of the path")
+    ap.add_argument("--workload", default="bs1", choices=["bs1", "batched"],
+                    help="batched: B forked sequences with 1600 cached rows each (informational line)")
+    ap.add_argument("--batch", type=int, default=16)
     ap.add_argument("--M", type=int, default=6)
     ap.add_argument("--N", type=int, default=32768)
     ap.add_argument("--K", type=int, default=4096)
@@ -414,6 +475,8 @@ def main():
         GAMMA = args.gamma
     if args.micro:
         return run_micro(args)
+    if args.workload == "batched":
+        return run_batched(args)
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
     if args.impl == "reference":
