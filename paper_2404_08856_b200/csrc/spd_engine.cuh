@@ -667,7 +667,8 @@ __device__ __forceinline__ void grid_barrier(unsigned* counter, unsigned& target
         break;
       }
     }
-    __threadfence();
+    // no fence here: the acquire load above orders this thread, the CTA barrier below hands
+    // that order on to the other compute threads (cumulativity)
   }
   named_sync(1, CONSUMER_THREADS);
 }
