@@ -35,10 +35,10 @@ sys.path.insert(0, os.path.join(ROOT, "tests"))
 import synth  # noqa: E402
 
 # DRAM traffic of the verify kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum) on
-# the 2-layer truncation of the same workload: 1.092901 GB read + 3.29 MB written against 1.093108 GB of
+# the 2-layer truncation of the same workload: 1.092901 GB read + 4.00 MB written against 1.093108 GB of
 # algorithmic bytes.  Weights dominate and grow in proportion to the layer count, so the full launch's
 # traffic is this ratio times its algorithmic bytes.  Set to None when the kernel has changed since.
-VERIFY_TRAFFIC_RATIO = (1.092901e9 + 3.290624e6) / 1.093107712e9
+VERIFY_TRAFFIC_RATIO = (1.092901e9 + 3.996416e6) / 1.093107712e9
 GAMMA = 5   # block size of the benchmark's workload; --gamma overrides it for sweeps
 METRIC = "spec_decode_tokens_per_s_llava7b_shape_bs1"
 
