@@ -134,6 +134,25 @@ spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m,
                        const float* draft_image_feats, const int32_t* prompt_ids, int n,
                        const float* u0, int32_t* first_token);
 
+/* Image adapter g_theta (Sec. 2.2: the image encodings H_1..H_m become the image embeddings
+ * V_i = g_theta(H_i) that the target conditions on; Appendix A.1: an MLP of two linear layers,
+ * 1024 -> 4096 -> 4096 for the 7B target, 1024 -> 1024 -> 1024 for a draft with its own
+ * adapter).  Computes out = GELU(feats W1^T) W2^T on the tensor cores.  The paper names neither
+ * the non-linearity nor biases: GELU in its exact form x * Phi(x) (LLaVA's projector) and no
+ * biases are used.  The result is what spd_prefill takes as image_embeds.
+ *   feats  fp32 [m, d_in], host or device (vision-encoder features; the encoder is not part
+ *          of this library)
+ *   w1     bf16 [d_hid, d_in], w2 bf16 [d_out, d_hid]: row-major, DEVICE, 16-byte aligned,
+ *          owned by the caller and only read
+ *   out    fp32 [m, d_out], DEVICE, 16-byte aligned
+ * d_in and d_hid must be multiples of 8.  Activations are carried as bf16 hi + lo pairs with
+ * fp32 accumulation, so the result matches an fp32 evaluation to ~1e-5 relative.  Uses the
+ * context's stream and keeps its scratch in the context; synchronises the stream before
+ * returning.  Errors: SPD_EINVAL (arguments, host weights), SPD_ENOMEM, SPD_ECUDA,
+ * SPD_ETIMEOUT.  May be called before or after spd_prefill; it does not touch the sequence. */
+spd_status spd_image_adapter(spd_ctx* ctx, const float* feats, int m, int d_in, const void* w1,
+                             int d_hid, const void* w2, int d_out, float* out);
+
 /* Draft step (Sec. 2.1): gamma tokens, one after the other, each drawn from the draft's
  * softmax(logits / T) with uniforms[j] (or argmax when greedy).
  *   uniforms     fp32 [gamma], host or device; may be NULL when greedy

@@ -21,7 +21,7 @@ STATUS_NAMES = ["SPD_OK", "SPD_EINVAL", "SPD_ESTATE", "SPD_ENOMEM", "SPD_EOVERFL
 EXPORTS = ["spd_create", "spd_destroy", "spd_fork", "spd_last_error", "spd_prefill", "spd_draft", "spd_verify",
            "spd_generate", "spd_get_logits", "spd_get_draft_logits", "spd_rollback", "spd_get_state",
            "spd_reject_sample", "spd_skinny_gemm", "spd_verify_bytes", "spd_trace",
-           "spd_skinny_gemm_noalloc"]
+           "spd_skinny_gemm_noalloc", "spd_image_adapter"]
 
 
 class SpdError(RuntimeError):
@@ -161,6 +161,13 @@ class Spd:
         self._check(lib().spd_prefill(self._ctx, _ptr(image_embeds), m, _ptr(draft_image_feats), _ptr(ids),
                                       int(ids.shape[0]), u, C.byref(first)))
         return first.value
+
+    def image_adapter(self, feats, w1, w2, out):
+        """out[m, d_out] = GELU(feats[m, d_in] w1[d_hid, d_in]^T) w2[d_out, d_hid]^T (see
+        spd_image_adapter): w1, w2 bf16 device tensors, out an fp32 device tensor."""
+        self._check(lib().spd_image_adapter(self._ctx, _ptr(feats), int(feats.shape[0]), int(feats.shape[1]),
+                                            _ptr(w1), int(w1.shape[0]), _ptr(w2), int(w2.shape[0]), _ptr(out)))
+        return out
 
     def draft(self, gamma: int, uniforms=None, probs_out=None):
         ids = np.zeros(gamma, dtype=np.int32)

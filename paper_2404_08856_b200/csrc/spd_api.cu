@@ -64,6 +64,12 @@ struct spd_ctx {
     __nv_bfloat16 *p_hi = nullptr, *p_lo = nullptr;
     float *wide = nullptr, *S = nullptr;
   } pf;
+  // scratch of spd_image_adapter, grown on demand
+  struct {
+    size_t cap_in = 0, cap_hid = 0;      // elements
+    float* feats = nullptr;              // staging for host features
+    __nv_bfloat16 *f_hi = nullptr, *f_lo = nullptr, *g_hi = nullptr, *g_lo = nullptr;
+  } ia;
   cudaStream_t gs = nullptr;             // internal stream: block graphs are captured and replayed here
   cudaGraphExec_t block_exec = nullptr;  // one speculative block (gamma draft steps + verify)
   int block_gamma = -1;
@@ -519,7 +525,8 @@ spd_status make_map(spd_ctx* ctx, CUtensorMap* m, const void* ptr, int inner, in
 
 struct Operand { const void* ptr; int inner, rows, batch; size_t row_stride, batch_stride; };
 
-spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const Operand& b, TcArgs args) {
+spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const Operand& b, TcArgs args,
+                   bool gelu = false) {
   CUtensorMap ma, ml, mb;
   spd_status s;
   if ((s = make_map(ctx, &ma, a_hi.ptr, a_hi.inner, a_hi.rows, a_hi.batch, a_hi.row_stride, a_hi.batch_stride))) return s;
@@ -527,13 +534,15 @@ spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const
   if ((s = make_map(ctx, &mb, b.ptr, b.inner, b.rows, b.batch, b.row_stride, b.batch_stride))) return s;
   static bool attr_set = false;
   if (!attr_set) {
-    CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
+    CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
+    CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
     attr_set = true;
   }
   args.split = 1;
   args.err = &ctx->st->err;
   dim3 grid((args.N + TC_BN - 1) / TC_BN, (args.M + TC_BM - 1) / TC_BM, a_hi.batch);
-  tc_gemm_kernel<<<grid, 128, TC_SMEM_BYTES, ctx->stream>>>(ma, ml, mb, args);
+  if (gelu) tc_gemm_kernel<true><<<grid, 128, TC_SMEM_BYTES, ctx->stream>>>(ma, ml, mb, args);
+  else tc_gemm_kernel<false><<<grid, 128, TC_SMEM_BYTES, ctx->stream>>>(ma, ml, mb, args);
   CU(cudaGetLastError());
   return SPD_OK;
 }
@@ -885,6 +894,55 @@ spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m, const flo
   }
   if ((s = sync_state(ctx))) return s;
   if (first_token) *first_token = ctx->st_host->pending;
+  return SPD_OK;
+}
+
+spd_status spd_image_adapter(spd_ctx* ctx, const float* feats, int m, int d_in, const void* w1, int d_hid,
+                             const void* w2, int d_out, float* out) {
+  if (!ctx) return SPD_EINVAL;
+  if (!feats || !w1 || !w2 || !out || m < 1 || d_in < 8 || d_hid < 8 || d_out < 1 || d_in % 8 || d_hid % 8)
+    return fail(ctx, SPD_EINVAL, "bad image adapter arguments (widths must be multiples of 8)");
+  if (!is_device_ptr(w1) || !is_device_ptr(w2) || !is_device_ptr(out))
+    return fail(ctx, SPD_EINVAL, "adapter weights and output must be device memory");
+  if ((reinterpret_cast<uintptr_t>(w1) | reinterpret_cast<uintptr_t>(w2) | reinterpret_cast<uintptr_t>(out)) & 15)
+    return fail(ctx, SPD_EINVAL, "adapter weights and output must be 16-byte aligned");
+  spd_status s;
+  auto& ia = ctx->ia;
+  const size_t n_in = (size_t)m * d_in, n_hid = (size_t)m * d_hid;
+  if (n_in > ia.cap_in) {   // earlier buffers stay in the context's allocation list until spd_destroy
+    if ((s = dalloc(ctx, &ia.feats, n_in))) return s;
+    if ((s = dalloc(ctx, &ia.f_hi, n_in))) return s;
+    if ((s = dalloc(ctx, &ia.f_lo, n_in))) return s;
+    ia.cap_in = n_in;
+  }
+  if (n_hid > ia.cap_hid) {
+    if ((s = dalloc(ctx, &ia.g_hi, n_hid))) return s;
+    if ((s = dalloc(ctx, &ia.g_lo, n_hid))) return s;
+    ia.cap_hid = n_hid;
+  }
+  const float* fdev = feats;
+  if (!is_device_ptr(feats)) {
+    CU(cudaMemcpyAsync(ia.feats, feats, n_in * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
+    fdev = ia.feats;
+  }
+  split_rows_kernel<<<592, 256, 0, ctx->stream>>>(fdev, ia.f_hi, ia.f_lo, n_in);
+  // hidden = GELU(H W1^T), kept as a bf16 hi/lo pair (the GELU runs in the GEMM epilogue)
+  TcArgs a{}; a.M = m; a.N = d_hid; a.K = d_in; a.mode = TC_OUT_SPLIT; a.alpha = 1.f;
+  a.out_hi = ia.g_hi; a.out_lo = ia.g_lo; a.ldo = d_hid;
+  if ((s = tc_gemm(ctx, {ia.f_hi, d_in, m, 1, (size_t)d_in * 2, n_in * 2}, {ia.f_lo, d_in, m, 1, (size_t)d_in * 2, n_in * 2},
+                   {w1, d_in, d_hid, 1, (size_t)d_in * 2, (size_t)d_hid * d_in * 2}, a, true))) return s;
+  // V = hidden W2^T
+  a = TcArgs{}; a.M = m; a.N = d_out; a.K = d_hid; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = out; a.ldo = d_out;
+  if ((s = tc_gemm(ctx, {ia.g_hi, d_hid, m, 1, (size_t)d_hid * 2, n_hid * 2}, {ia.g_lo, d_hid, m, 1, (size_t)d_hid * 2, n_hid * 2},
+                   {w2, d_hid, d_out, 1, (size_t)d_hid * 2, (size_t)d_out * d_hid * 2}, a))) return s;
+  // device-side waits are bounded; report one that ran out
+  int e = 0;
+  CU(cudaMemcpyAsync(&e, &ctx->st->err, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  if (e != DEV_OK) {
+    cudaMemsetAsync(&ctx->st->err, 0, sizeof(int), ctx->stream);
+    return check_dev_err(ctx, e);
+  }
   return SPD_OK;
 }
 

@@ -75,8 +75,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// GELU in its exact form x * Phi(x), the non-linearity between the two linear layers of the image
+// adapter g_theta (Sec. 2.2, Appendix A.1; the paper does not name it, LLaVA's projector uses it).
+__device__ __forceinline__ float gelu_exact(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
+
 // grid = (N tiles, M tiles, batch); 128 threads: thread 0 feeds TMA, thread 32 issues the MMAs,
 // all four warps read the accumulator back (warp w owns TMEM lanes 32w..32w+31 = tile rows).
+// GELU: the hi/lo output (TC_OUT_SPLIT) is gelu(alpha * accumulator) instead of alpha * accumulator.
+template <bool GELU>
 __global__ void __launch_bounds__(128, 2)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
                const __grid_constant__ CUtensorMap map_b, const TcArgs a) {
@@ -162,7 +168,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
               uint32_t hw[4], lw[4];
 #pragma unroll
               for (int q = 0; q < 4; ++q) {
-                const float x0 = __uint_as_float(v[j + 2 * q]) * a.alpha, x1 = __uint_as_float(v[j + 2 * q + 1]) * a.alpha;
+                float x0 = __uint_as_float(v[j + 2 * q]) * a.alpha, x1 = __uint_as_float(v[j + 2 * q + 1]) * a.alpha;
+                if (GELU) { x0 = gelu_exact(x0); x1 = gelu_exact(x1); }
                 const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
                 const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - __low2float(h), x1 - __high2float(h));
                 hw[q] = *reinterpret_cast<const uint32_t*>(&h);
@@ -173,7 +180,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             }
           } else {
             for (int j = 0; j < nv; j += 2) {
-              const float x0 = __uint_as_float(v[j]) * a.alpha, x1 = (j + 1 < nv) ? __uint_as_float(v[j + 1]) * a.alpha : 0.f;
+              float x0 = __uint_as_float(v[j]) * a.alpha, x1 = (j + 1 < nv) ? __uint_as_float(v[j + 1]) * a.alpha : 0.f;
+              if (GELU) { x0 = gelu_exact(x0); x1 = gelu_exact(x1); }
               const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
               a.out_hi[off + j] = h0;
               a.out_lo[off + j] = __float2bfloat16_rn(x0 - __bfloat162float(h0));

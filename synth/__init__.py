@@ -180,6 +180,20 @@ def image_features(wl: Workload) -> np.ndarray:
     return _normal(wl.seeds["inputs"], "image_feats", 0, (wl.n_image, max(wl.adapter_in, 1)), 1.0)
 
 
+def vision_features(seed: int, m: int, d_in: int) -> np.ndarray:
+    """Vision-encoder-shaped features H_1..H_m (CLIP ViT-L/14 gives 576 rows of width 1024),
+    fp32 [m, d_in] ~ N(0, 1)."""
+    return _normal(seed, f"vision_feats.{d_in}", 0, (m, d_in), 1.0)
+
+
+def adapter_mlp(seed: int, role: str, d_in: int, d_hid: int, d_out: int, std: float = 0.02):
+    """Weights of a two-layer image adapter as bfloat16 bit patterns (uint16), row-major
+    [out, in]: W1 [d_hid, d_in], W2 [d_out, d_hid] ~ N(0, std^2), no biases."""
+    w1 = _normal(seed, f"{role}.adapter_mlp.w1", 0, (d_hid, d_in), std)
+    w2 = _normal(seed, f"{role}.adapter_mlp.w2", 0, (d_out, d_hid), std)
+    return f32_to_bf16_bits(w1), f32_to_bf16_bits(w2)
+
+
 def prompt_ids(wl: Workload) -> np.ndarray:
     g = _rng(wl.seeds["inputs"], "prompt_ids")
     return g.integers(0, wl.target.vocab, size=wl.n_prompt, dtype=np.int32)
