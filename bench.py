@@ -40,6 +40,7 @@ import synth  # noqa: E402
 # traffic is this ratio times its algorithmic bytes.  Set to None when the kernel has changed since.
 VERIFY_TRAFFIC_RATIO = (1.092901e9 + 3.996416e6) / 1.093107712e9
 GAMMA = 5   # block size of the benchmark's workload; --gamma overrides it for sweeps
+DRAFT = "115m"   # "table1": the draft shape printed in the paper's Table 1 (informational run)
 METRIC = "spec_decode_tokens_per_s_llava7b_shape_bs1"
 
 
@@ -131,8 +132,10 @@ def run_reference(args, rank):
 
 
 def workload_config():
+    draft = ("115M text-only draft (12 layers, d 768, tied, bf16)" if DRAFT == "115m" else
+             "text-only draft of the paper's Table 1 (4 layers, d 1024, 8 heads, ffn 2816, untied, bf16)")
     return {"workload": "LLaVA-7B-shaped target (32 layers, d 4096, 32 heads, ffn 11008, vocab 32000, bf16) + "
-                        "115M text-only draft (12 layers, d 768, tied, bf16); 576 image rows + 64 prompt ids; "
+                        f"{draft}; 576 image rows + 64 prompt ids; "
                         f"gamma {GAMMA}; batch 1; greedy acceptance",
             "gamma": GAMMA, "kv_rows_at_start": 640, "l2": "inputs larger than L2 (13.2 GB of weights per step)",
             "parallelism": "replicas"}
@@ -206,7 +209,9 @@ def run_gpu(args, rank, world):
         build.build()
     if dist:
         dist.barrier()
-    wl = synth.llava7b_workload(gamma=GAMMA, n_layers=args.layers, draft_layers=args.draft_layers)
+    wl = synth.llava7b_workload(gamma=GAMMA, n_layers=args.layers, draft_layers=args.draft_layers, draft=DRAFT)
+    # cost ratio c of the memory-bound speed-up (Sec. 4 "Metrics"): draft / target parameter count
+    c_ratio = wl.draft.n_params() / wl.target.n_params()
     t0 = time.time()
     tw = synth.Weights(wl.target, wl.seeds["weights"], "target")
     dw = synth.Weights(wl.draft, wl.seeds["weights"], "draft")
@@ -306,8 +311,9 @@ def run_gpu(args, rank, world):
                 blocks += 1
             torch.cuda.synchronize()
             dt = time.perf_counter() - t0
-            injected.append({"alpha": alpha, "tau": (done - 1) / blocks, "tokens_per_s": (done - 1) / dt,
-                             "blocks": blocks})
+            tau_inj = (done - 1) / blocks
+            injected.append({"alpha": alpha, "tau": tau_inj, "tokens_per_s": (done - 1) / dt, "blocks": blocks,
+                             "mbsu": tau_inj / (c_ratio * GAMMA + 1.0)})
 
     # prefill again (scratch and tensor maps exist now): dense pass over 640 rows of both models
     pe = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
@@ -319,6 +325,21 @@ def run_gpu(args, rank, world):
     rows = wl.n_image + wl.n_prompt
     body = wl.target.n_layers * (4 * wl.target.d_model ** 2 + 3 * wl.target.d_model * wl.target.d_ffn)
     prefill_tflops = 2.0 * body * rows / (prefill_ms * 1e-3) / 1e12
+
+    # image adapter g_theta in front of the prefill (Sec. 2.2; Appendix A.1: 1024 -> 4096 -> 4096 on
+    # the 576 encoder rows), timed with events around the call's kernels
+    feats = torch.from_numpy(synth.vision_features(wl.seeds["inputs"], wl.n_image, 1024)).cuda()
+    aw = [torch.from_numpy(b.view(np.int16)).cuda().view(torch.bfloat16)
+          for b in synth.adapter_mlp(wl.seeds["weights"], "target", 1024, 4096, wl.target.d_model)]
+    v_out = torch.empty((wl.n_image, wl.target.d_model), device="cuda", dtype=torch.float32)
+    ctx.image_adapter(feats, aw[0], aw[1], v_out)
+    ae = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    ae[0].record(stream)
+    ctx.image_adapter(feats, aw[0], aw[1], v_out)
+    ae[1].record(stream)
+    torch.cuda.synchronize()
+    adapter_ms = ae[0].elapsed_time(ae[1])
+    adapter_flops = 2.0 * wl.n_image * (1024 * 4096 + 4096 * wl.target.d_model)
 
     value, ms = aggregate(float(tokens), ms, dist, "cuda")
     e2e, ms_e2e = aggregate(float(tokens_e2e), ms_e2e, dist, "cuda")
@@ -351,8 +372,13 @@ def run_gpu(args, rank, world):
             "prefill": {"ms": prefill_ms, "rows": rows, "projection_tflops": prefill_tflops,
                         "note": "target + draft; activations are fed as bf16 hi+lo, so the tensor cores do twice "
                                 "the projection flops counted here, plus attention"},
+            "image_adapter": {"ms": adapter_ms, "rows": wl.n_image, "shape": "1024 -> 4096 -> 4096, exact GELU",
+                              "tflops": adapter_flops / (adapter_ms * 1e-3) / 1e12,
+                              "note": "one call = split kernel + two tcgen05 GEMMs (hi+lo activations: twice "
+                                      "the flops counted) + stream synchronisation"},
+            "draft_over_target_params": c_ratio,
             "setup_s": {"weights": t_gen, "first_prefill": t_prefill}}
-    if rank == 0 and world == 1 and not args.layers:
+    if rank == 0 and world == 1 and not args.layers and DRAFT == "115m":
         tv, td, cores = oracle_block_seconds(2)
         line["cpu_baseline"] = {"value": 1.0 / (tv + GAMMA * td), "unit": "tokens/s", "cores": cores,
                                 "kind": "oracle", "sample": ORACLE_SAMPLE, "verify_s": tv, "draft_step_s": td}
@@ -468,8 +494,13 @@ def main():
     ap.add_argument("--M", type=int, default=6)
     ap.add_argument("--N", type=int, default=32768)
     ap.add_argument("--K", type=int, default=4096)
+    ap.add_argument("--draft", default="115m", choices=["115m", "table1"],
+                    help="draft shape: the configured 115M draft, or the draft column of the paper's Table 1")
     ap.add_argument("--gamma", type=int, default=None, help="block size (default 5; 3 and 7 for sweeps)")
     args = ap.parse_args()
+    if args.draft != "115m":
+        global DRAFT
+        DRAFT = args.draft
     if args.gamma is not None:
         global GAMMA
         GAMMA = args.gamma

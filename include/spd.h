@@ -67,7 +67,11 @@ typedef struct {
   float temperature;    /* both models' logits are divided by it before softmax */
   int greedy;           /* 1: argmax rule, probabilities and uniforms unused */
   int draft_adapter_in; /* 0: text-only draft (Sec. 3); else width of the image features
-                           its linear adapter projects (Sec. 4 "Draft Model Candidates") */
+                           its linear adapter projects (Sec. 4 "Draft Model Candidates").
+                           With draft_adapter_in == draft.d_model and no adapter matrix in the
+                           draft's weights, spd_prefill's draft_image_feats are image rows
+                           already in the draft's embedding space, e.g. the output of the
+                           draft's own two-layer adapter (Appendix A.1) from spd_image_adapter */
   void* stream;         /* cudaStream_t, may be NULL (legacy default stream) */
 } spd_cfg;
 
@@ -123,7 +127,8 @@ spd_status spd_fork(spd_ctx* parent, spd_ctx** out);
 /* Prefill (Eq. 1): the target reads [image_embeds ; embed(prompt_ids)] at positions
  * 0..m+n-1 and fills its KV cache; its last row gives the first generated token (argmax,
  * or a draw with *u0).  The draft reads embed(prompt_ids) only, or, with an adapter,
- * [draft_image_feats W_a^T ; embed(prompt_ids)].
+ * [draft_image_feats W_a^T ; embed(prompt_ids)] (or [draft_image_feats ; embed(prompt_ids)]
+ * when the rows are given in the draft's space, see spd_cfg.draft_adapter_in).
  *   image_embeds       fp32 [m, d_target], host or device; NULL iff m == 0
  *   draft_image_feats  fp32 [m, draft_adapter_in], host or device; NULL without adapter
  *   prompt_ids         int32 [n], host or device, n >= 1, each < vocab

@@ -7,7 +7,8 @@ Follows Sec. 2.1 and Sec. 3 of the paper, step by step (letters: p = target, q =
 1. prefill: the target reads [V_1..V_m ; embed(X_1..X_n)] (Eq. 1) and its last row gives
    the first generated token; the draft reads embed(X_1..X_n) only (Sec. 3), or, for the
    draft with an image adapter (Sec. 4 "Draft Model Candidates", Appendix A.1), the rows
-   [H W_a^T ; embed(X)];
+   [H W_a^T ; embed(X)] for a single linear adapter, or [rows ; embed(X)] when the caller
+   hands in the output of the draft's own two-layer adapter (oracle/adapter.py);
 2. draft: gamma tokens, auto-regressively, x_j ~ q_j(. | text so far) (Sec. 2.1);
 3. verify: ONE target call on [pending, x_1..x_gamma] gives p_1..p_{gamma+1}; the
    rejection rule of oracle/sampling.py decides the accepted count a and the next token;
@@ -65,8 +66,10 @@ class SpdOracle:
 
         drows = self.d.embed(prompt_ids)
         self.off = 0
-        if self.adapter_w is not None:
-            adapted = np.asarray(draft_image_feats, dtype=F32) @ self.adapter_w.T
+        if self.adapter_w is not None or draft_image_feats is not None:
+            adapted = np.asarray(draft_image_feats, dtype=F32)     # already in the draft's space ...
+            if self.adapter_w is not None:
+                adapted = adapted @ self.adapter_w.T                # ... or projected by W_a
             drows = np.concatenate([adapted, drows], axis=0)
             self.off = adapted.shape[0]
         self.d.forward(self.dc, drows, 0)

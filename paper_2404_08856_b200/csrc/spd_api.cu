@@ -31,6 +31,7 @@ struct ModelHost {
   struct RowMajor { __nv_bfloat16 *wqkv, *wo, *wgu, *wd; const float *attn_norm, *ffn_norm; };
   std::vector<RowMajor> rm;
   __nv_bfloat16* adapter_rm = nullptr;
+  bool rows_given = false;  // draft only: the image rows arrive already in the draft's space
 };
 
 }  // namespace
@@ -274,7 +275,8 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
   if (!w->final_norm) return fail(ctx, SPD_EINVAL, "missing final_norm");
   CU(cudaMemcpyAsync(fn, w->final_norm, d * sizeof(float), cudaMemcpyDefault, ctx->stream));
   md.final_norm = fn;
-  if (adapter_in > 0) {
+  mh.rows_given = adapter_in > 0 && !w->adapter && adapter_in == d;
+  if (adapter_in > 0 && !mh.rows_given) {
     if (!w->adapter) return fail(ctx, SPD_EINVAL, "draft_adapter_in > 0 but no adapter weights");
     char* ad = nullptr;
     if ((s = dalloc(ctx, &ad, packed_bytes(d, adapter_in, esz)))) return s;
@@ -329,7 +331,7 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
       mh.rm.push_back(r);
     }
   }
-  if (esz == 2 && adapter_in > 0) {
+  if (esz == 2 && adapter_in > 0 && !mh.rows_given) {
     if ((s = dalloc(ctx, &mh.adapter_rm, (size_t)d * adapter_in))) return s;
     CU(cudaMemcpyAsync(mh.adapter_rm, w->adapter, (size_t)d * adapter_in * 2, cudaMemcpyDefault, ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
@@ -827,7 +829,10 @@ spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m, const flo
     if ((s = prefill_scratch(ctx, Rt > Rd ? Rt : Rd))) return s;
     float* X = ctx->rows;
     dm.pos_base = 0;
-    if (ad > 0) {   // draft rows [H W_a^T ; embed(prompt)]
+    if (ad > 0 && dm.rows_given) {   // draft rows [given image rows ; embed(prompt)]
+      CU(cudaMemcpyAsync(X, draft_image_feats, (size_t)m * dd * sizeof(float), cudaMemcpyDefault, ctx->stream));
+      dm.pos_base = m;
+    } else if (ad > 0) {   // draft rows [H W_a^T ; embed(prompt)]
       CU(cudaMemcpyAsync(ctx->pf.wide, draft_image_feats, (size_t)m * ad * sizeof(float), cudaMemcpyDefault, ctx->stream));
       split_rows_kernel<<<592, 256, 0, ctx->stream>>>(ctx->pf.wide, ctx->pf.h_hi, ctx->pf.h_lo, (size_t)m * ad);
       TcArgs a{}; a.M = m; a.N = dd; a.K = ad; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = X; a.ldo = dd;
@@ -862,8 +867,9 @@ spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m, const flo
     float* fstage = ctx->rows + (size_t)ctx->cfg.max_seq * (ctx->target.cfg.d_model > dd ? ctx->target.cfg.d_model : dd) - (size_t)m * ad;
     if ((size_t)m * ad + (size_t)m * dd > (size_t)ctx->cfg.max_seq * (ctx->target.cfg.d_model > dd ? ctx->target.cfg.d_model : dd))
       return fail(ctx, SPD_EOVERFLOW, "image features do not fit the staging buffer");
-    CU(cudaMemcpyAsync(fstage, draft_image_feats, (size_t)m * ad * sizeof(float), cudaMemcpyDefault, ctx->stream));
-    for (int r = 0; r < m; r += MAX_M) {
+    CU(cudaMemcpyAsync(dm.rows_given ? outrows : fstage, draft_image_feats, (size_t)m * ad * sizeof(float),
+                       cudaMemcpyDefault, ctx->stream));
+    for (int r = 0; r < m && !dm.rows_given; r += MAX_M) {
       const int M = (m - r) < MAX_M ? (m - r) : MAX_M;
       StepArgs a = base_args(ctx, dm);
       a.mode = MODE_GEMM;

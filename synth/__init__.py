@@ -72,6 +72,7 @@ class Workload:
     gamma: int
     n_new: int
     adapter_in: int = 0   # 0: text-only draft; else width of the draft's image features
+    draft_mlp: bool = False  # the draft has its own two-layer adapter adapter_in -> d -> d
     seeds: dict = field(default_factory=lambda: {"weights": 1, "inputs": 2, "uniforms": 3})
 
 
@@ -79,6 +80,8 @@ TINY_TARGET = ModelCfg(2, 256, 4, 688, 1024, False, dtype="fp32")
 TINY_DRAFT = ModelCfg(1, 128, 2, 344, 1024, False, dtype="fp32")
 LLAVA7B_TARGET = ModelCfg(32, 4096, 32, 11008, 32000, False, dtype="bf16")
 DRAFT_115M = ModelCfg(12, 768, 12, 2048, 32000, True, dtype="bf16")
+# the draft column of the paper's Table 1: 4 layers, 8 heads, intermediate 2816, hidden 1024
+DRAFT_TABLE1 = ModelCfg(4, 1024, 8, 2816, 32000, False, dtype="bf16")
 
 
 def tiny_workload(gamma: int = 4, adapter: bool = False) -> Workload:
@@ -89,16 +92,22 @@ def tiny_workload(gamma: int = 4, adapter: bool = False) -> Workload:
 
 def llava7b_workload(gamma: int = 5, n_layers: int | None = None, adapter: bool = False,
                      n_image: int = 576, n_prompt: int = 64, n_new: int = 256,
-                     draft_layers: int | None = None) -> Workload:
+                     draft_layers: int | None = None, draft: str = "115m",
+                     draft_mlp: bool = False) -> Workload:
     """LLaVA-7B-shaped target with the 115M text-only draft.  ``n_layers`` truncates the
-    target (same per-layer shapes) for cases the CPU implementation must finish quickly."""
+    target (same per-layer shapes) for cases the CPU implementation must finish quickly.
+    ``draft="table1"`` selects the draft shape printed in the paper's Table 1; ``draft_mlp``
+    gives the draft its own two-layer image adapter 1024 -> d -> d (Appendix A.1)."""
     t = LLAVA7B_TARGET if n_layers is None else ModelCfg(
         n_layers, 4096, 32, 11008, 32000, False, dtype="bf16")
-    d = DRAFT_115M if draft_layers is None else ModelCfg(
-        draft_layers, 768, 12, 2048, 32000, True, dtype="bf16")
+    base = DRAFT_TABLE1 if draft == "table1" else DRAFT_115M
+    d = base if draft_layers is None else ModelCfg(
+        draft_layers, base.d_model, base.n_heads, base.d_ffn, base.vocab, base.tied_embeddings, dtype="bf16")
     name = "llava7b" if n_layers is None else f"llava7b-{n_layers}L"
-    return Workload(name + ("-adapter" if adapter else ""), t, d, n_image, n_prompt,
-                    gamma, n_new, adapter_in=1024 if adapter else 0)
+    name += "-t1draft" if draft == "table1" else ""
+    return Workload(name + ("-adapter" if adapter else "") + ("-mlp" if draft_mlp else ""), t, d, n_image,
+                    n_prompt, gamma, n_new, adapter_in=1024 if (adapter or draft_mlp) else 0,
+                    draft_mlp=draft_mlp)
 
 
 # ----------------------------------------------------------------------------- draws

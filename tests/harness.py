@@ -21,21 +21,22 @@ F32 = np.float32
 
 def build_weights(wl, std=0.02):
     tw = synth.Weights(wl.target, wl.seeds["weights"], "target", std=std)
-    dw = synth.Weights(wl.draft, wl.seeds["weights"], "draft", adapter_in=wl.adapter_in, std=std)
+    dw = synth.Weights(wl.draft, wl.seeds["weights"], "draft", adapter_in=0 if wl.draft_mlp else wl.adapter_in,
+                       std=std)
     return tw, dw
 
 
 def make_oracle(wl, tw, dw, max_seq, temperature=1.0, greedy=False):
     t = llama.Model(wl.target, tw, max_seq)
     d = llama.Model(wl.draft, dw, max_seq)
-    ad = dw.f32("adapter") if wl.adapter_in else None
+    ad = dw.f32("adapter") if wl.adapter_in and not wl.draft_mlp else None
     return SpdOracle(t, d, temperature, greedy, adapter_w=ad)
 
 
 def make_gpu(wl, tw, dw, max_seq, temperature=1.0, greedy=False, gamma_max=7):
     import paper_2404_08856_b200 as spd
     return spd.Spd(wl.target, wl.draft, tw.stored, dw.stored, max_seq, gamma_max, temperature, greedy,
-                   adapter_in=wl.adapter_in)
+                   adapter_in=wl.draft.d_model if wl.draft_mlp else wl.adapter_in)
 
 
 class SafeUniforms:

@@ -100,3 +100,37 @@ def test_adapter_in_front_of_the_prefill_two_layer_llava7b_shape(greedy):
 
     rep = lockstep(wl, greedy=greedy, temperature=1.0, n_blocks=2, logit_tol=5e-2, image_from=image_from)
     assert rep["blocks"] >= 1 and rep["max_logit_err"] < 1e-2
+
+
+@pytest.mark.gpu
+def test_table1_draft_with_its_own_two_layer_adapter():
+    """The paper's own draft column (Table 1: 4 layers, hidden 1024, 8 heads, intermediate 2816;
+    2 layers here) with the draft-side adapter 1024 -> 1024 -> 1024 of Appendix A.1: both
+    adapters run on the GPU, their outputs go to the prefill as device rows, then speculative
+    blocks follow in lock-step with the oracle."""
+    import torch
+    wl = synth.llava7b_workload(gamma=3, n_layers=2, draft_layers=2, draft="table1", draft_mlp=True)
+    feats = synth.vision_features(wl.seeds["inputs"], wl.n_image, 1024)
+    tw1, tw2 = synth.adapter_mlp(wl.seeds["weights"], "target", 1024, 4096, 4096)
+    dw1, dw2 = synth.adapter_mlp(wl.seeds["weights"], "draft", 1024, 1024, 1024)
+    dev = lambda b: torch.from_numpy(b.view(np.int16)).cuda().view(torch.bfloat16)
+
+    def image_from(gpu):
+        v_t = torch.empty((wl.n_image, 4096), device="cuda", dtype=torch.float32)
+        v_d = torch.empty((wl.n_image, 1024), device="cuda", dtype=torch.float32)
+        gpu.image_adapter(feats, dev(tw1), dev(tw2), v_t)
+        gpu.image_adapter(feats, dev(dw1), dev(dw2), v_d)
+        o_t = OA.image_adapter(feats, synth.bf16_bits_to_f32(tw1), synth.bf16_bits_to_f32(tw2)).astype(F32)
+        o_d = OA.image_adapter(feats, synth.bf16_bits_to_f32(dw1), synth.bf16_bits_to_f32(dw2)).astype(F32)
+        return v_t, o_t, v_d, o_d
+
+    rep = lockstep(wl, greedy=False, temperature=1.0, n_blocks=3, logit_tol=5e-2, image_from=image_from)
+    assert rep["blocks"] >= 1 and rep["max_logit_err"] < 1e-2 and rep["max_draft_logit_err"] < 1e-2
+
+
+@pytest.mark.gpu
+def test_table1_draft_text_only_lockstep():
+    """Text-only draft of the Table-1 shape against the 2-layer LLaVA-7B-shaped target."""
+    wl = synth.llava7b_workload(gamma=5, n_layers=2, draft_layers=4, draft="table1")
+    rep = lockstep(wl, greedy=True, temperature=1.0, n_blocks=2, logit_tol=5e-2)
+    assert rep["blocks"] >= 1 and rep["max_draft_logit_err"] < 1e-2

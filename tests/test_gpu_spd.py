@@ -158,8 +158,9 @@ def test_reject_sample_distribution_small_vocab():
 
 def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None, max_seq=None, gain_seed=None,
              image_from=None):
-    """`image_from(gpu_ctx) -> (device image rows, oracle image rows)` replaces the generated
-    image embeddings (used to put the image adapter in front of the prefill)."""
+    """`image_from(gpu_ctx) -> (device image rows, oracle image rows[, device draft rows, oracle
+    draft rows])` replaces the generated image embeddings (and the draft's image rows); used to
+    put the image adapters in front of the prefill."""
     spd = _lib()
     tw, dw = H.build_weights(wl, std)
     if gain_seed is not None:
@@ -176,9 +177,13 @@ def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None
     gpu = H.make_gpu(wl, tw, dw, max_seq, temperature, greedy)
     img = synth.image_embeds(wl) if wl.n_image else None
     gpu_img = img
-    if image_from is not None:
-        gpu_img, img = image_from(gpu)
     feats = synth.image_features(wl) if wl.adapter_in else None
+    gpu_feats = feats
+    if image_from is not None:
+        got = image_from(gpu)
+        gpu_img, img = got[0], got[1]
+        if len(got) == 4:
+            gpu_feats, feats = got[2], got[3]
     ids = synth.prompt_ids(wl)
     su = H.SafeUniforms(wl.seeds["uniforms"], f"lock.{wl.name}.{greedy}")
     report = {"max_logit_err": 0.0, "max_draft_logit_err": 0.0, "tolerated": 0, "blocks": 0, "accepted": 0}
@@ -191,7 +196,7 @@ def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None
         probe.prefill(img, ids, u0=0.5, draft_image_feats=feats)
         u0 = su.for_cdf(S.softmax_t(probe.prefill_logits, temperature))
         x0 = orc.prefill(img, ids, u0=u0, draft_image_feats=feats)
-    g0 = gpu.prefill(gpu_img, ids, u0=None if greedy else u0, draft_image_feats=feats)
+    g0 = gpu.prefill(gpu_img, ids, u0=None if greedy else u0, draft_image_feats=gpu_feats)
     err = float(np.abs(gpu.get_logits(1)[0] - orc.prefill_logits).max())
     report["prefill_logit_err"] = err
     report["max_logit_err"] = max(report["max_logit_err"], err)

@@ -94,3 +94,32 @@ def test_draft_with_image_adapter_sees_projected_features():
     t.prefill(img, ids)
     t.draft(4, None)
     assert np.abs(t.last_draft_logits[0] - want).max() > 1e-3
+
+
+def test_draft_rows_given_in_its_own_space_equal_the_linear_adapter_applied_outside():
+    """The draft's image rows may be handed in already projected (the output of its own
+    two-layer adapter): with rows = H W_a^T that must reproduce the run in which the loop
+    applies the linear adapter W_a itself, and the rows must matter (a text-only draft
+    proposes other tokens)."""
+    wl = synth.tiny_workload(4, adapter=True)
+    img, ids, feats = synth.image_embeds(wl), synth.prompt_ids(wl), synth.image_features(wl)
+    u = synth.uniforms(3, "rows.given", (12, 2 * 4 + 1))
+    a = build(wl, std=0.2)
+    a.prefill(img, ids, u0=0.3, draft_image_feats=feats)
+    out_a, st_a = a.generate(12, 4, u)
+    b = build(wl, std=0.2)
+    rows = feats.astype(F32) @ b.adapter_w.T
+    b.adapter_w = None
+    b.prefill(img, ids, u0=0.3, draft_image_feats=rows)
+    out_b, st_b = b.generate(12, 4, u)
+    assert np.array_equal(out_a, out_b) and st_a == st_b
+    assert b.off == wl.n_image
+    c = build(wl, std=0.2)
+    c.adapter_w = None
+    c.prefill(img, ids, u0=0.3)
+    assert c.off == 0
+    qa = build(wl, std=0.2)
+    qa.prefill(img, ids, u0=0.3, draft_image_feats=feats)
+    _, q_with = qa.draft(4, u[0, :4])
+    _, q_without = c.draft(4, u[0, :4])
+    assert np.abs(np.asarray(q_with[0]) - np.asarray(q_without[0])).max() > 1e-6
