@@ -40,6 +40,7 @@ import synth  # noqa: E402
 # traffic is this ratio times its algorithmic bytes.  Set to None when the kernel has changed since.
 VERIFY_TRAFFIC_RATIO = (1.092901e9 + 3.996416e6) / 1.093107712e9
 GAMMA = 5   # block size of the benchmark's workload; --gamma overrides it for sweeps
+SAMPLING = False   # --sampling: temperature-1 rejection sampling instead of greedy acceptance
 DRAFT = "115m"   # "table1": the draft shape printed in the paper's Table 1 (informational run)
 METRIC = "spec_decode_tokens_per_s_llava7b_shape_bs1"
 
@@ -136,7 +137,8 @@ def workload_config():
              "text-only draft of the paper's Table 1 (4 layers, d 1024, 8 heads, ffn 2816, untied, bf16)")
     return {"workload": "LLaVA-7B-shaped target (32 layers, d 4096, 32 heads, ffn 11008, vocab 32000, bf16) + "
                         f"{draft}; 576 image rows + 64 prompt ids; "
-                        f"gamma {GAMMA}; batch 1; greedy acceptance",
+                        f"gamma {GAMMA}; batch 1; " + ("temperature-1 speculative sampling" if SAMPLING
+                                                       else "greedy acceptance"),
             "gamma": GAMMA, "kv_rows_at_start": 640, "l2": "inputs larger than L2 (13.2 GB of weights per step)",
             "parallelism": "replicas"}
 
@@ -218,11 +220,21 @@ def run_gpu(args, rank, world):
     t_gen = time.time() - t0
     steps, warm = args.steps, max(args.warmup, 3)
     max_seq = wl.n_image + wl.n_prompt + max((GAMMA + 1) * (2 * (steps + warm) + 8), 128 + 4 * GAMMA) + 64
-    ctx = spd.Spd(wl.target, wl.draft, tw.stored, dw.stored, max_seq, GAMMA, 1.0, True)
+    greedy = not args.sampling
+    ctx = spd.Spd(wl.target, wl.draft, tw.stored, dw.stored, max_seq, GAMMA, 1.0, greedy)
     del tw, dw
+    # temperature-1 sampling: one row of 2*gamma+1 seeded uniforms per block, resident on the device
+    n_u = 4 * (steps + warm) + 64
+    u_host = None if greedy else synth.uniforms(wl.seeds["uniforms"], "bench", (n_u, 2 * GAMMA + 1))
+    u_dev = None if greedy else torch.from_numpy(u_host).cuda()
+    blk = [0]
+
+    def next_u():
+        blk[0] = (blk[0] + 1) % n_u
+        return blk[0]
     img, ids = synth.image_embeds(wl), synth.prompt_ids(wl)
     t0 = time.time()
-    ctx.prefill(img, ids)
+    ctx.prefill(img, ids, u0=None if greedy else 0.5)
     t_prefill = time.time() - t0
     n_text0, pend0 = ctx.get_state()
     prev0 = int(ids[-1])
@@ -232,16 +244,19 @@ def run_gpu(args, rank, world):
 
     def block_resident():
         e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        i = 0 if greedy else next_u()
         e[0].record(stream)
-        ctx.draft_async(GAMMA)
+        ctx.draft_async(GAMMA, None if greedy else u_dev[i, :GAMMA])
         e[1].record(stream)
-        ctx.verify_async(GAMMA)
+        ctx.verify_async(GAMMA, None if greedy else u_dev[i, GAMMA:])
         e[2].record(stream)
         ev.append(e)
 
     def block_host():
-        d = ctx.draft(GAMMA, None)                 # ids come back to the host ...
-        return ctx.verify(GAMMA, None, draft_ids=d)  # ... and are handed in again from the host
+        i = 0 if greedy else next_u()
+        d = ctx.draft(GAMMA, None if greedy else u_host[i, :GAMMA])   # ids come back to the host ...
+        # ... and are handed in again from the host (with the uniforms when sampling)
+        return ctx.verify(GAMMA, None if greedy else u_host[i, GAMMA:], draft_ids=d)
 
     def timed(fn, n):
         if dist:
@@ -271,9 +286,9 @@ def run_gpu(args, rank, world):
         verify_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
         # the same loop through spd_generate (one CUDA-graph replay per block) and target-only decoding
         ctx.rollback(n_text0, prev0, pend0)
-        _, st = ctx.generate(steps, GAMMA)
+        _, st = ctx.generate(steps, GAMMA, None if greedy else u_dev[:steps])
         ctx.rollback(n_text0, prev0, pend0)
-        _, st_ar = ctx.generate(max(steps, 8), 0)
+        _, st_ar = ctx.generate(max(steps, 8), 0, None if greedy else u_dev[:max(steps, 8), :1].contiguous())
     clocks = cs.summary()
     ctx.rollback(n_text0, prev0, pend0)
     for _ in range(2):
@@ -287,7 +302,7 @@ def run_gpu(args, rank, world):
     # Greedy speculative output equals the target's own output (Sec. 4 "Decoding"), so the
     # continuation is known from one target-only run.
     injected = []
-    if not args.no_injected:
+    if not args.no_injected and greedy:
         n_inj = 96
         ctx.rollback(n_text0, prev0, pend0)
         ar, _ = ctx.generate(n_inj + GAMMA + 2, 0)            # ar[0] is the pending token
@@ -318,7 +333,7 @@ def run_gpu(args, rank, world):
     # prefill again (scratch and tensor maps exist now): dense pass over 640 rows of both models
     pe = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
     pe[0].record(stream)
-    ctx.prefill(img, ids)
+    ctx.prefill(img, ids, u0=None if greedy else 0.5)
     pe[1].record(stream)
     torch.cuda.synchronize()
     prefill_ms = pe[0].elapsed_time(pe[1])
@@ -350,7 +365,8 @@ def run_gpu(args, rank, world):
             "dtype": "f32 accumulate on bf16 weights and bf16 KV cache", "data": "synthetic (seeded, random-init)",
             "config": dict(workload_config(), **({"truncated_layers": args.layers} if args.layers else {})),
             "clocks": clocks,
-            "e2e": {"value": e2e, "unit": "tokens/s", "h2d_bytes_per_step": GAMMA * 4, "d2h_bytes_per_step": (GAMMA + 2) * 4,
+            "e2e": {"value": e2e, "unit": "tokens/s", "h2d_bytes_per_step": GAMMA * 4 + (0 if greedy else (2 * GAMMA + 1) * 4),
+                    "d2h_bytes_per_step": (GAMMA + 2) * 4,
                     "ms_per_step": ms_e2e / steps},
             "gpu_launches": (GAMMA + 1) * steps,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -378,7 +394,7 @@ def run_gpu(args, rank, world):
                                       "the flops counted) + stream synchronisation"},
             "draft_over_target_params": c_ratio,
             "setup_s": {"weights": t_gen, "first_prefill": t_prefill}}
-    if rank == 0 and world == 1 and not args.layers and DRAFT == "115m":
+    if rank == 0 and world == 1 and not args.layers and DRAFT == "115m" and greedy:
         tv, td, cores = oracle_block_seconds(2)
         line["cpu_baseline"] = {"value": 1.0 / (tv + GAMMA * td), "unit": "tokens/s", "cores": cores,
                                 "kind": "oracle", "sample": ORACLE_SAMPLE, "verify_s": tv, "draft_step_s": td}
@@ -496,8 +512,13 @@ def main():
     ap.add_argument("--K", type=int, default=4096)
     ap.add_argument("--draft", default="115m", choices=["115m", "table1"],
                     help="draft shape: the configured 115M draft, or the draft column of the paper's Table 1")
+    ap.add_argument("--sampling", action="store_true",
+                    help="temperature-1 speculative sampling instead of greedy acceptance (informational line)")
     ap.add_argument("--gamma", type=int, default=None, help="block size (default 5; 3 and 7 for sweeps)")
     args = ap.parse_args()
+    if args.sampling:
+        global SAMPLING
+        SAMPLING = True
     if args.draft != "115m":
         global DRAFT
         DRAFT = args.draft

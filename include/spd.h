@@ -226,6 +226,25 @@ spd_status spd_reject_sample(const float* p, const float* q, const int32_t* ids,
                              const float* u, int B, int gamma, int V, int greedy,
                              int32_t* n_acc, int32_t* next, void* stream);
 
+/* Top-k / top-p (nucleus) truncation of probability rows ahead of the rule (Sec. 4 "Decoding"
+ * names sampling with top-p / top-k as future work; the paper itself decodes greedily).  Both
+ * the target's rows p and the draft's rows q are truncated and renormalised, the draft tokens
+ * are drawn from the truncated q, and spd_reject_sample is applied to the truncated rows; the
+ * emitted tokens then follow the truncated target distribution.
+ *   probs, out  fp32 [rows, V] DEVICE; out may be probs (in place)
+ *   top_k       keep the k most probable tokens; <= 0 or >= V: off
+ *   top_p       then keep the shortest most-probable prefix of what is left whose mass reaches
+ *               top_p times the mass left; >= 1: off; must be > 0
+ * Exact definitions: tokens are ordered by probability, equal probabilities by index (lower
+ * first); masses are the integers trunc(w * 2^32) and are summed as integers; the target
+ * mass is ceil(Z * trunc(top_p * 2^24) / 2^24), at least one token is kept; kept values are
+ * divided by float(kept mass) * 2^-32, the others become 0.  The result is therefore
+ * independent of any summation order.  Values <= 0 count as 0.
+ * V is limited by the shared memory of one CTA (V <= ~56000).  Asynchronous on stream.
+ * Errors: SPD_EINVAL (NULL, host pointers, sizes, top_p <= 0), SPD_ECUDA. */
+spd_status spd_truncate_probs(const float* probs, float* out, int rows, int V, int top_k,
+                              float top_p, void* stream);
+
 /* Y[M,N] = X[M,K] W[N,K]^T with the weight-streaming kernel of the verify projections
  * (Eq. 1's linear maps at M = gamma+1 rows).  x, y fp32 DEVICE, w DEVICE in `dtype`;
  * 1 <= M <= 8, K a multiple of 8.  Asynchronous on stream. */

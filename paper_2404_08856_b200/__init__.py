@@ -21,7 +21,7 @@ STATUS_NAMES = ["SPD_OK", "SPD_EINVAL", "SPD_ESTATE", "SPD_ENOMEM", "SPD_EOVERFL
 EXPORTS = ["spd_create", "spd_destroy", "spd_fork", "spd_last_error", "spd_prefill", "spd_draft", "spd_verify",
            "spd_generate", "spd_get_logits", "spd_get_draft_logits", "spd_rollback", "spd_get_state",
            "spd_reject_sample", "spd_skinny_gemm", "spd_verify_bytes", "spd_trace",
-           "spd_skinny_gemm_noalloc", "spd_image_adapter"]
+           "spd_skinny_gemm_noalloc", "spd_image_adapter", "spd_truncate_probs"]
 
 
 class SpdError(RuntimeError):
@@ -239,6 +239,16 @@ def reject_sample(p, q, ids, u, gamma: int, greedy: bool, n_acc, nxt, stream: in
                                  _ptr(nxt), C.c_void_p(stream))
     if st != SPD_OK:
         raise SpdError(st, "spd_reject_sample")
+
+
+def truncate_probs(probs, out, top_k: int = 0, top_p: float = 1.0, stream: int = 0):
+    """Top-k / top-p truncation and renormalisation of fp32 probability rows on the device
+    (see spd_truncate_probs); `out` may be `probs`."""
+    V = int(probs.shape[-1])
+    rows = int(probs.numel() // V)
+    st = lib().spd_truncate_probs(_ptr(probs), _ptr(out), rows, V, int(top_k), C.c_float(top_p), C.c_void_p(stream))
+    if st != SPD_OK:
+        raise SpdError(st, "spd_truncate_probs")
 
 
 def skinny_gemm(x, w, y, dtype: int, stream: int = 0):

@@ -11,6 +11,7 @@
 #include "../../include/spd.h"
 #include "spd_kernel.cuh"
 #include "spd_prefill.cuh"
+#include "spd_warp.cuh"
 
 using namespace spd;
 
@@ -232,6 +233,7 @@ spd_status alloc_sequence_state(spd_ctx* ctx, ModelHost& mh) {
   if ((s = dalloc(ctx, &md.aml, (size_t)H * md.nsplit * MAX_M * 2))) return s;
   if ((s = dalloc(ctx, &md.head_cnt, (size_t)H))) return s;
   if ((s = dalloc(ctx, &md.stat_part, (size_t)ctx->n_sm * MAX_M * 4))) return s;
+  if ((s = dalloc(ctx, &md.cdf_part, (size_t)ctx->n_sm * 2))) return s;
   if ((s = dalloc(ctx, &mh.logits, (size_t)MAX_M * V))) return s;
   return SPD_OK;
 }
@@ -417,7 +419,16 @@ spd_status launch_forward(spd_ctx* ctx, int M, int dtype, StepArgs a, cudaStream
   a.bar = bar;
   CU(cudaMemsetAsync(bar, 0, sizeof(unsigned), stream));
   void* params[] = {&a};
+  a.sample_r0 = M - 1;
   CU(cudaLaunchCooperativeKernel((const void*)fn, dim3(n_sm), dim3(ENGINE_THREADS), params, lc.smem, stream));
+  // sampling (not greedy): the forward kernel has left logits and per-slice row statistics; two
+  // small kernels spread the draw over the grid and commit the step
+  const bool samples = a.mode == MODE_VERIFY || a.mode == MODE_DRAFT || (a.mode == MODE_ROWS && a.want_sample);
+  if (samples && !a.greedy) {
+    sample_slices_kernel<<<n_sm, SAMPLE_THREADS, 0, stream>>>(a);
+    sample_pick_kernel<<<1, SAMPLE_THREADS, 0, stream>>>(a, n_sm);
+    CU(cudaGetLastError());
+  }
   return SPD_OK;
 }
 
@@ -1203,6 +1214,25 @@ spd_status spd_reject_sample(const float* p, const float* q, const int32_t* ids,
   if (!greedy && (!u || (gamma > 0 && !q))) return SPD_EINVAL;
   reject_sample_kernel<<<B, SAMPLE_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(p, q, ids, u, gamma, V, greedy,
                                                                                     n_acc, next);
+  return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ECUDA;
+}
+
+spd_status spd_truncate_probs(const float* probs, float* out, int rows, int V, int top_k, float top_p, void* stream) {
+  if (!probs || !out || rows < 1 || V < 1 || !(top_p > 0.0f)) return SPD_EINVAL;
+  if (!is_device_ptr(probs) || !is_device_ptr(out)) return SPD_EINVAL;
+  int dev = 0, optin = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+    return SPD_ECUDA;
+  const size_t smem = (size_t)V * sizeof(float);
+  if (smem + sizeof(TruncScratch) + 1024 > (size_t)optin) {
+    fprintf(stderr, "spd_truncate_probs: a row of %d probabilities does not fit shared memory\n", V);
+    return SPD_EINVAL;
+  }
+  if (cudaFuncSetAttribute((const void*)truncate_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+      cudaSuccess)
+    return SPD_ECUDA;
+  truncate_rows_kernel<<<rows, WARP_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(probs, out, V, top_k, top_p);
   return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ECUDA;
 }
 

@@ -74,6 +74,7 @@ struct ModelDev {
   float *apart, *aml;                 // attention partials [H][nsplit][8][dh], [H][nsplit][8][2]
   unsigned* head_cnt;                 // [H]
   float* stat_part;                   // [grid][8][4]: row max, row sum, argmax value, argmax index
+  unsigned long long* cdf_part;       // [grid][2]: integer mass of the CTA's vocabulary slice, (max weight, index)
   const LayerDev* layers;
 };
 
@@ -102,6 +103,7 @@ struct StepArgs {
   const int* row_ids;     // MODE_ROWS with rows == NULL: token ids [M]
   int rows_pos0, want_sample, init_n_text, init_prev;
   int skip_layers;        // MODE_ROWS: rows are the final residual stream (md.x); run the LM head only
+  int sample_r0;          // row of `logits` a draft step / a prefill chunk samples from (set at launch)
   // uniforms
   const float* uniforms;
   int u_stride, u_by_block;

@@ -4,87 +4,57 @@
 
 namespace spd {
 
-// Verification (Sec. 2.1 / Sec. 3; p = target, q = draft), run by CTA 0 after the row
-// statistics are merged.  Rows r0..r0+gamma of `logits` are p_1..p_{gamma+1}.
-template <int M>
-__device__ void verify_sample(const StepArgs& a, const ModelDev& md, DevState* st, Ctrl* ctl, int G, int r0,
-                              int gamma, const float* u, const int* ids /*gamma draft ids*/, int pending) {
-  const int tid = threadIdx.x;
-  const int V = md.V;
-  float* rmax = ctl->rowmax;
-  float* rsum = ctl->rowsum;
-  int* rarg = ctl->sc.aidx;
-  __shared__ int s_arg[MAX_M];
-  merge_stats(md.stat_part, G, gamma + 1, ctl, rmax, rsum, s_arg);
-  (void)rarg;
-  int r = gamma, tok;
-  if (a.greedy) {
-    for (int j = 0; j < gamma; ++j)
-      if (s_arg[j] != ids[j]) { r = j; break; }
-    tok = s_arg[r];
-  } else {
-    for (int j = 0; j < gamma; ++j) {
-      const int x = ids[j];
-      const float p = prob_of(ldcg(a.logits + (size_t)(r0 + j) * V + x), a.temperature, rmax[j], rsum[j]);
-      const float q = ldcg(a.q_in + (size_t)j * V + x);
-      if (!accept_test(u[j], p, q)) { r = j; break; }
+// Commit of a step by one thread: accepted count r, next token tok (Sec. 2.1: x_1..x_r and the
+// replacement / bonus token are emitted; the KV length follows the accepted count).
+__device__ __forceinline__ void commit_step(const StepArgs& a, DevState* st, int r, int tok, const int* ids, int pending) {
+  st->n_acc = r;
+  st->next = tok;
+  if (a.mode == MODE_ROWS) {           // prefill: the sequence starts here
+    st->n_text = a.init_n_text;
+    st->prev = a.init_prev;
+    st->pending = tok;
+    st->block = 0;
+    st->n_emitted = 0;
+    if (a.out_ids && st->out_cap > 0) { a.out_ids[0] = tok; st->n_emitted = 1; }
+  } else {                              // commit x_1..x_r and the next token
+    int ne = st->n_emitted;
+    if (a.out_ids) {
+      for (int j = 0; j < r; ++j)
+        if (ne < st->out_cap) a.out_ids[ne++] = ids[j];
+      if (ne < st->out_cap) a.out_ids[ne++] = tok;
     }
-    const float* lrow = a.logits + (size_t)(r0 + r) * V;
-    const float mx = rmax[r], sm = rsum[r], T = a.temperature;
-    if (r < gamma) {
-      const float* qrow = a.q_in + (size_t)r * V;
-      tok = block_sample(
-          [&](int k) { return fmaxf(0.0f, __fsub_rn(prob_of(ldcg(lrow + k), T, mx, sm), ldcg(qrow + k))); }, V,
-          u[gamma], &ctl->sc);
-    } else {
-      tok = block_sample([&](int k) { return prob_of(ldcg(lrow + k), T, mx, sm); }, V, u[gamma], &ctl->sc);
-    }
-  }
-  if (tid == 0) {
-    st->n_acc = r;
-    st->next = tok;
-    if (a.mode == MODE_ROWS) {           // prefill: the sequence starts here
-      st->n_text = a.init_n_text;
-      st->prev = a.init_prev;
-      st->pending = tok;
-      st->block = 0;
-      st->n_emitted = 0;
-      if (a.out_ids && st->out_cap > 0) { a.out_ids[0] = tok; st->n_emitted = 1; }
-    } else {                              // commit x_1..x_r and the next token
-      int ne = st->n_emitted;
-      if (a.out_ids) {
-        for (int j = 0; j < r; ++j)
-          if (ne < st->out_cap) a.out_ids[ne++] = ids[j];
-        if (ne < st->out_cap) a.out_ids[ne++] = tok;
-      }
-      st->n_emitted = ne;
-      st->n_text += r + 1;
-      st->prev = r >= 1 ? ids[r - 1] : pending;
-      st->pending = tok;
-      st->block += 1;
-    }
+    st->n_emitted = ne;
+    st->n_text += r + 1;
+    st->prev = r >= 1 ? ids[r - 1] : pending;
+    st->pending = tok;
+    st->block += 1;
   }
 }
 
-// Draft step j: q_j = softmax(logits/T) written to q_out row j, x_j drawn from it.
+// Greedy decoding (Sec. 4 "Decoding"), run by CTA 0 after the row statistics are merged: a draft
+// token is accepted iff it is the argmax of the target's row; the next token is the argmax of the
+// first mismatching row, or of row gamma.  Rows r0..r0+gamma of `logits` are p_1..p_{gamma+1}.
+// (With sampling the forward kernel stops after the row statistics and the two sampling kernels
+// below finish the step.)
 template <int M>
-__device__ void draft_sample(const StepArgs& a, const ModelDev& md, DevState* st, Ctrl* ctl, int G, int row,
-                             const float* u) {
-  const int tid = threadIdx.x, V = md.V;
+__device__ void verify_greedy(const StepArgs& a, const ModelDev& md, DevState* st, Ctrl* ctl, int G, int r0,
+                              int gamma, const int* ids /*gamma draft ids*/, int pending) {
+  const int tid = threadIdx.x;
   __shared__ int s_arg[MAX_M];
-  // statistics were computed for the single row `row`, stored at index 0
+  merge_stats(md.stat_part, G, gamma + 1, ctl, ctl->rowmax, ctl->rowsum, s_arg);
+  int r = gamma;
+  for (int j = 0; j < gamma; ++j)
+    if (s_arg[j] != ids[j]) { r = j; break; }
+  if (tid == 0) commit_step(a, st, r, s_arg[r], ids, pending);
+  (void)r0;
+}
+
+// Greedy draft step j: x_j = argmax of the row whose statistics sit at index 0.
+template <int M>
+__device__ void draft_greedy(const StepArgs& a, const ModelDev& md, DevState* st, Ctrl* ctl, int G) {
+  __shared__ int s_arg[MAX_M];
   merge_stats(md.stat_part, G, 1, ctl, ctl->rowmax, ctl->rowsum, s_arg);
-  int tok;
-  if (a.greedy) {
-    tok = s_arg[0];
-  } else {
-    const float* lrow = a.logits + (size_t)row * V;
-    const float mx = ctl->rowmax[0], sm = ctl->rowsum[0], T = a.temperature;
-    float* qrow = a.q_out + (size_t)a.j * V;
-    for (int k = tid; k < V; k += CONSUMER_THREADS) stcg(qrow + k, prob_of(ldcg(lrow + k), T, mx, sm));
-    tok = block_sample([&](int k) { return prob_of(ldcg(lrow + k), T, mx, sm); }, V, u[a.j], &ctl->sc);
-  }
-  if (tid == 0) st->d_ids[a.j] = tok;
+  if (threadIdx.x == 0) st->d_ids[a.j] = s_arg[0];
 }
 
 template <int M, typename WT>
@@ -261,16 +231,10 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
         else { r0 = M - 1; nrows = 1; }
         stats_phase<M>(a.logits, md.V, r0, nrows, a.temperature, cta, G, md.stat_part, ctl);
         stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
-        if (cta == 0) {
-          const float* u = a.uniforms ? a.uniforms + (a.u_by_block ? (size_t)st->block * a.u_stride : 0) : nullptr;
-          if (a.mode == MODE_VERIFY) {
-            verify_sample<M>(a, md, st, ctl, G, 0, a.gamma, u ? u + (a.u_by_block ? a.gamma : 0) : nullptr, ctl->tok + 1,
-                             pending);
-          } else if (a.mode == MODE_DRAFT) {
-            draft_sample<M>(a, md, st, ctl, G, M - 1, u);
-          } else {
-            verify_sample<M>(a, md, st, ctl, G, M - 1, 0, u, ctl->tok, 0);
-          }
+        if (cta == 0 && a.greedy) {
+          if (a.mode == MODE_VERIFY) verify_greedy<M>(a, md, st, ctl, G, 0, a.gamma, ctl->tok + 1, pending);
+          else if (a.mode == MODE_DRAFT) draft_greedy<M>(a, md, st, ctl, G);
+          else verify_greedy<M>(a, md, st, ctl, G, M - 1, 0, ctl->tok, 0);
         }
         stamp();
       }
@@ -284,6 +248,105 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
   if (*err != DEV_OK) {
     // a wait gave up: let copies that are still in flight land before the CTA retires
     for (int i = 0; i < 200; ++i) __nanosleep(1000);
+  }
+}
+
+// ------------------------------------------------------------------------------ sampling kernels
+// Speculative sampling proper (Sec. 2.1 / Sec. 3; p = target, q = draft): accept x_j iff
+// u_j < min(1, p_j(x_j) / q_j(x_j)); the first rejected token is replaced by a draw from
+// max(0, p_r - q_r) / sum, and if none is rejected a bonus token is drawn from p_{gamma+1}.
+// The work that touches a whole vocabulary row is spread over the grid, in two small launches
+// behind the forward kernel (which has left the logits and the per-slice row statistics):
+//   sample_slices_kernel  every CTA merges the row statistics, repeats the (cheap, deterministic)
+//                         accept tests to find r, and reduces its contiguous vocabulary slice of
+//                         the weights the next token is drawn from to an integer mass; a draft
+//                         step also writes its slice of q_j = softmax(logits / T);
+//   sample_pick_kernel    one CTA finds the slice and the token, and commits the step.
+// They are separate kernels, not phases of the forward kernel, because that kernel's weight
+// streaming loop lost 1.5-2 % of its speed whenever this code was compiled into it.
+
+struct SampleShared {
+  float rowmax[MAX_M], rowsum[MAX_M];
+  int arg[MAX_M];
+  SampleScratch sc;
+};
+
+struct SamplePlan {
+  int r0, gamma;  // first row and number of draft tokens
+  int r;          // accepted draft tokens = row the next token is drawn from
+  const float* u; // uniforms of this step: gamma accept tests, then the draw
+};
+
+__device__ __forceinline__ const float* step_uniforms(const StepArgs& a, const DevState* st) {
+  const float* u = a.uniforms + (a.u_by_block ? (size_t)st->block * a.u_stride : 0);
+  return (a.mode == MODE_VERIFY && a.u_by_block) ? u + a.gamma : u;
+}
+
+// Every thread of every CTA computes the same plan (same inputs, same arithmetic).
+__device__ SamplePlan sample_plan(const StepArgs& a, const DevState* st, SampleShared* sh, int G) {
+  const int V = a.md.V;
+  SamplePlan pl;
+  pl.gamma = a.mode == MODE_VERIFY ? a.gamma : 0;
+  pl.r0 = a.mode == MODE_VERIFY ? 0 : a.sample_r0;
+  pl.u = step_uniforms(a, st);
+  merge_stats(a.md.stat_part, G, pl.gamma + 1, nullptr, sh->rowmax, sh->rowsum, sh->arg);
+  pl.r = pl.gamma;
+  for (int j = 0; j < pl.gamma; ++j) {
+    int x = st->d_ids[j];
+    if ((unsigned)x >= (unsigned)V) x = 0;   // the forward kernel has flagged it; stay in bounds
+    const float p = prob_of(ldcg(a.logits + (size_t)(pl.r0 + j) * V + x), a.temperature, sh->rowmax[j], sh->rowsum[j]);
+    const float q = ldcg(a.q_in + (size_t)j * V + x);
+    if (!accept_test(pl.u[j], p, q)) { pl.r = j; break; }
+  }
+  return pl;
+}
+
+// Calls f(weight function) with the weights of the row the next token is drawn from.
+template <class F>
+__device__ __forceinline__ void with_weights(const StepArgs& a, const SamplePlan& pl, const SampleShared* sh, F f) {
+  const int V = a.md.V;
+  const float* lrow = a.logits + (size_t)(pl.r0 + pl.r) * V;
+  const float mx = sh->rowmax[pl.r], sm = sh->rowsum[pl.r], T = a.temperature;
+  if (a.mode == MODE_DRAFT || pl.r == pl.gamma) {
+    f([=](int k) { return prob_of(ldcg(lrow + k), T, mx, sm); });
+  } else {
+    const float* qrow = a.q_in + (size_t)pl.r * V;
+    f([=](int k) { return fmaxf(0.0f, __fsub_rn(prob_of(ldcg(lrow + k), T, mx, sm), ldcg(qrow + k))); });
+  }
+}
+
+__global__ void __launch_bounds__(SAMPLE_THREADS) sample_slices_kernel(const __grid_constant__ StepArgs a) {
+  __shared__ SampleShared sh;
+  const int cta = blockIdx.x, G = gridDim.x, V = a.md.V;
+  const SamplePlan pl = sample_plan(a, a.st, &sh, G);
+  with_weights(a, pl, &sh, [&](auto wf) {
+    if (a.mode == MODE_DRAFT) {   // this CTA's slice of q_j
+      float* qrow = a.q_out + (size_t)a.j * V;
+      const int VS = (V + G - 1) / G;
+      const int k0 = cta * VS, k1 = min(V, k0 + VS);
+      for (int k = k0 + threadIdx.x; k < k1; k += SAMPLE_THREADS) stcg(qrow + k, wf(k));
+    }
+    slice_mass(wf, V, cta, G, a.md.cdf_part, &sh.sc);
+  });
+}
+
+// One CTA; G = number of slices = the grid of the two kernels before it.
+__global__ void __launch_bounds__(SAMPLE_THREADS) sample_pick_kernel(const __grid_constant__ StepArgs a, int G) {
+  __shared__ SampleShared sh;
+  DevState* st = a.st;
+  const SamplePlan pl = sample_plan(a, st, &sh, G);
+  int tok = 0;
+  with_weights(a, pl, &sh, [&](auto wf) {
+    tok = pick_from_slices(wf, a.md.V, G, a.md.cdf_part, a.mode == MODE_DRAFT ? pl.u[a.j] : pl.u[pl.gamma], &sh.sc);
+  });
+  if (threadIdx.x == 0) {
+    if (a.mode == MODE_DRAFT) {
+      st->d_ids[a.j] = tok;
+      st->t_draft1 = globaltimer();
+    } else {
+      commit_step(a, st, pl.r, tok, st->d_ids, st->pending);
+      if (a.mode == MODE_VERIFY) st->t_verify1 = globaltimer();
+    }
   }
 }
 

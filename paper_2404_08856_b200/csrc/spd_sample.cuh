@@ -109,6 +109,132 @@ __device__ int block_sample(WF wf, int V, float u, SampleScratch* sc) {
   return r;
 }
 
+// The same draw spread over the grid.  Step 1, every CTA: integer mass and largest weight of its
+// contiguous vocabulary slice [cta * VS, (cta + 1) * VS) -> part[cta].  Step 2 (after a grid
+// barrier), one CTA: the slice in which the running total crosses the threshold, then the token
+// inside it.  Integer sums make the result identical to block_sample's.
+template <class WF>
+__device__ void slice_mass(WF wf, int V, int cta, int G, unsigned long long* part, SampleScratch* sc) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int VS = (V + G - 1) / G;
+  const int k0 = cta * VS, k1 = min(V, k0 + VS);
+  unsigned long long s = 0;
+  float bm = -1.0f;
+  int bi = 0x7fffffff;
+  for (int k = k0 + tid; k < k1; k += SAMPLE_THREADS) {
+    const float w = wf(k);
+    s += to_fixed(w);
+    if (w > bm) { bm = w; bi = k; }
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) {
+    s += __shfl_xor_sync(0xffffffffu, s, o);
+    const float om = __shfl_xor_sync(0xffffffffu, bm, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (om > bm || (om == bm && oi < bi)) { bm = om; bi = oi; }
+  }
+  if (lane == 0) { sc->wsum[warp] = s; sc->amax[warp] = bm; sc->aidx[warp] = bi; }
+  named_sync(1, SAMPLE_THREADS);
+  if (tid == 0) {
+    unsigned long long z = 0;
+    float m = -1.0f;
+    int idx = 0x7fffffff;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+      z += sc->wsum[w];
+      if (sc->amax[w] > m || (sc->amax[w] == m && sc->aidx[w] < idx)) { m = sc->amax[w]; idx = sc->aidx[w]; }
+    }
+    __stcg(part + 2 * cta, z);
+    __stcg(part + 2 * cta + 1, ((unsigned long long)__float_as_uint(fmaxf(m, 0.0f)) << 32) | (unsigned)idx);
+  }
+  named_sync(1, SAMPLE_THREADS);
+}
+
+// All 256 threads of ONE CTA call this after every CTA's slice_mass is visible (grid barrier).
+template <class WF>
+__device__ int pick_from_slices(WF wf, int V, int G, const unsigned long long* part, float u, SampleScratch* sc) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int VS = (V + G - 1) / G;
+  if (tid < 32) {
+    constexpr int CH = 8;                       // up to 256 slices
+    unsigned long long v[CH];
+    unsigned long long Z = 0;
+#pragma unroll
+    for (int i = 0; i < CH; ++i) {
+      const int c = i * 32 + lane;
+      v[i] = c < G ? __ldcg(part + 2 * c) : 0ull;
+      Z += v[i];
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) Z += __shfl_xor_sync(0xffffffffu, Z, o);
+    int found;
+    if (Z == 0) {
+      // no mass at all (underflow): the largest weight, lowest index on ties
+      float bm = -1.0f;
+      int bi = 0x7fffffff;
+      for (int c = lane; c < G; c += 32) {
+        const unsigned long long pk = __ldcg(part + 2 * c + 1);
+        const float m = __uint_as_float((unsigned)(pk >> 32));
+        const int idx = (int)(unsigned)pk;
+        if (idx != 0x7fffffff && (m > bm || (m == bm && idx < bi))) { bm = m; bi = idx; }
+      }
+#pragma unroll
+      for (int o = 16; o; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, bm, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (om > bm || (om == bm && oi < bi)) { bm = om; bi = oi; }
+      }
+      found = bi == 0x7fffffff ? 0 : bi;
+    } else {
+      const unsigned long long T = threshold(Z, u);
+      unsigned long long base = 0;
+      int cs = G - 1;
+      bool hit = false;
+#pragma unroll
+      for (int i = 0; i < CH; ++i) {
+        unsigned long long inc = v[i];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned long long t = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += t;
+        }
+        const unsigned long long tot = __shfl_sync(0xffffffffu, inc, 31);
+        if (!hit && T < base + tot) {
+          const unsigned mask = __ballot_sync(0xffffffffu, base + inc > T);
+          const int l = __ffs(mask) - 1;
+          cs = i * 32 + l;
+          base += __shfl_sync(0xffffffffu, inc - v[i], l);
+          hit = true;
+        }
+        if (!hit) base += tot;
+      }
+      const int k0 = min(V, cs * VS), k1 = min(V, k0 + VS);
+      found = k1 - 1;
+      for (int kb = k0; kb < k1; kb += 32) {
+        const int k = kb + lane;
+        unsigned long long inc = (k < k1) ? to_fixed(wf(k)) : 0ull;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned long long t = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += t;
+        }
+        const unsigned long long tot = __shfl_sync(0xffffffffu, inc, 31);
+        if (T < base + tot) {
+          const unsigned mask = __ballot_sync(0xffffffffu, base + inc > T);
+          found = kb + __ffs(mask) - 1;
+          break;
+        }
+        base += tot;
+      }
+    }
+    if (lane == 0) sc->result = found;
+  }
+  named_sync(1, SAMPLE_THREADS);
+  const int r = sc->result;
+  named_sync(1, SAMPLE_THREADS);
+  return r;
+}
+
 // argmax with lowest index on ties over f(k), k < V; all 256 threads call.
 template <class F>
 __device__ int block_argmax(F f, int V, SampleScratch* sc) {
