@@ -233,7 +233,7 @@ spd_status alloc_sequence_state(spd_ctx* ctx, ModelHost& mh) {
   if ((s = dalloc(ctx, &md.aml, (size_t)H * md.nsplit * MAX_M * 2))) return s;
   if ((s = dalloc(ctx, &md.head_cnt, (size_t)H))) return s;
   if ((s = dalloc(ctx, &md.stat_part, (size_t)ctx->n_sm * MAX_M * 4))) return s;
-  if ((s = dalloc(ctx, &md.cdf_part, (size_t)ctx->n_sm * 2))) return s;
+  if ((s = dalloc(ctx, &md.cdf_part, (size_t)ctx->n_sm * 2 + 2))) return s;
   if ((s = dalloc(ctx, &mh.logits, (size_t)MAX_M * V))) return s;
   return SPD_OK;
 }

@@ -74,7 +74,8 @@ struct ModelDev {
   float *apart, *aml;                 // attention partials [H][nsplit][8][dh], [H][nsplit][8][2]
   unsigned* head_cnt;                 // [H]
   float* stat_part;                   // [grid][8][4]: row max, row sum, argmax value, argmax index
-  unsigned long long* cdf_part;       // [grid][2]: integer mass of the CTA's vocabulary slice, (max weight, index)
+  unsigned long long* cdf_part;       // [grid][2]: integer mass of the CTA's vocabulary slice, (max weight, index);
+                                      // then [2]: accepted count r, (max, sum exp) of row r for the pick kernel
   const LayerDev* layers;
 };
 

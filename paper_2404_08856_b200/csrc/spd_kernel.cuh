@@ -319,6 +319,11 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) sample_slices_kernel(const __g
   __shared__ SampleShared sh;
   const int cta = blockIdx.x, G = gridDim.x, V = a.md.V;
   const SamplePlan pl = sample_plan(a, a.st, &sh, G);
+  if (cta == 0 && threadIdx.x == 0) {   // the plan travels to the pick kernel behind the slice masses
+    __stcg(a.md.cdf_part + 2 * G, (unsigned long long)pl.r);
+    __stcg(a.md.cdf_part + 2 * G + 1,
+           ((unsigned long long)__float_as_uint(sh.rowmax[pl.r]) << 32) | __float_as_uint(sh.rowsum[pl.r]));
+  }
   with_weights(a, pl, &sh, [&](auto wf) {
     if (a.mode == MODE_DRAFT) {   // this CTA's slice of q_j
       float* qrow = a.q_out + (size_t)a.j * V;
@@ -334,7 +339,18 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) sample_slices_kernel(const __g
 __global__ void __launch_bounds__(SAMPLE_THREADS) sample_pick_kernel(const __grid_constant__ StepArgs a, int G) {
   __shared__ SampleShared sh;
   DevState* st = a.st;
-  const SamplePlan pl = sample_plan(a, st, &sh, G);
+  SamplePlan pl;   // r and the statistics of row r as the slices kernel found them
+  pl.gamma = a.mode == MODE_VERIFY ? a.gamma : 0;
+  pl.r0 = a.mode == MODE_VERIFY ? 0 : a.sample_r0;
+  pl.u = step_uniforms(a, st);
+  pl.r = (int)__ldcg(a.md.cdf_part + 2 * G);
+  if (pl.r < 0 || pl.r > pl.gamma) pl.r = pl.gamma;
+  if (threadIdx.x == 0) {
+    const unsigned long long ms = __ldcg(a.md.cdf_part + 2 * G + 1);
+    sh.rowmax[pl.r] = __uint_as_float((unsigned)(ms >> 32));
+    sh.rowsum[pl.r] = __uint_as_float((unsigned)ms);
+  }
+  named_sync(1, SAMPLE_THREADS);
   int tok = 0;
   with_weights(a, pl, &sh, [&](auto wf) {
     tok = pick_from_slices(wf, a.md.V, G, a.md.cdf_part, a.mode == MODE_DRAFT ? pl.u[a.j] : pl.u[pl.gamma], &sh.sc);
