@@ -356,6 +356,21 @@ def run_gpu(args, rank, world):
     adapter_ms = ae[0].elapsed_time(ae[1])
     adapter_flops = 2.0 * wl.n_image * (1024 * 4096 + 4096 * wl.target.d_model)
 
+    # top-k / top-p truncation of the 2*gamma+1 probability rows of one block (gamma+1 target rows,
+    # gamma draft rows), as it would sit in front of the rule; one CTA per row
+    t_logits, _ = synth.microbench_logits(1, 2 * GAMMA, wl.target.vocab, 0.5)
+    probs = torch.softmax(torch.from_numpy(t_logits[0]).cuda(), dim=-1).contiguous()
+    trunc_out = torch.empty_like(probs)
+    for _ in range(3):
+        spd.truncate_probs(probs, trunc_out, 50, 0.9)
+    te = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    te[0].record(stream)
+    for _ in range(20):
+        spd.truncate_probs(probs, trunc_out, 50, 0.9)
+    te[1].record(stream)
+    torch.cuda.synchronize()
+    truncate_ms = te[0].elapsed_time(te[1]) / 20
+
     value, ms = aggregate(float(tokens), ms, dist, "cuda")
     e2e, ms_e2e = aggregate(float(tokens_e2e), ms_e2e, dist, "cuda")
     peak, peak_kind = measured_peak()
@@ -394,6 +409,8 @@ def run_gpu(args, rank, world):
                               "tflops": adapter_flops / (adapter_ms * 1e-3) / 1e12,
                               "note": "one call = split kernel + two tcgen05 GEMMs (hi+lo activations: twice "
                                       "the flops counted) + stream synchronisation"},
+            "truncate_probs": {"ms": truncate_ms, "rows": int(probs.shape[0]), "vocab": wl.target.vocab,
+                               "top_k": 50, "top_p": 0.9, "note": "stand-alone kernel, not part of the timed block"},
             "draft_over_target_params": c_ratio,
             "setup_s": {"weights": t_gen, "first_prefill": t_prefill}}
     if rank == 0 and world == 1 and not args.layers and DRAFT == "115m" and greedy:
