@@ -447,6 +447,57 @@ def test_state_and_overflow_errors():
 # ------------------------------------------------------------------ full size
 
 @pytest.mark.gpu
+def test_llava7b_full_size_sampling_properties():
+    """Speculative sampling in the benchmark's configuration (all 32 target layers, 12 draft
+    layers, gamma 5, temperature 1), checked by properties that hold at any size: the block loop
+    through spd_generate (CUDA-graph replay) emits exactly what step-by-step spd_draft /
+    spd_verify calls emit for the same uniforms; a second run from the same state reproduces it;
+    the statistics add up (every block emits its accepted tokens plus one, at most gamma + 1); the
+    draft rows q_j handed to the rule are probability rows; each emitted draft token is one the
+    draft proposed."""
+    import torch
+    spd = _lib()
+    wl = synth.llava7b_workload(gamma=5)
+    tw, dw = H.build_weights(wl)
+    gamma, n_new = 5, 24
+    gpu = H.make_gpu(wl, tw, dw, wl.n_image + wl.n_prompt + 8 * n_new + 64, 1.0, False)
+    del tw, dw
+    img, ids = synth.image_embeds(wl), synth.prompt_ids(wl)
+    u = synth.uniforms(7, "full.sampling", (n_new, 2 * gamma + 1))
+    first = gpu.prefill(img, ids, u0=0.375)
+    n_text0, pend0 = gpu.get_state()
+    assert pend0 == first and n_text0 == len(ids)
+    out1, st1 = gpu.generate(n_new, gamma, u)
+    assert out1[0] == first and out1.min() >= 0 and out1.max() < wl.target.vocab
+    assert st1["tokens"] == n_new and st1["blocks"] >= 1
+    assert st1["blocks"] + st1["accepted"] >= n_new - 1 and st1["accepted"] <= gamma * st1["blocks"]
+    assert 1.0 <= st1["tau"] <= gamma + 1
+    # same state, same uniforms: identical output
+    gpu.rollback(n_text0, int(ids[-1]), pend0)
+    out2, st2 = gpu.generate(n_new, gamma, u)
+    assert np.array_equal(out1, out2) and st2["blocks"] == st1["blocks"] and st2["accepted"] == st1["accepted"]
+    # step by step through spd_draft / spd_verify
+    gpu.rollback(n_text0, int(ids[-1]), pend0)
+    q = torch.empty((gamma, wl.target.vocab), device="cuda", dtype=torch.float32)
+    emitted, blocks, accepted = [first], 0, 0
+    while len(emitted) < n_new:
+        d_ids = gpu.draft(gamma, u[blocks, :gamma], probs_out=q)
+        sums = q.sum(dim=1).cpu().numpy()
+        assert np.all(np.abs(sums - 1.0) < 1e-3) and float(q.min()) >= 0.0
+        assert all(float(q[j, int(d_ids[j])]) > 0.0 for j in range(gamma))
+        a, nxt = gpu.verify(gamma, u[blocks, gamma:])
+        assert 0 <= a <= gamma and 0 <= nxt < wl.target.vocab
+        emitted += [int(x) for x in d_ids[:a]] + [nxt]
+        blocks += 1
+        accepted += a
+    assert emitted[:n_new] == out1.tolist()
+    assert blocks == st1["blocks"] and accepted == st1["accepted"]
+    n_text, pend = gpu.get_state()
+    assert n_text == len(ids) + len(emitted) - 1 and pend == emitted[-1]
+    gpu.close()
+
+
+@pytest.mark.gpu
 def test_llava7b_full_size_greedy_blocks_match_oracle():
     """The benchmark's own configuration: all 32 layers of the LLaVA-7B-shaped target and the
     12-layer draft, 576 image rows + 64 prompt ids, gamma 5, greedy acceptance.  Prefill
