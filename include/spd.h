@@ -103,9 +103,9 @@ typedef struct {
 } spd_stats;
 
 /* Validates cfg, copies and repacks the weights, allocates KV caches and workspaces,
- * builds the rotary table.  Shapes must satisfy: d_model <= 4096 and a multiple of 8 per
- * head pair (d_head even), d_ffn and d_model multiples of 8, gamma_max <= 7, equal vocab
- * for both models.  *out is NULL on failure. */
+ * builds the rotary table.  Shapes must satisfy: d_model <= 4096 and a multiple of 32,
+ * d_head = d_model / n_heads in {32, 64, 128}, d_ffn a multiple of 8, gamma_max <= 7, max_seq >= 16,
+ * equal vocab for both models.  *out is NULL on failure. */
 spd_status spd_create(const spd_weights* target_w, const spd_weights* draft_w,
                       const spd_cfg* cfg, spd_ctx** out);
 void spd_destroy(spd_ctx* ctx);
@@ -131,7 +131,9 @@ spd_status spd_fork(spd_ctx* parent, spd_ctx** out);
  * when the rows are given in the draft's space, see spd_cfg.draft_adapter_in).
  *   image_embeds       fp32 [m, d_target], host or device; NULL iff m == 0
  *   draft_image_feats  fp32 [m, draft_adapter_in], host or device; NULL without adapter
- *   prompt_ids         int32 [n], host or device, n >= 1, each < vocab
+ *   prompt_ids         int32 [n], host or device, n >= 1, each in [0, vocab): host ids are checked
+ *                      before any work, device ids on the device (an offender is read as token 0,
+ *                      the call returns SPD_EINVAL and the context stays un-prefilled)
  *   u0                 host, one uniform in [0,1); may be NULL when greedy
  *   first_token        host, out, may be NULL
  * Resets any earlier sequence. SPD_EOVERFLOW if m + n + gamma_max + 1 > max_seq. */
@@ -219,7 +221,8 @@ spd_status spd_trace(spd_ctx* ctx, uint64_t* stamps, int cap, int* n);
 /* The rejection rule alone (Sec. 2.1) on given probabilities, B independent sequences:
  *   p [B, gamma+1, V], q [B, gamma, V] fp32 DEVICE (q may be NULL when greedy)
  *   ids int32 [B, gamma], u fp32 [B, gamma+1] DEVICE (u may be NULL when greedy)
- *   n_acc, next int32 [B] DEVICE, out
+ *   n_acc, next int32 [B] DEVICE, out; both are -1 for a sequence with a draft id outside [0, V)
+ *   (the ids live in device memory, so the host cannot check them before the launch)
  * Integer inverse-CDF sampling (weights truncated to 32 fractional bits, summed as
  * integers) makes the result independent of summation order. Asynchronous on stream. */
 spd_status spd_reject_sample(const float* p, const float* q, const int32_t* ids,
@@ -250,6 +253,25 @@ spd_status spd_truncate_probs(const float* probs, float* out, int rows, int V, i
  * 1 <= M <= 8, K a multiple of 8.  Asynchronous on stream. */
 spd_status spd_skinny_gemm(const float* x, const void* w, int dtype, int M, int N, int K,
                            float* y, void* stream);
+
+/* Status of the last spd_skinny_gemm (noalloc = 0) or spd_skinny_gemm_noalloc (noalloc = 1) on the
+ * current device.  Both calls are asynchronous and have no context, so a bounded device-side
+ * wait that ran out inside them (Conventions above) can only be seen afterwards: this call
+ * synchronises `stream`, returns SPD_ETIMEOUT if the kernel's status word is set (y is then
+ * garbage) and clears it, else SPD_OK; SPD_ESTATE before the first such call on this device.
+ * spd_skinny_gemm_noalloc clears its status word at the start of every call, so ask before the
+ * next call; spd_skinny_gemm's stays set (and its results garbage) until it is asked for. */
+spd_status spd_skinny_gemm_status(int noalloc, void* stream);
+
+/* Bounded waits, exercised (no counterpart in the paper; Conventions: no call may hang the
+ * device).  Launches a small kernel on the context's stream that runs one of the forward
+ * kernel's wait primitives on a condition that never becomes true, limited to `polls`
+ * iterations (1 .. 2^20): which = 0 the shared-memory barrier wait of the weight ring, which = 1
+ * the grid barrier with a target one arrival beyond the grid size.  The wait gives up, the
+ * kernel returns normally and this call returns SPD_ETIMEOUT -- the status any call of this
+ * library reports when one of its waits runs out.  The error word is cleared; the context and
+ * its sequence are untouched and stay usable.  Synchronises the stream. */
+spd_status spd_wait_selftest(spd_ctx* ctx, int which, unsigned polls);
 
 /* The same product as spd_skinny_gemm for callers that must not allocate device memory.
  * (The paper has no counterpart for this entry point; it exists for integration reasons.)

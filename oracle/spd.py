@@ -78,19 +78,6 @@ class SpdOracle:
         self.n_prompt = len(prompt_ids)
         return x0
 
-    def set_state(self, seq):
-        """Replace the committed sequence (prompt + emitted tokens) by one that shares a
-        prefix with the current one; caches keep the rows of the shared prefix."""
-        seq = [int(x) for x in seq]
-        common = 0
-        for a, b in zip(seq, self.seq):
-            if a != b:
-                break
-            common += 1
-        self.d_fed = min(self.d_fed, common, len(seq) - 1)
-        self.seq = seq
-        self.tc.length = self.m + len(seq) - 1
-
     # ---- step 2
     def draft(self, gamma: int, u_draft):
         ids, probs, raw, used = [], [], [], []

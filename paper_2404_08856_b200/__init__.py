@@ -21,7 +21,8 @@ STATUS_NAMES = ["SPD_OK", "SPD_EINVAL", "SPD_ESTATE", "SPD_ENOMEM", "SPD_EOVERFL
 EXPORTS = ["spd_create", "spd_destroy", "spd_fork", "spd_last_error", "spd_prefill", "spd_draft", "spd_verify",
            "spd_generate", "spd_get_logits", "spd_get_draft_logits", "spd_rollback", "spd_get_state",
            "spd_reject_sample", "spd_skinny_gemm", "spd_verify_bytes", "spd_trace",
-           "spd_skinny_gemm_noalloc", "spd_image_adapter", "spd_truncate_probs"]
+           "spd_skinny_gemm_noalloc", "spd_image_adapter", "spd_truncate_probs", "spd_skinny_gemm_status",
+           "spd_wait_selftest"]
 
 
 class SpdError(RuntimeError):
@@ -177,7 +178,8 @@ class Spd:
 
     def verify(self, gamma: int, uniforms=None, draft_ids=None, draft_probs=None):
         u = None if uniforms is None else np.ascontiguousarray(uniforms, dtype=np.float32)
-        ids = None if draft_ids is None else np.ascontiguousarray(draft_ids, dtype=np.int32)
+        ids = draft_ids if (draft_ids is None or hasattr(draft_ids, "data_ptr")) \
+            else np.ascontiguousarray(draft_ids, dtype=np.int32)
         a, nxt = C.c_int32(0), C.c_int32(0)
         self._check(lib().spd_verify(self._ctx, gamma, _ptr(ids), _ptr(draft_probs), _ptr(u), C.byref(a),
                                      C.byref(nxt)))
@@ -226,6 +228,11 @@ class Spd:
         self._check(lib().spd_trace(self._ctx, _ptr(out), 1024, C.byref(n)))
         return out[: n.value].copy()
 
+    def wait_selftest(self, which: int, polls: int = 2000) -> int:
+        """Runs a bounded device-side wait that cannot succeed (see spd_wait_selftest) and returns
+        the status the library reports for it (SPD_ETIMEOUT when the give-up path works)."""
+        return int(lib().spd_wait_selftest(self._ctx, int(which), C.c_uint(polls)))
+
     def verify_bytes(self, gamma: int) -> float:
         b = C.c_double(0)
         self._check(lib().spd_verify_bytes(self._ctx, gamma, C.byref(b)))
@@ -258,6 +265,11 @@ def skinny_gemm(x, w, y, dtype: int, stream: int = 0):
     st = lib().spd_skinny_gemm(_ptr(x), _ptr(w), dtype, M, N, K, _ptr(y), C.c_void_p(stream))
     if st != SPD_OK:
         raise SpdError(st, "spd_skinny_gemm")
+
+
+def skinny_gemm_status(noalloc: bool, stream: int = 0) -> int:
+    """Status of the last stand-alone GEMM call on the current device (see spd_skinny_gemm_status)."""
+    return int(lib().spd_skinny_gemm_status(int(noalloc), C.c_void_p(stream)))
 
 
 NOALLOC_MAX_PACKED_BYTES = 16 << 20

@@ -388,9 +388,17 @@ KernelFn pick_kernel(int M, int dtype) { return dtype == 1 ? pick_m<__nv_bfloat1
 
 struct LaunchCfg { int nstage; size_t smem; };
 
+constexpr int MAX_DEV = 64;   // devices per process that the per-device tables below cover
+
 spd_status launch_cfg(spd_ctx* ctx, KernelFn fn, int M, int n_sm, int smem_optin, LaunchCfg* lc) {
-  static LaunchCfg cache[2 * (MAX_M + 1)];   // per kernel variant; filled on first use
-  static KernelFn cache_fn[2 * (MAX_M + 1)];
+  // per device and kernel variant; filled on first use (the shared-memory attribute of a kernel
+  // belongs to the device it was set on)
+  static LaunchCfg cache_all[MAX_DEV][2 * (MAX_M + 1)];
+  static KernelFn cache_fn_all[MAX_DEV][2 * (MAX_M + 1)];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEV) return fail(ctx, SPD_ECUDA, "no current device");
+  LaunchCfg* cache = cache_all[dev];
+  KernelFn* cache_fn = cache_fn_all[dev];
   for (int i = 0; i < 2 * (MAX_M + 1); ++i)
     if (cache_fn[i] == fn) { *lc = cache[i]; return SPD_OK; }
   cudaFuncAttributes fa{};
@@ -545,11 +553,12 @@ spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const
   if ((s = make_map(ctx, &ma, a_hi.ptr, a_hi.inner, a_hi.rows, a_hi.batch, a_hi.row_stride, a_hi.batch_stride))) return s;
   if ((s = make_map(ctx, &ml, a_lo.ptr, a_lo.inner, a_lo.rows, a_lo.batch, a_lo.row_stride, a_lo.batch_stride))) return s;
   if ((s = make_map(ctx, &mb, b.ptr, b.inner, b.rows, b.batch, b.row_stride, b.batch_stride))) return s;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[MAX_DEV];
+  if (ctx->device < 0 || ctx->device >= MAX_DEV) return fail(ctx, SPD_ECUDA, "device index out of range");
+  if (!attr_set[ctx->device]) {
     CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
     CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
-    attr_set = true;
+    attr_set[ctx->device] = true;
   }
   args.split = 1;
   args.err = &ctx->st->err;
@@ -560,11 +569,18 @@ spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const
   return SPD_OK;
 }
 
-__global__ void gather_rows_kernel(const int* ids, const float* table, float* out, int n, int d) {
+// Embedding rows of n token ids.  An id outside [0, V) (possible when the ids live in device
+// memory, which the host cannot inspect) is read as token 0 and recorded in *err.
+__global__ void gather_rows_kernel(const int* ids, const float* table, float* out, int n, int d, int V, int* err) {
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < (size_t)n * (d >> 2);
        i += (size_t)gridDim.x * blockDim.x) {
     const int r = (int)(i / (d >> 2)), c = (int)(i - (size_t)r * (d >> 2));
-    reinterpret_cast<float4*>(out + (size_t)r * d)[c] = reinterpret_cast<const float4*>(table + (size_t)ids[r] * d)[c];
+    int id = ids[r];
+    if ((unsigned)id >= (unsigned)V) {
+      if (c == 0) atomicCAS(err, DEV_OK, DEV_BAD_TOKEN);
+      id = 0;
+    }
+    reinterpret_cast<float4*>(out + (size_t)r * d)[c] = reinterpret_cast<const float4*>(table + (size_t)id * d)[c];
   }
 }
 
@@ -665,14 +681,9 @@ spd_status alloc_ctx_buffers(spd_ctx* ctx) {
   return SPD_OK;
 }
 
-bool use_tc_prefill(const ModelHost& mh) {
-  static int forced = -1;   // SPD_PREFILL=rows keeps the 8-row kernel (comparison runs)
-  if (forced < 0) {
-    const char* e = getenv("SPD_PREFILL");
-    forced = (e && !strcmp(e, "rows")) ? 1 : 0;
-  }
-  return !forced && mh.cfg.dtype == 1;
-}
+// bf16 models take the dense tensor-core prefill; fp32 models go through the M <= 8 kernel in
+// chunks of 8 rows.
+bool use_tc_prefill(const ModelHost& mh) { return mh.cfg.dtype == 1; }
 
 }  // namespace
 
@@ -852,13 +863,14 @@ spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m, const flo
                        {dm.adapter_rm, ad, dd, 1, (size_t)ad * 2, (size_t)dd * ad * 2}, a))) return s;
       dm.pos_base = m;
     }
-    gather_rows_kernel<<<592, 256, 0, ctx->stream>>>(ctx->ids_dev, dm.md.embed, X + (size_t)dm.pos_base * dd, n, dd);
+    gather_rows_kernel<<<592, 256, 0, ctx->stream>>>(ctx->ids_dev, dm.md.embed, X + (size_t)dm.pos_base * dd, n, dd, V,
+                                                       &ctx->st->err);
     if ((s = prefill_tc(ctx, dm, X, Rd))) return s;
     // ---- target rows [V_1..V_m ; embed(prompt)] (Eq. 1); last row -> first generated token
     tm.pos_base = m;
     if (m > 0)
       CU(cudaMemcpyAsync(X, image_embeds, (size_t)m * dt * sizeof(float), cudaMemcpyDefault, ctx->stream));
-    gather_rows_kernel<<<592, 256, 0, ctx->stream>>>(ctx->ids_dev, tm.md.embed, X + (size_t)m * dt, n, dt);
+    gather_rows_kernel<<<592, 256, 0, ctx->stream>>>(ctx->ids_dev, tm.md.embed, X + (size_t)m * dt, n, dt, V, &ctx->st->err);
     if ((s = prefill_tc(ctx, tm, X, Rt))) return s;
     CU(cudaMemcpyAsync(tm.md.x, X + (size_t)(Rt - 1) * dt, dt * sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));
     StepArgs a = base_args(ctx, tm);
@@ -899,7 +911,7 @@ spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m, const flo
   }
   if ((s = feed_rows(ctx, tm, nullptr, ctx->ids_dev, 0, n, m, true, n, last_id))) return s;
   }
-  ctx->prefilled = true;
+  ctx->prefilled = false;   // until the device has reported no error below
   ctx->drafted_gamma = -1;
   ctx->n_prompt = n; ctx->m_image = m;
   ctx->last_verify_rows = 1; ctx->last_draft_rows = 0;
@@ -910,6 +922,7 @@ spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m, const flo
       CU(cudaMemcpyAsync(tm.logits, tm.logits + (size_t)(lastM - 1) * V, V * sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));
   }
   if ((s = sync_state(ctx))) return s;
+  ctx->prefilled = true;
   if (first_token) *first_token = ctx->st_host->pending;
   return SPD_OK;
 }
@@ -1236,42 +1249,71 @@ spd_status spd_truncate_probs(const float* probs, float* out, int rows, int V, i
   return cudaGetLastError() == cudaSuccess ? SPD_OK : SPD_ECUDA;
 }
 
+// Scratch of the two stand-alone GEMM entry points, per device: a grid-barrier word, a status
+// block (DevState: only its error word is used) and, for spd_skinny_gemm, the tile-packed copy of w.
+struct GemmScratch {
+  bool ready = false;
+  unsigned* bar = nullptr;
+  DevState* st = nullptr;
+  char* packed = nullptr;
+  size_t packed_cap = 0;
+  int n_sm = 0, smem_optin = 0;
+};
+static GemmScratch g_gemm_scratch[MAX_DEV];      // spd_skinny_gemm (allocated on first use)
+static GemmScratch g_noalloc_state[MAX_DEV];     // spd_skinny_gemm_noalloc (points into g_noalloc_scratch)
+
 spd_status spd_skinny_gemm(const float* x, const void* w, int dtype, int M, int N, int K, float* y, void* stream) {
   if (!x || !w || !y || M < 1 || M > MAX_M || N < 1 || K < 8 || K % 8 || (dtype != 0 && dtype != 1)) return SPD_EINVAL;
-  // per-process scratch: a grid-barrier word, a status block and the tile-packed copy of w
-  static unsigned* bar = nullptr;
-  static DevState* st = nullptr;
-  static char* packed = nullptr;
-  static size_t packed_cap = 0;
-  static int n_sm = 0, smem_optin = 0;
   spd_ctx* ctx = nullptr;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  if (!bar) {
-    int dev = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEV) return SPD_ECUDA;
+  GemmScratch& g = g_gemm_scratch[dev];
+  if (!g.ready) {
     cudaDeviceProp prop{};
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return SPD_ECUDA;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return SPD_ECUDA;
     if (prop.major != 10) return SPD_ECUDA;
-    n_sm = prop.multiProcessorCount;
-    smem_optin = (int)prop.sharedMemPerBlockOptin;
-    if (cudaMalloc(&bar, 256) != cudaSuccess || cudaMalloc(&st, sizeof(DevState)) != cudaSuccess) return SPD_ENOMEM;
-    cudaMemset(st, 0, sizeof(DevState));
+    unsigned* bar = nullptr;
+    DevState* st = nullptr;
+    if (cudaMalloc(&bar, 256) != cudaSuccess) return SPD_ENOMEM;
+    if (cudaMalloc(&st, sizeof(DevState)) != cudaSuccess) { cudaFree(bar); return SPD_ENOMEM; }
+    if (cudaMemset(st, 0, sizeof(DevState)) != cudaSuccess) { cudaFree(bar); cudaFree(st); return SPD_ECUDA; }
+    g.bar = bar; g.st = st;
+    g.n_sm = prop.multiProcessorCount;
+    g.smem_optin = (int)prop.sharedMemPerBlockOptin;
+    g.ready = true;   // only now: a failed set-up is repeated by the next call
   }
   const size_t esz = dtype == 1 ? 2 : 4;
   const size_t need = packed_bytes(N, K, esz);
-  if (need > packed_cap) {
+  if (need > g.packed_cap) {
     cudaStreamSynchronize(cs);
-    if (packed) cudaFree(packed);
-    packed = nullptr; packed_cap = 0;
-    if (cudaMalloc(&packed, need) != cudaSuccess) return SPD_ENOMEM;
-    packed_cap = need;
+    if (g.packed) cudaFree(g.packed);
+    g.packed = nullptr; g.packed_cap = 0;
+    if (cudaMalloc(&g.packed, need) != cudaSuccess) return SPD_ENOMEM;
+    g.packed_cap = need;
   }
-  spd_status s = pack_tiles(ctx, packed, w, N, K, esz, n_sm, cs);
+  spd_status s = pack_tiles(ctx, g.packed, w, N, K, esz, g.n_sm, cs);
   if (s) return s;
   StepArgs a{};
   a.mode = MODE_GEMM;
-  a.st = st;
-  a.gx = x; a.gw = packed; a.gy = y; a.gN = N; a.gK = K;
-  return launch_forward(ctx, M, dtype, a, cs, n_sm, smem_optin, bar);
+  a.st = g.st;
+  a.gx = x; a.gw = g.packed; a.gy = y; a.gN = N; a.gK = K;
+  return launch_forward(ctx, M, dtype, a, cs, g.n_sm, g.smem_optin, g.bar);
+}
+
+spd_status spd_skinny_gemm_status(int noalloc, void* stream) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEV) return SPD_ECUDA;
+  const GemmScratch& g = noalloc ? g_noalloc_state[dev] : g_gemm_scratch[dev];
+  if (!g.ready) return SPD_ESTATE;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  int e = 0;
+  if (cudaMemcpyAsync(&e, &g.st->err, sizeof(int), cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
+      cudaStreamSynchronize(cs) != cudaSuccess)
+    return SPD_ECUDA;
+  if (e == DEV_OK) return SPD_OK;
+  cudaMemsetAsync(&g.st->err, 0, sizeof(int), cs);
+  return SPD_ETIMEOUT;
 }
 
 spd_status spd_skinny_gemm_noalloc(const float* x, const void* w, int dtype, int M, int N, int K, float* y,
@@ -1286,33 +1328,44 @@ spd_status spd_skinny_gemm_noalloc(const float* x, const void* w, int dtype, int
   }
   // Per-device set-up on the first call with that device current: the array's name is only a
   // host-side handle, the device address comes from the runtime.
-  constexpr int MAX_DEV = 64;
-  static unsigned char* base[MAX_DEV];
-  static int n_sm[MAX_DEV], smem_optin[MAX_DEV];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEV) return SPD_ECUDA;
-  if (!base[dev]) {
+  GemmScratch& g = g_noalloc_state[dev];
+  if (!g.ready) {
     cudaDeviceProp prop{};
     if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess || prop.major != 10) return SPD_ECUDA;
     unsigned char* ptr = nullptr;
     if (cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return SPD_ECUDA;
-    n_sm[dev] = prop.multiProcessorCount;
-    smem_optin[dev] = (int)prop.sharedMemPerBlockOptin;
-    base[dev] = ptr;
+    g.n_sm = prop.multiProcessorCount;
+    g.smem_optin = (int)prop.sharedMemPerBlockOptin;
+    g.bar = reinterpret_cast<unsigned*>(ptr);
+    g.st = reinterpret_cast<DevState*>(ptr + 256);
+    g.packed = reinterpret_cast<char*>(ptr + NOALLOC_HEADER);
+    g.packed_cap = SPD_NOALLOC_MAX_PACKED_BYTES;
+    g.ready = true;
   }
   spd_ctx* ctx = nullptr;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  unsigned char* sc = base[dev];
   // the array keeps whatever the last call left: the barrier word and the status block must
   // start at zero (launch_forward clears the barrier word, the status block is cleared here)
-  if (cudaMemsetAsync(sc + 256, 0, 256, cs) != cudaSuccess) return SPD_ECUDA;
-  spd_status s = pack_tiles(ctx, sc + NOALLOC_HEADER, w, N, K, esz, n_sm[dev], cs);
+  if (cudaMemsetAsync(g.st, 0, 256, cs) != cudaSuccess) return SPD_ECUDA;
+  spd_status s = pack_tiles(ctx, g.packed, w, N, K, esz, g.n_sm, cs);
   if (s) return s;
   StepArgs a{};
   a.mode = MODE_GEMM;
-  a.st = reinterpret_cast<DevState*>(sc + 256);
-  a.gx = x; a.gw = sc + NOALLOC_HEADER; a.gy = y; a.gN = N; a.gK = K;
-  return launch_forward(ctx, M, dtype, a, cs, n_sm[dev], smem_optin[dev], reinterpret_cast<unsigned*>(sc));
+  a.st = g.st;
+  a.gx = x; a.gw = g.packed; a.gy = y; a.gN = N; a.gK = K;
+  return launch_forward(ctx, M, dtype, a, cs, g.n_sm, g.smem_optin, g.bar);
+}
+
+spd_status spd_wait_selftest(spd_ctx* ctx, int which, unsigned polls) {
+  if (!ctx) return SPD_EINVAL;
+  if ((which != 0 && which != 1) || polls < 1 || polls > (1u << 20)) return fail(ctx, SPD_EINVAL, "bad selftest arguments");
+  unsigned* bar = next_bar(ctx);
+  CU(cudaMemsetAsync(bar, 0, sizeof(unsigned), ctx->stream));
+  wait_selftest_kernel<<<ctx->n_sm, CONSUMER_THREADS, 0, ctx->stream>>>(ctx->st, bar, which, polls);
+  CU(cudaGetLastError());
+  return sync_state(ctx);   // reads the error word, clears it, maps it to SPD_ETIMEOUT
 }
 
 spd_status spd_verify_bytes(spd_ctx* ctx, int gamma, double* bytes) {

@@ -47,8 +47,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
 }
 // Bounded wait: returns false (and records `code`) if the phase never completes or if
 // another wait already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, volatile int* err, int code) {
-  for (unsigned it = 0; it < SPIN_LIMIT_MBAR; ++it) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, volatile int* err, int code,
+                                          unsigned limit = SPIN_LIMIT_MBAR) {
+  for (unsigned it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 1023u) == 1023u && *err != DEV_OK) return false;
   }

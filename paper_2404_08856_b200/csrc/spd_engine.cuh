@@ -92,6 +92,7 @@ struct DevState {
   // %globaltimer (ns) at the start / end of the last draft steps and verify step
   unsigned long long t_draft0, t_draft1, t_verify0, t_verify1;
 };
+static_assert(sizeof(DevState) <= 256, "the fixed scratch of spd_skinny_gemm_noalloc reserves 256 bytes for it");
 
 struct StepArgs {
   ModelDev md;            // by value: read through the constant bank
@@ -658,14 +659,15 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, const XSrc& src, c
 
 // ------------------------------------------------------------------------------ grid barrier
 
-__device__ __forceinline__ void grid_barrier(unsigned* counter, unsigned& target, unsigned G, volatile int* err) {
+__device__ __forceinline__ void grid_barrier(unsigned* counter, unsigned& target, unsigned G, volatile int* err,
+                                             unsigned limit = SPIN_LIMIT_GRID) {
   named_sync(1, CONSUMER_THREADS);
   if (threadIdx.x == 0) {
     target += G;
     asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(counter) : "memory");
     unsigned it = 0;
     while (ld_acquire(counter) < target) {
-      if (++it > SPIN_LIMIT_GRID || ((it & 255u) == 0 && *err != DEV_OK)) {
+      if (++it > limit || ((it & 255u) == 0 && *err != DEV_OK)) {
         atomicCAS(const_cast<int*>(err), DEV_OK, DEV_TIMEOUT_GRID);
         break;
       }

@@ -251,6 +251,26 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
   }
 }
 
+// ------------------------------------------------------------------------------ bounded waits, exercised
+// Runs the two wait primitives of the forward kernel on conditions that never come true, with a
+// small poll limit, so that the give-up path (sticky error word, normal return) can be checked on
+// a healthy device: which = 0 waits for a phase of a shared-memory barrier nobody arrives at,
+// which = 1 enters a grid barrier whose target is one arrival more than the grid will ever make.
+// Nothing here can wait longer than `limit` polls.
+__global__ void __launch_bounds__(CONSUMER_THREADS) wait_selftest_kernel(DevState* st, unsigned* bar, int which,
+                                                                         unsigned limit) {
+  __shared__ uint64_t never;
+  volatile int* err = &st->err;
+  if (threadIdx.x == 0) { mbar_init(&never, 1); mbar_fence_init(); }
+  __syncthreads();
+  if (which == 0) {
+    if (threadIdx.x < 32) mbar_wait(&never, 0u, err, DEV_TIMEOUT_FULL, limit);
+  } else {
+    unsigned target = 1;   // grid_barrier adds G: G arrivals can never reach G + 1
+    grid_barrier(bar, target, gridDim.x, err, limit);
+  }
+}
+
 // ------------------------------------------------------------------------------ sampling kernels
 // Speculative sampling proper (Sec. 2.1 / Sec. 3; p = target, q = draft): accept x_j iff
 // u_j < min(1, p_j(x_j) / q_j(x_j)); the first rejected token is replaced by a draw from

@@ -279,6 +279,13 @@ reject_sample_kernel(const float* __restrict__ p, const float* __restrict__ q, c
   const int* idb = ids + (size_t)b * gamma;
   const float* ub = u ? u + (size_t)b * (gamma + 1) : nullptr;
   int r = gamma, tok;
+  // a draft id outside [0, V) cannot index a row: the sequence is reported as n_acc = next = -1
+  bool bad = false;
+  for (int j = 0; j < gamma; ++j) bad |= (unsigned)idb[j] >= (unsigned)V;
+  if (bad) {
+    if (threadIdx.x == 0) { n_acc[b] = -1; next[b] = -1; }
+    return;
+  }
   if (greedy) {
     tok = -1;
     for (int j = 0; j <= gamma; ++j) {

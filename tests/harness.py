@@ -2,11 +2,16 @@
 the same seeded inputs, and drive both in lock-step.
 
 Sampling decisions compare a floating-point quantity with a uniform.  The two sides agree
-bit for bit only when that quantity is not within rounding distance of the uniform, so the
-harness lets the ORACLE choose each uniform from a seeded stream and skip candidates that
-fall too close to a decision boundary (the margins below).  Inputs therefore depend on the
-oracle and the seed only, never on the CUDA path, and every compared decision has exactly
-one correct answer.
+bit for bit only when that quantity is not within rounding distance of the uniform.  Two
+uniform sources exist:
+
+* SafeUniforms: the ORACLE chooses each uniform from a seeded stream and skips candidates that
+  fall inside the stated tolerance of a decision boundary: |u - min(1, p/q)| <= 1e-4 for an
+  accept test (the tolerance this path is held to), 2e-6 * Z around a CDF step for a draw.
+  Inputs depend on the oracle and the seed only, never on the CUDA path, and every compared
+  decision then has exactly one answer inside the tolerance.
+* PlainUniforms: the seeded stream taken as it is.  A differing decision must then lie inside
+  the tolerance (checked by the caller with the helpers below) and is counted.
 """
 from __future__ import annotations
 
@@ -17,6 +22,8 @@ from oracle import llama, sampling as S
 from oracle.spd import SpdOracle
 
 F32 = np.float32
+ACCEPT_TOL = 1e-4          # accept/reject decisions may differ only where |u - min(1, p/q)| < 1e-4
+CDF_TOL_FP32 = 2.0 ** -20  # fp32 models: a drawn token may differ only if u*Z is this close (x Z) to a CDF step
 
 
 def build_weights(wl, std=0.02):
@@ -43,7 +50,7 @@ class SafeUniforms:
     """Seeded stream of uniforms on the 2^-24 grid from which the oracle side picks the
     first candidate that keeps a decision away from its boundary."""
 
-    def __init__(self, seed, tag, accept_margin=2e-3, cdf_margin=2e-6, n=1 << 16):
+    def __init__(self, seed, tag, accept_margin=ACCEPT_TOL, cdf_margin=2e-6, n=1 << 16):
         self.pool = synth.uniforms(seed, tag, n)
         self.i = 0
         self.skipped = 0
@@ -93,6 +100,33 @@ class SafeUniforms:
         w = p[gamma] if r == gamma else np.maximum(F32(0), p[r] - q[r])
         u[gamma] = self.for_cdf(w)
         return u
+
+
+class PlainUniforms(SafeUniforms):
+    """The seeded stream as it is: no candidate is skipped."""
+
+    def for_cdf(self, w):
+        return self._next()
+
+    def for_accept(self, p_x, q_x):
+        return self._next()
+
+
+def accept_distance(p_x, q_x, u):
+    """|u - min(1, p/q)| with the oracle's values: how far a uniform is from flipping the test."""
+    return abs(float(u) - float(S.accept_prob(p_x, q_x)))
+
+
+def cdf_band(fp32_model, err_p, err_q=0.0, residual_mass=1.0):
+    """Relative half-width (in units of Z) of the region around a CDF step in which the two sides
+    may draw neighbouring tokens.  A logit error eps moves every probability by a factor within
+    exp(+-2 eps), so a normalised prefix sum of a softmax row moves by at most 2 eps; for the
+    residual max(0, p - q) the weights move by 2 eps_p p + 2 eps_q q and are normalised by the
+    residual's own mass, which gives 2 (eps_p + eps_q) / mass.  fp32 models are held to the fixed
+    2^-20 instead (their logit error is ~1e-5, below the skip margin of SafeUniforms)."""
+    if fp32_model:
+        return CDF_TOL_FP32
+    return 2.0 * (err_p + err_q) / max(residual_mass, 1e-6) + 1e-6
 
 
 def top2_gap(row):

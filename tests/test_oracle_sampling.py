@@ -217,3 +217,29 @@ def test_mbsu_reading():
     c = 115e6 / 6.74e9
     assert 2.3 < mbsu(2.5, c, 3) < 2.4
     assert c * 2.5 / (c * 3 + 1) < 0.05
+
+
+def test_batch_form_is_the_rule_applied_to_each_sequence():
+    """reject_sample_batch (the expected value of the bit-exact device tests) must be nothing but
+    reject_sample per sequence: checked on sequences whose outcome is known in closed form --
+    identical rows accept everything, disjoint supports reject at once, and a dyadic pair whose
+    accept probability 1/2 is decided by the uniform -- stacked in one batch, sampling and greedy."""
+    V, gamma = 8, 2
+    e = lambda k: np.eye(V, dtype=F32)[k]
+    half = (e(0) + e(1)) * F32(0.5)
+    p = np.stack([np.stack([half] * 3), np.stack([e(3)] * 3), np.stack([e(0), e(0), e(0)]),
+                  np.stack([(e(0) + e(2)) * F32(0.5)] * 3)])
+    q = np.stack([np.stack([half] * 2), np.stack([e(4)] * 2), np.stack([e(0), e(0)]), np.stack([e(0)] * 2)])
+    ids = np.array([[0, 1], [4, 4], [0, 0], [0, 0]], np.int32)
+    u = np.array([[0.9, 0.9, 0.75], [0.0, 0.0, 0.5], [0.5, 0.5, 0.1], [0.25, 0.75, 0.3]], F32)
+    a, n = S.reject_sample_batch(p, q, ids, u)
+    # seq 0: p == q, all accepted, bonus from (1/2, 1/2) at u = .75 -> token 1
+    # seq 1: p(x) = 0 -> rejected at once, residual = p -> token 3
+    # seq 2: p == q point masses -> all accepted, bonus token 0
+    # seq 3: p/q = 1/2: u = .25 accepts, u = .75 rejects; residual = (0, 0, 1/2) -> token 2
+    assert a.tolist() == [2, 0, 2, 1] and n.tolist() == [1, 3, 0, 2]
+    for b in range(4):
+        assert (a[b], n[b]) == S.reject_sample(p[b], q[b], ids[b], u[b])
+    ag, ng = S.reject_sample_batch(p, None, ids, None, greedy=True)
+    assert ag.tolist() == [1, 0, 2, 2] and ng.tolist() == [0, 3, 0, 0]
+    assert a.dtype == np.int32 and n.dtype == np.int32

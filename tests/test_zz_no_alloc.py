@@ -5,9 +5,11 @@ cudaFree: programs whose device memory belongs to another allocator, latency-cri
 loops that cannot afford the device-wide synchronisation an allocation implies, processes
 with a memory budget fixed at start-up.  It keeps its scratch (barrier word, status block,
 repacked weights) in a fixed array inside the library, shared by all calls.  This test calls
-it twice in a row with different shapes and data -- the second call sees whatever the first
-left in the scratch -- and compares each result with spd_skinny_gemm on the same inputs,
-then checks that a matrix too large for the fixed scratch is refused.
+it several times in a row with different shapes and data -- each call sees whatever the one
+before left in the scratch -- and compares each result with spd_skinny_gemm on the same inputs
+and with an fp64 matrix product, checks that a warmed call leaves the amount of free device
+memory exactly as it found it, that its status word reads clean afterwards, and that a matrix
+too large for the fixed scratch is refused.
 
 The file name sorts last on purpose: a run that stops at the first failure has then
 already run every other test.
@@ -44,12 +46,21 @@ def test_noalloc_gemm_matches_regular_entry_point_twice_in_a_row():
         y_ref = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
         y_new = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
         spd.skinny_gemm(xd, wd, y_ref, dtype)
-        spd.skinny_gemm_noalloc(xd, wd, y_new, dtype)
+        spd.skinny_gemm_noalloc(xd, wd, y_new, dtype)      # the first call per device does the set-up
         torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        y_new.fill_(float("nan"))
+        spd.skinny_gemm_noalloc(xd, wd, y_new, dtype)      # warmed: must not allocate or free anything
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
+        assert spd.skinny_gemm_status(True) == spd.SPD_OK and spd.skinny_gemm_status(False) == spd.SPD_OK
         ref, new = y_ref.cpu().numpy(), y_new.cpu().numpy()
         assert np.isfinite(new).all()
         # same kernel, same arithmetic: the tolerance of the GEMM parity test is ample
         assert np.abs(new - ref).max() < 2e-4 * np.sqrt(K) * 0.05
+        w_used = synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(w)) if dtype == 1 else w
+        want = x.astype(np.float64) @ w_used.astype(np.float64).T
+        assert np.abs(new - want).max() < 2e-4 * np.sqrt(K) * 0.05
 
 
 @pytest.mark.gpu
