@@ -73,6 +73,12 @@ typedef struct {
                            already in the draft's embedding space, e.g. the output of the
                            draft's own two-layer adapter (Appendix A.1) from spd_image_adapter */
   void* stream;         /* cudaStream_t, may be NULL (legacy default stream) */
+  int grid_mode;        /* launch shape of the decode kernel.  0 or 1: one CTA per SM with a barrier in
+                           global memory (the default and the measured best for both model sizes);
+                           2: each model runs as one thread-block cluster of 16 CTAs (8 if 16 cannot be
+                           placed) that synchronise through each other's shared memory -- cheaper
+                           barriers, but only 16 SMs' worth of streaming (115M draft: 0.61 ms per step
+                           against 0.31 ms).  Results do not depend on it beyond summation order. */
 } spd_cfg;
 
 /* Host or device pointers; per-layer entries are HOST arrays of n_layers pointers. */

@@ -33,6 +33,8 @@ struct ModelHost {
   std::vector<RowMajor> rm;
   __nv_bfloat16* adapter_rm = nullptr;
   bool rows_given = false;  // draft only: the image rows arrive already in the draft's space
+  int grid = 0;             // CTAs of this model's forward launches (its weights are packed for that count)
+  int cluster = 0;          // > 0: those CTAs form one thread-block cluster of this size
 };
 
 }  // namespace
@@ -247,7 +249,7 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
   const int max_seq = ctx->cfg.max_seq;
   ModelDev& md = mh.md;
   md.L = L; md.d = d; md.H = H; md.dh = dh; md.f = f; md.V = V; md.max_seq = max_seq;
-  md.nsplit = ctx->n_sm / H > 0 ? ctx->n_sm / H : 1;
+  md.nsplit = mh.grid / H > 0 ? mh.grid / H : 1;
   md.eps = c.rms_eps;
   md.scale = (float)(1.0 / sqrt((double)dh));
   spd_status s;
@@ -269,7 +271,7 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
     char* lm = nullptr;
     if ((s = dalloc(ctx, &lm, packed_bytes(V, d, esz)))) return s;
     if ((s = put_rows(ctx, rm, c.tied_embeddings ? w->tok_embed : w->lm_head, staging, V, d, esz, 1, 0, 0))) return s;
-    if ((s = pack_tiles(ctx, lm, rm, V, d, esz, ctx->n_sm, ctx->stream))) return s;
+    if ((s = pack_tiles(ctx, lm, rm, V, d, esz, mh.grid, ctx->stream))) return s;
     md.lm_head = lm;
   }
   float* fn = nullptr;
@@ -283,7 +285,7 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
     char* ad = nullptr;
     if ((s = dalloc(ctx, &ad, packed_bytes(d, adapter_in, esz)))) return s;
     if ((s = put_rows(ctx, rm, w->adapter, staging, d, adapter_in, esz, 1, 0, 0))) return s;
-    if ((s = pack_tiles(ctx, ad, rm, d, adapter_in, esz, ctx->n_sm, ctx->stream))) return s;
+    if ((s = pack_tiles(ctx, ad, rm, d, adapter_in, esz, mh.grid, ctx->stream))) return s;
     mh.adapter = ad;
   }
   std::vector<LayerDev> layers(L);
@@ -302,14 +304,14 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
     if ((s = put_rows(ctx, rm, w->wq[l], staging, d, d, esz, 1, 0, dh))) return s;
     if ((s = put_rows(ctx, rm + (size_t)d * d * esz, w->wk[l], staging, d, d, esz, 1, 0, dh))) return s;
     if ((s = put_rows(ctx, rm + (size_t)2 * d * d * esz, w->wv[l], staging, d, d, esz, 1, 0, 0))) return s;
-    if ((s = pack_tiles(ctx, wqkv, rm, 3 * d, d, esz, ctx->n_sm, ctx->stream))) return s;
+    if ((s = pack_tiles(ctx, wqkv, rm, 3 * d, d, esz, mh.grid, ctx->stream))) return s;
     if ((s = put_rows(ctx, rm, w->wo[l], staging, d, d, esz, 1, 0, 0))) return s;
-    if ((s = pack_tiles(ctx, wo, rm, d, d, esz, ctx->n_sm, ctx->stream))) return s;
+    if ((s = pack_tiles(ctx, wo, rm, d, d, esz, mh.grid, ctx->stream))) return s;
     if ((s = put_rows(ctx, rm, w->w_gate[l], staging, f, d, esz, 2, 0, 0))) return s;
     if ((s = put_rows(ctx, rm, w->w_up[l], staging, f, d, esz, 2, 1, 0))) return s;
-    if ((s = pack_tiles(ctx, wgu, rm, 2 * f, d, esz, ctx->n_sm, ctx->stream))) return s;
+    if ((s = pack_tiles(ctx, wgu, rm, 2 * f, d, esz, mh.grid, ctx->stream))) return s;
     if ((s = put_rows(ctx, rm, w->w_down[l], staging, d, f, esz, 1, 0, 0))) return s;
-    if ((s = pack_tiles(ctx, wd, rm, d, f, esz, ctx->n_sm, ctx->stream))) return s;
+    if ((s = pack_tiles(ctx, wd, rm, d, f, esz, mh.grid, ctx->stream))) return s;
     if (!w->attn_norm[l] || !w->ffn_norm[l]) return fail(ctx, SPD_EINVAL, "missing norm gain");
     CU(cudaMemcpyAsync(an, w->attn_norm[l], d * sizeof(float), cudaMemcpyDefault, ctx->stream));
     CU(cudaMemcpyAsync(fnw, w->ffn_norm[l], d * sizeof(float), cudaMemcpyDefault, ctx->stream));
@@ -417,27 +419,64 @@ spd_status launch_cfg(spd_ctx* ctx, KernelFn fn, int M, int n_sm, int smem_optin
   return SPD_OK;
 }
 
-spd_status launch_forward(spd_ctx* ctx, int M, int dtype, StepArgs a, cudaStream_t stream, int n_sm, int smem_optin,
-                          unsigned* bar) {
+unsigned* next_bar(spd_ctx* ctx);
+
+// One cluster of `cs` CTAs with this kernel's shared memory must be able to run.
+bool cluster_fits(KernelFn fn, int cs, size_t smem) {
+  if (cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(cs); cfg.blockDim = dim3(ENGINE_THREADS); cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, (const void*)fn, &cfg) != cudaSuccess) { cudaGetLastError(); return false; }
+  return n >= 1;
+}
+
+// grid = CTAs of the launch; cluster > 0: they form one thread-block cluster (then grid == cluster)
+// and synchronise inside it, otherwise it is a cooperative launch with the barrier word `bar`.
+spd_status launch_forward(spd_ctx* ctx, int M, int dtype, StepArgs a, cudaStream_t stream, int grid, int cluster,
+                          int smem_optin, unsigned* bar, int n_sm_sampling) {
   KernelFn fn = pick_kernel(M, dtype);
   LaunchCfg lc{};
-  spd_status s = launch_cfg(ctx, fn, M, n_sm, smem_optin, &lc);
+  spd_status s = launch_cfg(ctx, fn, M, grid, smem_optin, &lc);
   if (s) return s;
   a.nstage = lc.nstage;
   a.bar = bar;
-  CU(cudaMemsetAsync(bar, 0, sizeof(unsigned), stream));
-  void* params[] = {&a};
+  a.cluster_ctas = cluster;
+  a.fwd_grid = grid;
   a.sample_r0 = M - 1;
-  CU(cudaLaunchCooperativeKernel((const void*)fn, dim3(n_sm), dim3(ENGINE_THREADS), params, lc.smem, stream));
+  void* params[] = {&a};
+  if (cluster > 0) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(ENGINE_THREADS); cfg.dynamicSmemBytes = lc.smem; cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = cluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    CU(cudaLaunchKernelExC(&cfg, (const void*)fn, params));
+  } else {
+    CU(cudaMemsetAsync(bar, 0, sizeof(unsigned), stream));
+    CU(cudaLaunchCooperativeKernel((const void*)fn, dim3(grid), dim3(ENGINE_THREADS), params, lc.smem, stream));
+  }
   // sampling (not greedy): the forward kernel has left logits and per-slice row statistics; two
-  // small kernels spread the draw over the grid and commit the step
+  // small kernels spread the draw over the whole device and commit the step
   const bool samples = a.mode == MODE_VERIFY || a.mode == MODE_DRAFT || (a.mode == MODE_ROWS && a.want_sample);
   if (samples && !a.greedy) {
-    sample_slices_kernel<<<n_sm, SAMPLE_THREADS, 0, stream>>>(a);
-    sample_pick_kernel<<<1, SAMPLE_THREADS, 0, stream>>>(a, n_sm);
+    sample_slices_kernel<<<n_sm_sampling, SAMPLE_THREADS, 0, stream>>>(a);
+    sample_pick_kernel<<<1, SAMPLE_THREADS, 0, stream>>>(a, n_sm_sampling);
     CU(cudaGetLastError());
   }
   return SPD_OK;
+}
+
+spd_status launch_model(spd_ctx* ctx, ModelHost& mh, int M, StepArgs a, cudaStream_t stream) {
+  return launch_forward(ctx, M, mh.cfg.dtype, a, stream, mh.grid, mh.cluster, ctx->smem_optin, next_bar(ctx), ctx->n_sm);
 }
 
 unsigned* next_bar(spd_ctx* ctx) {
@@ -503,7 +542,7 @@ spd_status feed_rows(spd_ctx* ctx, ModelHost& mh, const float* rows_dev, const i
     a.init_prev = init_prev;
     a.uniforms = ctx->ubuf + 8;
     a.out_ids = ctx->out_dev;
-    spd_status s = launch_forward(ctx, M, mh.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx));
+    spd_status s = launch_model(ctx, mh, M, a, ctx->stream);
     if (s) return s;
   }
   return SPD_OK;
@@ -795,6 +834,29 @@ spd_status spd_create(const spd_weights* target_w, const spd_weights* draft_w, c
     cudaFree(staging);
     return bail(fail(ctx, SPD_ENOMEM, "staging allocation failed"));
   }
+  // Launch shape per model.  Default: one CTA per SM, barrier in global memory.  grid_mode 2 runs a
+  // model as ONE thread-block cluster (16 CTAs, else 8) whose members synchronise through each
+  // other's shared memory: barriers cost a hop between SMs instead of two trips to L2, but 16 SMs'
+  // compute warps consume a weight stage every 0.3 us each, far less than 148 do, and the 115M
+  // draft's step took 0.61 ms that way against 0.31 ms on the full grid -- so it is not chosen
+  // automatically.  The weights are packed for the CTA count of the model.
+  for (ModelHost* mh : {&ctx->target, &ctx->draft}) {
+    const spd_model_cfg& c = mh == &ctx->target ? cfg->target : cfg->draft;
+    mh->grid = ctx->n_sm; mh->cluster = 0;
+    const double bytes = ((double)c.n_layers * (4.0 * c.d_model * c.d_model + 3.0 * c.d_model * c.d_ffn) +
+                          (double)c.vocab * c.d_model) * (c.dtype ? 2 : 4);
+    (void)bytes;
+    if (cfg->grid_mode != 2) continue;
+    for (int cs : {16, 8}) {
+      bool ok = true;
+      for (int M = 1; M <= MAX_M && ok; ++M) {
+        KernelFn fn = pick_kernel(M, c.dtype);
+        LaunchCfg lc{};
+        ok = launch_cfg(ctx, fn, M, cs, ctx->smem_optin, &lc) == SPD_OK && cluster_fits(fn, cs, lc.smem);
+      }
+      if (ok) { mh->grid = cs; mh->cluster = cs; break; }
+    }
+  }
   s = build_model(ctx, ctx->target, cfg->target, target_w, 0, staging, rowmajor);
   if (!s) s = build_model(ctx, ctx->draft, cfg->draft, draft_w, cfg->draft_adapter_in, staging, rowmajor);
   cudaStreamSynchronize(ctx->stream);
@@ -878,7 +940,7 @@ spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m, const flo
     a.rows = tm.md.x; a.rows_pos0 = Rt - 1;
     a.init_n_text = n; a.init_prev = last_id;
     a.uniforms = ctx->ubuf + 8; a.out_ids = ctx->out_dev;
-    if ((s = launch_forward(ctx, 1, tm.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx)))) return s;
+    if ((s = launch_model(ctx, tm, 1, a, ctx->stream))) return s;
     moved_logits = true;
   } else {
   // ---- draft: [adapter(features) ; embed(prompt)] or embed(prompt) alone (Sec. 3)
@@ -897,7 +959,7 @@ spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m, const flo
       StepArgs a = base_args(ctx, dm);
       a.mode = MODE_GEMM;
       a.gx = fstage + (size_t)r * ad; a.gw = dm.adapter; a.gy = outrows + (size_t)r * dd; a.gN = dd; a.gK = ad;
-      if ((s = launch_forward(ctx, M, dm.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx)))) return s;
+      if ((s = launch_model(ctx, dm, M, a, ctx->stream))) return s;
     }
     if ((s = feed_rows(ctx, dm, outrows, nullptr, 0, m, 0, false, 0, 0))) return s;
     dm.pos_base = m;
@@ -997,7 +1059,7 @@ spd_status spd_draft(spd_ctx* ctx, int gamma, const float* uniforms, int32_t* dr
     a.uniforms = ctx->ubuf;
     a.q_out = ctx->qbuf;
     a.logits = dm.logits;
-    spd_status s = launch_forward(ctx, 2, dm.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx));
+    spd_status s = launch_model(ctx, dm, 2, a, ctx->stream);
     if (s) return s;
     // keep this step's logits row (row 1) for spd_get_draft_logits: rows 2.. of the buffer
     if (j + 2 < MAX_M)
@@ -1045,7 +1107,7 @@ spd_status spd_verify(spd_ctx* ctx, int gamma, const int32_t* draft_ids, const f
   a.q_in = draft_probs ? draft_probs : ctx->qbuf;
   a.out_ids = nullptr;
   a.trace = ctx->trace;
-  spd_status s = launch_forward(ctx, gamma + 1, tm.cfg.dtype, a, ctx->stream, ctx->n_sm, ctx->smem_optin, next_bar(ctx));
+  spd_status s = launch_model(ctx, tm, gamma + 1, a, ctx->stream);
   if (s) return s;
   ctx->drafted_gamma = -1;
   ctx->len_ub += gamma + 1;
@@ -1099,13 +1161,13 @@ spd_status spd_generate(spd_ctx* ctx, int n_new, int gamma, const float* uniform
       a.mode = MODE_DRAFT; a.gamma = gamma; a.j = j;
       a.uniforms = uniforms ? ctx->upool : nullptr; a.u_stride = us; a.u_by_block = 1;
       a.q_out = ctx->qbuf; a.logits = dm.logits;
-      if ((r = launch_forward(ctx, 2, dm.cfg.dtype, a, cs, ctx->n_sm, ctx->smem_optin, next_bar(ctx)))) return r;
+      if ((r = launch_model(ctx, dm, 2, a, cs))) return r;
     }
     StepArgs a = base_args(ctx, tm);
     a.mode = MODE_VERIFY; a.gamma = gamma;
     a.uniforms = uniforms ? ctx->upool : nullptr; a.u_stride = us; a.u_by_block = 1;
     a.q_in = ctx->qbuf; a.out_ids = ctx->out_dev;
-    return launch_forward(ctx, gamma + 1, tm.cfg.dtype, a, cs, ctx->n_sm, ctx->smem_optin, next_bar(ctx));
+    return launch_model(ctx, tm, gamma + 1, a, cs);
   };
   const float* pool_key = uniforms ? ctx->upool : nullptr;
   if (ctx->graphs_ok && (!ctx->block_exec || ctx->block_gamma != gamma || ctx->block_upool != pool_key)) {
@@ -1298,7 +1360,7 @@ spd_status spd_skinny_gemm(const float* x, const void* w, int dtype, int M, int 
   a.mode = MODE_GEMM;
   a.st = g.st;
   a.gx = x; a.gw = g.packed; a.gy = y; a.gN = N; a.gK = K;
-  return launch_forward(ctx, M, dtype, a, cs, g.n_sm, g.smem_optin, g.bar);
+  return launch_forward(ctx, M, dtype, a, cs, g.n_sm, 0, g.smem_optin, g.bar, g.n_sm);
 }
 
 spd_status spd_skinny_gemm_status(int noalloc, void* stream) {
@@ -1355,7 +1417,7 @@ spd_status spd_skinny_gemm_noalloc(const float* x, const void* w, int dtype, int
   a.mode = MODE_GEMM;
   a.st = g.st;
   a.gx = x; a.gw = g.packed; a.gy = y; a.gN = N; a.gK = K;
-  return launch_forward(ctx, M, dtype, a, cs, g.n_sm, g.smem_optin, g.bar);
+  return launch_forward(ctx, M, dtype, a, cs, g.n_sm, 0, g.smem_optin, g.bar, g.n_sm);
 }
 
 spd_status spd_wait_selftest(spd_ctx* ctx, int which, unsigned polls) {

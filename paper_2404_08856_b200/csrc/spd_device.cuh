@@ -57,6 +57,32 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, volati
   return false;
 }
 
+// ---- thread-block cluster: CTAs of one cluster synchronise through each other's shared memory
+// (a remote arrival on every member's barrier), without a round trip through global memory.
+__device__ __forceinline__ uint32_t cluster_map(uint32_t local_smem_addr, unsigned cta_rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(cta_rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Hardware barrier over every thread of the cluster (all threads of all its CTAs must call it).
+__device__ __forceinline__ void cluster_sync_all_threads() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // 1-D bulk copy global -> this CTA's shared memory, completion counted on an mbarrier.
 // Source, destination and size must be multiples of 16 bytes.
 __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src, unsigned bytes, uint64_t* bar,

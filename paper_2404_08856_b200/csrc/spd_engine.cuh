@@ -99,6 +99,8 @@ struct StepArgs {
   DevState* st;
   unsigned* bar;          // grid-barrier counter, zero at launch
   int mode, gamma, j, pos_base, nstage, greedy;
+  int cluster_ctas;       // > 0: the grid is ONE thread-block cluster of that many CTAs (small models)
+  int fwd_grid;           // CTAs of the forward kernel that left the row statistics (set at launch)
   float temperature;
   // MODE_ROWS
   const float* rows;      // fp32 [M, d] input rows (already embeddings), or NULL: ids
@@ -124,6 +126,7 @@ struct Ctrl {
   uint64_t full[NSTAGE_MAX];
   uint64_t empty[NSTAGE_MAX];
   uint64_t xbar;                    // completion of the activation rows' bulk copies
+  uint64_t cbar;                    // cluster launches: one arrival per CTA of the cluster per barrier
   SampleScratch sc;
   float red[8][MAX_M];
   float inv[MAX_M];
@@ -675,6 +678,28 @@ __device__ __forceinline__ void grid_barrier(unsigned* counter, unsigned& target
     // no fence here: the acquire load above orders this thread, the CTA barrier below hands
     // that order on to the other compute threads (cumulativity)
   }
+  named_sync(1, CONSUMER_THREADS);
+}
+
+// The same barrier for a grid that is one thread-block cluster: the first G threads each arrive
+// on the barrier word in one member's shared memory, thread 0 waits for the G arrivals on its
+// own.  Release / acquire at cluster scope order the global-memory traffic around it like the
+// red.release / ld.acquire pair above does at gpu scope; the cost is a hop between SMs instead
+// of two trips to L2.
+__device__ __forceinline__ void cluster_barrier(uint64_t* cbar, unsigned& phase, unsigned G, volatile int* err,
+                                                unsigned limit = SPIN_LIMIT_GRID) {
+  named_sync(1, CONSUMER_THREADS);
+  if (threadIdx.x < G) mbar_arrive_remote(cluster_map(smem_u32(cbar), threadIdx.x));
+  if (threadIdx.x == 0) {
+    unsigned it = 0;
+    while (!mbar_try_wait_cluster(cbar, phase)) {
+      if (++it > limit || ((it & 255u) == 0 && *err != DEV_OK)) {
+        atomicCAS(const_cast<int*>(err), DEV_OK, DEV_TIMEOUT_GRID);
+        break;
+      }
+    }
+  }
+  phase ^= 1u;
   named_sync(1, CONSUMER_THREADS);
 }
 

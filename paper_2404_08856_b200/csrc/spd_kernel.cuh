@@ -78,6 +78,7 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
       mbar_init(&ctl->empty[i], CONSUMER_THREADS / 32);
     }
     mbar_init(&ctl->xbar, 1);
+    if (a.cluster_ctas) mbar_init(&ctl->cbar, (unsigned)a.cluster_ctas);
     mbar_fence_init();
   }
   if (tid < ZERO_BYTES / 4) reinterpret_cast<uint32_t*>(smem + CTRL_BYTES)[tid] = 0u;
@@ -88,6 +89,8 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
       reinterpret_cast<uint64_t*>(lay_s)[i] = reinterpret_cast<const uint64_t*>(md.layers)[i];
   const LayerDev* layers = lay_in_smem ? lay_s : md.layers;
   __syncthreads();
+  // a cluster launch: every member's barrier word must exist before anyone arrives on it
+  if (a.cluster_ctas) cluster_sync_all_threads();
 
   const bool gemm_only = a.mode == MODE_GEMM;
   const bool want_head = gemm_only ? false : (a.mode != MODE_ROWS || a.want_sample);
@@ -112,7 +115,12 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
   } else {
     // ---------------- compute warps
     Ring ring{0, 0u, a.nstage};
-    unsigned bar_target = 0, xphase = 0;
+    unsigned bar_target = 0, xphase = 0, cphase = 0;
+    // all CTAs wait for each other: through global memory, or inside the cluster
+    auto sync_grid = [&]() {
+      if (a.cluster_ctas) cluster_barrier(&ctl->cbar, cphase, (unsigned)G, err);
+      else grid_barrier(a.bar, bar_target, G, err);
+    };
     if (tid == 0) { ctl->trace = cta == 0 ? a.trace : nullptr; ctl->trace_n = 0; }
     named_sync(1, CONSUMER_THREADS);
     auto stamp = [&](int id = 3) { trace_stamp(ctl, id); };
@@ -217,11 +225,11 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
         }
         consume_gemm<M, WT>(g, e, src, norm_w, md.eps, copy_out, ssq_in, cta, G, ring, ctl, X, xphase, red, pre_s,
                             zero_addr, stages, err);
-        stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
+        stamp(3); sync_grid(); stamp(4);
         if (!head && which == 0) {
           if constexpr (sizeof(WT) == 2) attn_phase_mma<M>(md, l, pos0, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
           else attn_phase<M, WT>(md, l, pos0, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
-          stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
+          stamp(3); sync_grid(); stamp(4);
         }
       }
       if (want_head) {
@@ -230,7 +238,7 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
         if (a.mode == MODE_VERIFY) { r0 = 0; nrows = a.gamma + 1; }
         else { r0 = M - 1; nrows = 1; }
         stats_phase<M>(a.logits, md.V, r0, nrows, a.temperature, cta, G, md.stat_part, ctl);
-        stamp(3); grid_barrier(a.bar, bar_target, G, err); stamp(4);
+        stamp(3); sync_grid(); stamp(4);
         if (cta == 0 && a.greedy) {
           if (a.mode == MODE_VERIFY) verify_greedy<M>(a, md, st, ctl, G, 0, a.gamma, ctl->tok + 1, pending);
           else if (a.mode == MODE_DRAFT) draft_greedy<M>(a, md, st, ctl, G);
@@ -249,6 +257,8 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
     // a wait gave up: let copies that are still in flight land before the CTA retires
     for (int i = 0; i < 200; ++i) __nanosleep(1000);
   }
+  // no member of a cluster retires while another may still arrive on its barrier word
+  if (a.cluster_ctas) cluster_sync_all_threads();
 }
 
 // ------------------------------------------------------------------------------ bounded waits, exercised
@@ -309,7 +319,7 @@ __device__ SamplePlan sample_plan(const StepArgs& a, const DevState* st, SampleS
   pl.gamma = a.mode == MODE_VERIFY ? a.gamma : 0;
   pl.r0 = a.mode == MODE_VERIFY ? 0 : a.sample_r0;
   pl.u = step_uniforms(a, st);
-  merge_stats(a.md.stat_part, G, pl.gamma + 1, nullptr, sh->rowmax, sh->rowsum, sh->arg);
+  merge_stats(a.md.stat_part, a.fwd_grid, pl.gamma + 1, nullptr, sh->rowmax, sh->rowsum, sh->arg);
   pl.r = pl.gamma;
   for (int j = 0; j < pl.gamma; ++j) {
     int x = st->d_ids[j];

@@ -175,6 +175,32 @@ class Weights:
         a = self.stored[name] if layer is None else self.stored[name][layer]
         return bf16_bits_to_f32(a) if a.dtype == np.uint16 else a
 
+    # -- several processes on one host (one replica per GPU) share one copy of the stored arrays
+    def save(self, directory: str) -> None:
+        """Writes every stored array as `<directory>/<name>[.<layer>].npy`."""
+        os.makedirs(directory, exist_ok=True)
+        for name, a in self.stored.items():
+            if name == "lm_head" and self.cfg.tied_embeddings:
+                continue
+            for layer, arr in (enumerate(a) if isinstance(a, list) else [(None, a)]):
+                np.save(os.path.join(directory, name + ("" if layer is None else f".{layer}") + ".npy"), arr)
+
+    @classmethod
+    def load(cls, cfg: ModelCfg, seed: int, role: str, directory: str) -> "Weights":
+        """The arrays written by `save`, memory-mapped read-only (no second copy in RAM)."""
+        self = cls.__new__(cls)
+        self.cfg, self.seed, self.role, self.stored = cfg, seed, role, {}
+        for fn in sorted(os.listdir(directory)):
+            parts = fn[:-4].split(".")
+            arr = np.load(os.path.join(directory, fn), mmap_mode="r")
+            if len(parts) == 1:
+                self.stored[parts[0]] = arr
+            else:
+                self.stored.setdefault(parts[0], [None] * cfg.n_layers)[int(parts[1])] = arr
+        if cfg.tied_embeddings:
+            self.stored["lm_head"] = self.stored["tok_embed"]
+        return self
+
 
 def image_embeds(wl: Workload) -> np.ndarray:
     """Projected image embeddings V_1..V_m handed to the target, fp32 [m, d_target].

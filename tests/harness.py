@@ -40,10 +40,10 @@ def make_oracle(wl, tw, dw, max_seq, temperature=1.0, greedy=False):
     return SpdOracle(t, d, temperature, greedy, adapter_w=ad)
 
 
-def make_gpu(wl, tw, dw, max_seq, temperature=1.0, greedy=False, gamma_max=7):
+def make_gpu(wl, tw, dw, max_seq, temperature=1.0, greedy=False, gamma_max=7, grid_mode=0):
     import paper_2404_08856_b200 as spd
     return spd.Spd(wl.target, wl.draft, tw.stored, dw.stored, max_seq, gamma_max, temperature, greedy,
-                   adapter_in=wl.draft.d_model if wl.draft_mlp else wl.adapter_in)
+                   adapter_in=wl.draft.d_model if wl.draft_mlp else wl.adapter_in, grid_mode=grid_mode)
 
 
 class SafeUniforms:

@@ -44,3 +44,20 @@ def test_single_rank_aggregation_and_reference_line_shape():
     assert bench.aggregate(50.0, 250.0) == (200.0, 250.0)
     cfg = bench.workload_config()
     assert "workload" in cfg and "model" not in cfg
+
+
+def test_gpus_flag_spawns_replicas_that_share_one_weight_copy():
+    """`python bench.py --gpus 2` with no launcher around it starts two ranks itself (the stand-in
+    step of --selftest-launcher replaces the GPU work): both ranks rendezvous on 127.0.0.1, map
+    the weights rank 0 generated, and rank 0 prints the whole-job value."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--selftest-launcher"],
+                       capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                      # rank 0 alone prints
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2 and out["ms_max"] == 800.0 and abs(out["value"] - 180.0 / 0.8) < 1e-9
+    assert out["weights_identical_on_all_ranks"] is True

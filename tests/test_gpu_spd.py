@@ -157,7 +157,7 @@ def test_reject_sample_distribution_small_vocab():
 # ------------------------------------------------------------------ whole path, lock-step
 
 def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None, max_seq=None, gain_seed=None,
-             image_from=None, uniforms="safe"):
+             image_from=None, uniforms="safe", grid_mode=0):
     """Drives the CUDA context and the oracle block by block on the same inputs and compares
     logits, draft tokens, accept decisions and drawn tokens.
 
@@ -176,7 +176,8 @@ def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None
     `image_from(gpu_ctx) -> (device image rows, oracle image rows[, device draft rows, oracle
     draft rows])` replaces the generated image embeddings (and the draft's image rows); used to
     put the image adapters in front of the prefill.  `uniforms`: "safe" (the oracle skips
-    candidates inside the tolerance of a boundary) or "plain" (the seeded stream as it is)."""
+    candidates inside the tolerance of a boundary) or "plain" (the seeded stream as it is).
+    `grid_mode`: launch shape (spd_cfg.grid_mode; 2 = one thread-block cluster per model)."""
     spd = _lib()
     tw, dw = H.build_weights(wl, std)
     if gain_seed is not None:
@@ -191,7 +192,7 @@ def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None
     max_seq = max_seq or (wl.n_image + wl.n_prompt + 8 * (n_blocks + 2) + 16)
     fp32 = wl.target.dtype == "fp32"
     orc = H.make_oracle(wl, tw, dw, max_seq, temperature, greedy)
-    gpu = H.make_gpu(wl, tw, dw, max_seq, temperature, greedy)
+    gpu = H.make_gpu(wl, tw, dw, max_seq, temperature, greedy, grid_mode=grid_mode)
     img = synth.image_embeds(wl) if wl.n_image else None
     gpu_img = img
     feats = synth.image_features(wl) if wl.adapter_in else None
@@ -327,10 +328,13 @@ def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("grid_mode", [1, 2])
 @pytest.mark.parametrize("greedy", [True, False])
-def test_tiny_lockstep(greedy):
+def test_tiny_lockstep(greedy, grid_mode):
+    """grid_mode 1: one CTA per SM and the barrier in global memory; 2: one 16-CTA cluster."""
     wl = synth.tiny_workload(4)
-    r = lockstep(wl, greedy, 1.0, 10, 2e-4, std=0.2 if greedy else 0.1, gammas=[4, 1, 7, 3, 2, 5, 6])
+    r = lockstep(wl, greedy, 1.0, 10, 2e-4, std=0.2 if greedy else 0.1, gammas=[4, 1, 7, 3, 2, 5, 6],
+                 grid_mode=grid_mode)
     assert r["blocks"] == 10
     assert r["accept_within_tol"] == 0 and r["accept_beyond_tol"] == 0 and r["cdf_band_tokens"] == 0
     if not greedy:
@@ -408,7 +412,9 @@ def test_small_bf16_models_where_most_ctas_own_no_rows():
     t = synth.ModelCfg(2, 256, 4, 688, 1024, False, dtype="bf16")
     d = synth.ModelCfg(1, 128, 2, 344, 1024, False, dtype="bf16")
     wl = synth.Workload("tiny-bf16", t, d, 16, 16, 4, 32)
-    r = lockstep(wl, False, 1.0, 4, 2e-2, std=0.08, gain_seed=9)
+    r = lockstep(wl, False, 1.0, 4, 2e-2, std=0.08, gain_seed=9, grid_mode=1)
+    assert r["blocks"] == 4
+    r = lockstep(wl, False, 1.0, 4, 2e-2, std=0.08, gain_seed=9, grid_mode=2)
     assert r["blocks"] == 4
 
 
@@ -417,6 +423,16 @@ def test_llava7b_shaped_two_layer_greedy():
     wl = synth.llava7b_workload(gamma=5, n_layers=2, draft_layers=2)
     r = lockstep(wl, True, 1.0, 3, 5e-2)
     assert r["blocks"] == 3
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("grid_mode", [1, 2])
+def test_llava7b_shaped_two_layer_forced_launch_shapes(grid_mode):
+    """Both launch shapes at the 7B / 115M layer shapes: one CTA per SM (1, the default) and one
+    16-CTA cluster per model (2)."""
+    wl = synth.llava7b_workload(gamma=5, n_layers=2, draft_layers=2)
+    r = lockstep(wl, False, 1.0, 2, 5e-2, grid_mode=grid_mode)
+    assert r["blocks"] == 2 and r["max_logit_err"] < 1e-2
 
 
 @pytest.mark.gpu
