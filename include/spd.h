@@ -79,6 +79,15 @@ typedef struct {
                            placed) that synchronise through each other's shared memory -- cheaper
                            barriers, but only 16 SMs' worth of streaming (115M draft: 0.61 ms per step
                            against 0.31 ms).  Results do not depend on it beyond summation order. */
+  int top_k;            /* sampling only: keep the k most probable tokens of every row (0: off) */
+  float top_p;          /* sampling only: then the shortest most-probable prefix whose mass reaches top_p
+                           times what is left (0 or >= 1: off).  Sec. 4 "Decoding" names sampling with
+                           top-p / top-k as future work and defines neither; here BOTH the target's rows
+                           and the draft's rows are truncated and renormalised (the exact definitions
+                           are those of spd_truncate_probs), the draft tokens are drawn from the
+                           truncated draft rows, draft_probs holds those rows, and the unchanged rule
+                           of Sec. 2.1 runs on the truncated rows: the emitted tokens then follow the
+                           truncated target distribution.  top_k = 1 reproduces greedy decoding. */
 } spd_cfg;
 
 /* Host or device pointers; per-layer entries are HOST arrays of n_layers pointers. */

@@ -25,7 +25,9 @@ the storage format of the model (`kv_dtype`).
 Pinned by tests/test_oracle_forward.py: primitives against closed forms and fp64 library
 routines, the whole stack against an independent library LLaMA in fp64, cached block
 forward == cache-free recompute, one M-row call == M one-row calls, rollback == never
-having fed the rejected rows, RoPE norm preservation and relative-position property.
+having fed the rejected rows, RoPE norm preservation and relative-position property;
+`forward_tree` (tests/test_oracle_tree.py): a chain-shaped tree == `forward`, and every
+root-to-leaf path of a branching tree == that path fed alone as a chain.
 """
 from __future__ import annotations
 
@@ -152,6 +154,52 @@ class Model:
         for l in range(self.cfg.n_layers):
             x = self._layer(l, x, cache, pos0)
         cache.length = pos0 + x.shape[0]
+        h = rmsnorm(x, self.w.f32("final_norm"), self.cfg.rms_eps)
+        return h @ self.w.f32("lm_head").T
+
+    # -- draft TREE: rows are nodes of a token tree hanging off the last committed token ----
+    def forward_tree(self, cache: KVCache, rows: np.ndarray, origin: int, slots, depths, sees) -> np.ndarray:
+        """Tree-based speculative decoding (the paper's Sec. 5 names it as the next step and
+        cites SpecInfer / Medusa-style token trees): the M input rows are nodes of a tree whose
+        root sits at sequence position `origin`.  Row i is a node at depth depths[i] below the
+        root (the root itself has depth 0), so its rotary position is origin + depths[i]; its K/V
+        go to cache row origin + slots[i] (every node has its own row, siblings share a position
+        but not a row); it attends every cache row below `origin` (the committed prefix) and, of
+        the rows from `origin` on, exactly those whose slot is in sees[i] (its ancestors and
+        itself).  A chain (slots = depths = 0..M-1, sees[i] = {0..i}) is `forward`.  Returns
+        logits [M, vocab]; cache.length is left to the caller (which rows survive is decided by
+        the verification)."""
+        c, w = self.cfg, self.w
+        x = np.ascontiguousarray(rows, dtype=F32)
+        M, H = x.shape[0], c.n_heads
+        dh = c.d_model // H
+        slots = [int(s) for s in slots]
+        pos = np.asarray([origin + int(d) for d in depths])
+        n_slots = max(max(slots), max((max(s) for s in sees if len(s)), default=0)) + 1
+        n_ctx = origin + n_slots
+        assert n_ctx <= self.max_seq and min(slots) >= 0
+        visible = np.zeros((M, n_ctx), dtype=bool)
+        visible[:, :origin] = True
+        for i in range(M):
+            for s_ in sees[i]:
+                visible[i, origin + int(s_)] = True
+        scale = F32(1.0 / np.sqrt(float(dh)))
+        for l in range(c.n_layers):
+            h = rmsnorm(x, w.f32("attn_norm", l), c.rms_eps)
+            q = apply_rope(h @ w.f32("wq", l).T, pos, self.cos, self.sin, H)
+            k = apply_rope(h @ w.f32("wk", l).T, pos, self.cos, self.sin, H)
+            v = h @ w.f32("wv", l).T
+            for i in range(M):
+                cache.store(l, origin + slots[i], k[i:i + 1], v[i:i + 1])
+            o = np.empty((M, c.d_model), dtype=F32)
+            for hd in range(H):
+                sl = slice(hd * dh, (hd + 1) * dh)
+                s = (q[:, sl] @ cache.k[l, :n_ctx, sl].T) * scale
+                s = np.where(visible, s, F32(-np.inf))
+                o[:, sl] = softmax_rows(s) @ cache.v[l, :n_ctx, sl]
+            x = x + o @ w.f32("wo", l).T
+            h = rmsnorm(x, w.f32("ffn_norm", l), c.rms_eps)
+            x = x + (silu(h @ w.f32("w_gate", l).T) * (h @ w.f32("w_up", l).T)) @ w.f32("w_down", l).T
         h = rmsnorm(x, self.w.f32("final_norm"), self.cfg.rms_eps)
         return h @ self.w.f32("lm_head").T
 

@@ -40,7 +40,7 @@ class ModelCfgC(C.Structure):
 class CfgC(C.Structure):
     _fields_ = [("target", ModelCfgC), ("draft", ModelCfgC), ("max_seq", C.c_int), ("gamma_max", C.c_int),
                 ("temperature", C.c_float), ("greedy", C.c_int), ("draft_adapter_in", C.c_int),
-                ("stream", C.c_void_p), ("grid_mode", C.c_int)]
+                ("stream", C.c_void_p), ("grid_mode", C.c_int), ("top_k", C.c_int), ("top_p", C.c_float)]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -117,12 +117,12 @@ class Spd:
 
     def __init__(self, target_cfg, draft_cfg, target_stored: dict, draft_stored: dict, max_seq: int,
                  gamma_max: int, temperature: float = 1.0, greedy: bool = False, adapter_in: int = 0,
-                 stream: int = 0, grid_mode: int = 0):
+                 stream: int = 0, grid_mode: int = 0, top_k: int = 0, top_p: float = 0.0):
         L = lib()
         self.vocab = target_cfg.vocab
         self.greedy = greedy
         cfg = CfgC(model_cfg_c(target_cfg), model_cfg_c(draft_cfg), max_seq, gamma_max, temperature,
-                   int(greedy), adapter_in, C.c_void_p(stream), int(grid_mode))
+                   int(greedy), adapter_in, C.c_void_p(stream), int(grid_mode), int(top_k), float(top_p))
         tw, k1 = weights_c(target_stored, target_cfg.n_layers)
         dw, k2 = weights_c(draft_stored, draft_cfg.n_layers)
         self._ctx = C.c_void_p(0)

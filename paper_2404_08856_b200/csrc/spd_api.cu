@@ -49,6 +49,8 @@ struct spd_ctx {
   int bar_next = 0;
   float* ubuf = nullptr;        // [16] uniforms of direct calls: [0..7] draft, [8..15] verify
   float* qbuf = nullptr;        // [gamma_max][V] draft distributions
+  float* prow = nullptr;        // [MAX_M][V] probability rows of the step being sampled (top-k / top-p only)
+  bool truncate = false;        // top-k / top-p switched on
   float* rows = nullptr;        // prefill rows staging [max_seq][d_max]
   int* ids_dev = nullptr;       // prompt ids [max_seq]
   float* upool = nullptr; size_t upool_cap = 0;
@@ -468,8 +470,17 @@ spd_status launch_forward(spd_ctx* ctx, int M, int dtype, StepArgs a, cudaStream
   // small kernels spread the draw over the whole device and commit the step
   const bool samples = a.mode == MODE_VERIFY || a.mode == MODE_DRAFT || (a.mode == MODE_ROWS && a.want_sample);
   if (samples && !a.greedy) {
-    sample_slices_kernel<<<n_sm_sampling, SAMPLE_THREADS, 0, stream>>>(a);
-    sample_pick_kernel<<<1, SAMPLE_THREADS, 0, stream>>>(a, n_sm_sampling);
+    if (ctx && ctx->truncate) {
+      // top-k / top-p: probability rows -> truncated and renormalised in place -> the rule on rows
+      const int nrows = a.mode == MODE_VERIFY ? a.gamma + 1 : 1;
+      prob_rows_kernel<<<n_sm_sampling, SAMPLE_THREADS, 0, stream>>>(a, ctx->prow);
+      truncate_rows_kernel<<<nrows, WARP_THREADS, (size_t)a.md.V * sizeof(float), stream>>>(
+          ctx->prow, ctx->prow, a.md.V, ctx->cfg.top_k, ctx->cfg.top_p > 0.f ? ctx->cfg.top_p : 1.0f);
+      sample_rows_kernel<<<1, SAMPLE_THREADS, 0, stream>>>(a, ctx->prow);
+    } else {
+      sample_slices_kernel<<<n_sm_sampling, SAMPLE_THREADS, 0, stream>>>(a);
+      sample_pick_kernel<<<1, SAMPLE_THREADS, 0, stream>>>(a, n_sm_sampling);
+    }
     CU(cudaGetLastError());
   }
   return SPD_OK;
@@ -708,6 +719,16 @@ spd_status alloc_ctx_buffers(spd_ctx* ctx) {
   if ((s = dalloc(ctx, &ctx->bars, (size_t)32 * BAR_POOL))) return s;
   if ((s = dalloc(ctx, &ctx->ubuf, 16))) return s;
   if ((s = dalloc(ctx, &ctx->qbuf, (size_t)(cfg->gamma_max > 0 ? cfg->gamma_max : 1) * V))) return s;
+  ctx->truncate = !cfg->greedy && ((cfg->top_k >= 1 && cfg->top_k < V) || (cfg->top_p > 0.f && cfg->top_p < 1.f));
+  if (ctx->truncate) {
+    if ((s = dalloc(ctx, &ctx->prow, (size_t)MAX_M * V))) return s;
+    // one CTA holds a whole row in shared memory
+    if ((size_t)V * sizeof(float) + sizeof(TruncScratch) + 1024 > (size_t)ctx->smem_optin)
+      return fail(ctx, SPD_EINVAL, "top-k / top-p: a vocabulary row does not fit the shared memory of one CTA");
+    if (cudaFuncSetAttribute((const void*)truncate_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)((size_t)V * sizeof(float))) != cudaSuccess)
+      return fail(ctx, SPD_ECUDA, "cannot size the truncation kernel's shared memory");
+  }
   if ((s = dalloc(ctx, &ctx->rows, (size_t)cfg->max_seq * dmax))) return s;
   if ((s = dalloc(ctx, &ctx->ids_dev, (size_t)cfg->max_seq))) return s;
   ctx->out_cap = cfg->max_seq + MAX_M;
@@ -811,6 +832,7 @@ spd_status spd_create(const spd_weights* target_w, const spd_weights* draft_w, c
   if (cfg->max_seq < 16) return bail(fail(ctx, SPD_EINVAL, "max_seq too small"));
   if (!cfg->greedy && !(cfg->temperature > 0.f)) return bail(fail(ctx, SPD_EINVAL, "temperature must be > 0"));
   if (cfg->draft_adapter_in < 0 || cfg->draft_adapter_in % 8) return bail(fail(ctx, SPD_EINVAL, "bad draft_adapter_in"));
+  if (cfg->top_k < 0 || !(cfg->top_p >= 0.f)) return bail(fail(ctx, SPD_EINVAL, "top_k and top_p must not be negative"));
   if (cudaGetDevice(&ctx->device) != cudaSuccess) return bail(fail(ctx, SPD_ECUDA, "no CUDA device"));
   cudaDeviceProp prop{};
   if (cudaGetDeviceProperties(&prop, ctx->device) != cudaSuccess) return bail(fail(ctx, SPD_ECUDA, "no device properties"));

@@ -396,4 +396,64 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) sample_pick_kernel(const __gri
   }
 }
 
+// ------------------------------------------------------------------------------ top-k / top-p on the decoding path
+// With truncation switched on (Sec. 4 "Decoding" names sampling with top-p / top-k as future work) the
+// draw needs whole probability rows: the target's rows p_j and the draft's rows q_j are truncated
+// and renormalised (truncate_rows_kernel) and the unchanged rule of Sec. 2.1 runs on those rows.
+//   prob_rows_kernel    every CTA merges the row statistics and writes its vocabulary slice of
+//                       softmax(logits / T) for the rows the step needs -> prow [rows][V];
+//   (truncate_rows_kernel in place on prow)
+//   sample_rows_kernel  one CTA: draft step -> x_j drawn from the truncated row, which is also
+//                       stored as q_j; verify step -> the rule on (prow, q_in), commit; prefill ->
+//                       the first token drawn from the truncated row.
+
+__device__ __forceinline__ int rows_needed(const StepArgs& a) { return a.mode == MODE_VERIFY ? a.gamma + 1 : 1; }
+
+__global__ void __launch_bounds__(SAMPLE_THREADS) prob_rows_kernel(const __grid_constant__ StepArgs a, float* prow) {
+  __shared__ SampleShared sh;
+  const int cta = blockIdx.x, G = gridDim.x, V = a.md.V;
+  const int nrows = rows_needed(a), r0 = a.mode == MODE_VERIFY ? 0 : a.sample_r0;
+  // the statistics sit at indices 0..nrows-1 (a draft step / a prefill chunk left one row's at index 0)
+  merge_stats(a.md.stat_part, a.fwd_grid, nrows, nullptr, sh.rowmax, sh.rowsum, sh.arg);
+  const int VS = (V + G - 1) / G;
+  const int k0 = cta * VS, k1 = min(V, k0 + VS);
+  for (int r = 0; r < nrows; ++r) {
+    const float* lrow = a.logits + (size_t)(r0 + r) * V;
+    const float mx = sh.rowmax[r], sm = sh.rowsum[r];
+    for (int k = k0 + threadIdx.x; k < k1; k += SAMPLE_THREADS)
+      stcg(prow + (size_t)r * V + k, prob_of(ldcg(lrow + k), a.temperature, mx, sm));
+  }
+}
+
+__global__ void __launch_bounds__(SAMPLE_THREADS) sample_rows_kernel(const __grid_constant__ StepArgs a,
+                                                                     const float* prow) {
+  __shared__ SampleScratch sc;
+  __shared__ int s_ids[MAX_M];
+  DevState* st = a.st;
+  const int V = a.md.V;
+  const float* u = step_uniforms(a, st);
+  if (a.mode == MODE_VERIFY) {
+    if (threadIdx.x < a.gamma) {
+      const int x = st->d_ids[threadIdx.x];
+      s_ids[threadIdx.x] = (unsigned)x < (unsigned)V ? x : 0;   // the forward kernel has flagged it
+    }
+    named_sync(1, SAMPLE_THREADS);
+    int r, tok;
+    reject_rule_block(prow, a.q_in, s_ids, u, a.gamma, V, 0, &sc, r, tok);
+    if (threadIdx.x == 0) {
+      commit_step(a, st, r, tok, st->d_ids, st->pending);
+      st->t_verify1 = globaltimer();
+    }
+  } else {
+    const int tok = block_sample([&](int k) { return ldcg(prow + k); }, V, a.mode == MODE_DRAFT ? u[a.j] : u[0], &sc);
+    if (a.mode == MODE_DRAFT) {
+      float* qrow = a.q_out + (size_t)a.j * V;
+      for (int k = threadIdx.x; k < V; k += SAMPLE_THREADS) stcg(qrow + k, ldcg(prow + k));
+      if (threadIdx.x == 0) { st->d_ids[a.j] = tok; st->t_draft1 = globaltimer(); }
+    } else if (threadIdx.x == 0) {
+      commit_step(a, st, 0, tok, st->d_ids, st->pending);
+    }
+  }
+}
+
 }  // namespace spd

@@ -267,6 +267,35 @@ __device__ int block_argmax(F f, int V, SampleScratch* sc) {
   return idx;
 }
 
+// The rejection rule (Sec. 2.1) on given probability rows, run by one CTA of SAMPLE_THREADS threads:
+// pb [gamma+1][V] target rows, qb [gamma][V] draft rows (unused when greedy), idb [gamma] draft ids
+// (each already known to lie in [0, V)), ub [gamma+1] uniforms.  Returns the accepted count in r and
+// the next token in tok (the same values in every thread).
+__device__ void reject_rule_block(const float* pb, const float* qb, const int* idb, const float* ub, int gamma, int V,
+                                  int greedy, SampleScratch* sc, int& r, int& tok) {
+  r = gamma;
+  if (greedy) {
+    tok = -1;
+    for (int j = 0; j <= gamma; ++j) {
+      const float* row = pb + (size_t)j * V;
+      tok = block_argmax([&](int k) { return row[k]; }, V, sc);
+      if (j < gamma && tok != idb[j]) { r = j; break; }
+    }
+  } else {
+    for (int j = 0; j < gamma; ++j) {
+      const int x = idb[j];
+      if (!accept_test(ub[j], pb[(size_t)j * V + x], qb[(size_t)j * V + x])) { r = j; break; }
+    }
+    const float* prow = pb + (size_t)r * V;
+    if (r < gamma) {
+      const float* qrow = qb + (size_t)r * V;
+      tok = block_sample([&](int k) { return fmaxf(0.0f, __fsub_rn(prow[k], qrow[k])); }, V, ub[gamma], sc);
+    } else {
+      tok = block_sample([&](int k) { return prow[k]; }, V, ub[gamma], sc);
+    }
+  }
+}
+
 // The rejection rule on given probability rows: one block per sequence.
 __global__ void __launch_bounds__(SAMPLE_THREADS)
 reject_sample_kernel(const float* __restrict__ p, const float* __restrict__ q, const int* __restrict__ ids,
@@ -278,7 +307,6 @@ reject_sample_kernel(const float* __restrict__ p, const float* __restrict__ q, c
   const float* qb = q ? q + (size_t)b * gamma * V : nullptr;
   const int* idb = ids + (size_t)b * gamma;
   const float* ub = u ? u + (size_t)b * (gamma + 1) : nullptr;
-  int r = gamma, tok;
   // a draft id outside [0, V) cannot index a row: the sequence is reported as n_acc = next = -1
   bool bad = false;
   for (int j = 0; j < gamma; ++j) bad |= (unsigned)idb[j] >= (unsigned)V;
@@ -286,26 +314,8 @@ reject_sample_kernel(const float* __restrict__ p, const float* __restrict__ q, c
     if (threadIdx.x == 0) { n_acc[b] = -1; next[b] = -1; }
     return;
   }
-  if (greedy) {
-    tok = -1;
-    for (int j = 0; j <= gamma; ++j) {
-      const float* row = pb + (size_t)j * V;
-      tok = block_argmax([&](int k) { return row[k]; }, V, &sc);
-      if (j < gamma && tok != idb[j]) { r = j; break; }
-    }
-  } else {
-    for (int j = 0; j < gamma; ++j) {
-      const int x = idb[j];
-      if (!accept_test(ub[j], pb[(size_t)j * V + x], qb[(size_t)j * V + x])) { r = j; break; }
-    }
-    const float* prow = pb + (size_t)r * V;
-    if (r < gamma) {
-      const float* qrow = qb + (size_t)r * V;
-      tok = block_sample([&](int k) { return fmaxf(0.0f, __fsub_rn(prow[k], qrow[k])); }, V, ub[gamma], &sc);
-    } else {
-      tok = block_sample([&](int k) { return prow[k]; }, V, ub[gamma], &sc);
-    }
-  }
+  int r, tok;
+  reject_rule_block(pb, qb, idb, ub, gamma, V, greedy, &sc, r, tok);
   if (threadIdx.x == 0) { n_acc[b] = r; next[b] = tok; }
 }
 

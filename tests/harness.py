@@ -18,7 +18,7 @@ from __future__ import annotations
 import numpy as np
 
 import synth
-from oracle import llama, sampling as S
+from oracle import llama, sampling as S, warp as W
 from oracle.spd import SpdOracle
 
 F32 = np.float32
@@ -33,17 +33,18 @@ def build_weights(wl, std=0.02):
     return tw, dw
 
 
-def make_oracle(wl, tw, dw, max_seq, temperature=1.0, greedy=False):
+def make_oracle(wl, tw, dw, max_seq, temperature=1.0, greedy=False, top_k=0, top_p=1.0):
     t = llama.Model(wl.target, tw, max_seq)
     d = llama.Model(wl.draft, dw, max_seq)
     ad = dw.f32("adapter") if wl.adapter_in and not wl.draft_mlp else None
-    return SpdOracle(t, d, temperature, greedy, adapter_w=ad)
+    return SpdOracle(t, d, temperature, greedy, adapter_w=ad, top_k=top_k, top_p=top_p)
 
 
-def make_gpu(wl, tw, dw, max_seq, temperature=1.0, greedy=False, gamma_max=7, grid_mode=0):
+def make_gpu(wl, tw, dw, max_seq, temperature=1.0, greedy=False, gamma_max=7, grid_mode=0, top_k=0, top_p=0.0):
     import paper_2404_08856_b200 as spd
     return spd.Spd(wl.target, wl.draft, tw.stored, dw.stored, max_seq, gamma_max, temperature, greedy,
-                   adapter_in=wl.draft.d_model if wl.draft_mlp else wl.adapter_in, grid_mode=grid_mode)
+                   adapter_in=wl.draft.d_model if wl.draft_mlp else wl.adapter_in, grid_mode=grid_mode,
+                   top_k=top_k, top_p=top_p)
 
 
 class SafeUniforms:
@@ -127,6 +128,42 @@ def cdf_band(fp32_model, err_p, err_q=0.0, residual_mass=1.0):
     if fp32_model:
         return CDF_TOL_FP32
     return 2.0 * (err_p + err_q) / max(residual_mass, 1e-6) + 1e-6
+
+
+def cut_zone(w_raw, top_k, top_p, eps):
+    """What a logit error of at most `eps` leaves open about the top-k / top-p cut of a row.
+
+    w_raw: the oracle's un-truncated probabilities.  The other side's probabilities lie within a
+    factor exp(+-2 eps) of them, so (i) two tokens can swap places in the order only if their
+    probabilities are within exp(4 eps) of each other: a token of the top k is surely kept if it
+    exceeds the (k+1)-th probability by that factor, a token outside is surely dropped if it is
+    below the k-th by that factor; (ii) every prefix mass relative to the total moves by at most
+    exp(+-4 eps), so the nucleus ends somewhere between the cuts for top_p * exp(-10 eps) and
+    top_p * exp(+10 eps) (the extra 2 eps covers (i) changing the total).  Returns
+    `sure` (kept on both sides), `maybe` (kept on at least one side, a superset of `sure`),
+    `rho` (relative uncertainty of any renormalised probability of a `sure` token: its own factor
+    exp(2 eps) times that of the kept mass) and `amb` (mass of maybe-but-not-sure tokens relative
+    to the sure mass)."""
+    w = np.asarray(w_raw, dtype=F32)
+    V = w.shape[0]
+    w64 = w.astype(np.float64)
+    sure_k = np.ones(V, dtype=bool)
+    maybe_k = np.ones(V, dtype=bool)
+    if 1 <= top_k < V:
+        srt = np.sort(w64)[::-1]
+        sure_k = w64 > srt[top_k] * np.exp(4 * eps)
+        maybe_k = w64 >= srt[top_k - 1] * np.exp(-4 * eps)
+    in_p = 0.0 < top_p < 1.0
+    lo = W.kept_set(w, top_k, top_p * np.exp(-10 * eps) if in_p else top_p)
+    mid = W.kept_set(w, top_k, top_p)
+    hi = W.kept_set(w, top_k, top_p * np.exp(10 * eps) if in_p else top_p)
+    sure = lo & sure_k
+    maybe = hi | mid | (maybe_k & ~sure_k & (w64 >= (w64[mid].min() if mid.any() else 0.0) * np.exp(-4 * eps)))
+    maybe |= sure
+    s_sure, s_mid, s_maybe = w64[sure].sum(), w64[mid].sum(), w64[maybe].sum()
+    rho = float(np.exp(4 * eps) * max(s_mid / max(s_sure, 1e-30), s_maybe / max(s_mid, 1e-30)) - 1.0)
+    amb = float((s_maybe - s_sure) / max(s_sure, 1e-30))
+    return {"sure": sure, "maybe": maybe, "rho": rho, "amb": amb}
 
 
 def top2_gap(row):

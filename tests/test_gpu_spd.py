@@ -157,7 +157,7 @@ def test_reject_sample_distribution_small_vocab():
 # ------------------------------------------------------------------ whole path, lock-step
 
 def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None, max_seq=None, gain_seed=None,
-             image_from=None, uniforms="safe", grid_mode=0):
+             image_from=None, uniforms="safe", grid_mode=0, top_k=0, top_p=0.0):
     """Drives the CUDA context and the oracle block by block on the same inputs and compares
     logits, draft tokens, accept decisions and drawn tokens.
 
@@ -177,7 +177,14 @@ def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None
     draft rows])` replaces the generated image embeddings (and the draft's image rows); used to
     put the image adapters in front of the prefill.  `uniforms`: "safe" (the oracle skips
     candidates inside the tolerance of a boundary) or "plain" (the seeded stream as it is).
-    `grid_mode`: launch shape (spd_cfg.grid_mode; 2 = one thread-block cluster per model)."""
+    `grid_mode`: launch shape (spd_cfg.grid_mode; 2 = one thread-block cluster per model).
+
+    `top_k`, `top_p`: truncated sampling on both sides.  The two sides may then also disagree on
+    which tokens survive the cut when a token's probability is within the logit error of it
+    (H.cut_zone): a decision that involves such a token is exempt (`cut_ambiguous`), and every
+    other probability of a truncated row is uncertain by the relative amount `rho` of its zone,
+    which widens the accept tolerance to 1e-4 + (p/q) * ((1 + rho_p)(1 + rho_q) - 1) and the CDF
+    band to (rho_p + rho_q + ambiguous mass) / (mass of the weights drawn from)."""
     spd = _lib()
     tw, dw = H.build_weights(wl, std)
     if gain_seed is not None:
@@ -191,8 +198,13 @@ def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None
             w.stored["final_norm"] = g.uniform(0.5, 1.5, cfg.d_model).astype(np.float32)
     max_seq = max_seq or (wl.n_image + wl.n_prompt + 8 * (n_blocks + 2) + 16)
     fp32 = wl.target.dtype == "fp32"
-    orc = H.make_oracle(wl, tw, dw, max_seq, temperature, greedy)
-    gpu = H.make_gpu(wl, tw, dw, max_seq, temperature, greedy, grid_mode=grid_mode)
+    trunc = (not greedy) and (top_k >= 1 or 0.0 < top_p < 1.0)
+    okp = top_p if 0.0 < top_p < 1.0 else 1.0
+    orc = H.make_oracle(wl, tw, dw, max_seq, temperature, greedy, top_k, okp)
+    gpu = H.make_gpu(wl, tw, dw, max_seq, temperature, greedy, grid_mode=grid_mode, top_k=top_k, top_p=top_p)
+
+    def zone(logits_row, eps):
+        return H.cut_zone(S.softmax_t(logits_row, temperature), top_k, okp, eps)
     img = synth.image_embeds(wl) if wl.n_image else None
     gpu_img = img
     feats = synth.image_features(wl) if wl.adapter_in else None
@@ -206,15 +218,15 @@ def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None
     su = (H.SafeUniforms if uniforms == "safe" else H.PlainUniforms)(wl.seeds["uniforms"], f"lock.{wl.name}.{greedy}")
     report = {"max_logit_err": 0.0, "max_draft_logit_err": 0.0, "tolerated": 0, "blocks": 0, "accepted": 0,
               "accept_within_tol": 0, "accept_beyond_tol": 0, "cdf_band_tokens": 0, "greedy_near_ties": 0,
-              "reprefills": 0, "decisions": 0, "draws": 0}
+              "reprefills": 0, "decisions": 0, "draws": 0, "cut_ambiguous": 0}
 
     # prefill: first token from the target's last row (Eq. 1)
     x0 = orc.prefill(img, ids, u0=None, draft_image_feats=feats) if greedy else None
     if not greedy:
         # choose u0 on the oracle side after seeing the row: run the target once to get it
-        probe = H.make_oracle(wl, tw, dw, max_seq, temperature, greedy)
+        probe = H.make_oracle(wl, tw, dw, max_seq, temperature, greedy, top_k, okp)
         probe.prefill(img, ids, u0=0.5, draft_image_feats=feats)
-        u0 = su.for_cdf(S.softmax_t(probe.prefill_logits, temperature))
+        u0 = su.for_cdf(probe._probs(probe.prefill_logits))
         del probe
         x0 = orc.prefill(img, ids, u0=u0, draft_image_feats=feats)
     g0 = gpu.prefill(gpu_img, ids, u0=None if greedy else u0, draft_image_feats=gpu_feats)
@@ -226,6 +238,12 @@ def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None
         if greedy:
             assert H.top2_gap(orc.prefill_logits) < 1e-2, "first token differs"
             report["greedy_near_ties"] += 1
+        elif trunc:
+            z = zone(orc.prefill_logits, err)
+            amb = z["maybe"] & ~z["sure"]
+            assert amb[g0] or amb[x0] or H.token_within_cdf_band(orc._probs(orc.prefill_logits), u0, g0,
+                                                                 z["rho"] + z["amb"] + 1e-6), "first token"
+            report["cut_ambiguous" if (amb[g0] or amb[x0]) else "cdf_band_tokens"] += 1
         else:
             assert H.token_within_cdf_band(S.softmax_t(orc.prefill_logits, temperature), u0, g0,
                                            H.cdf_band(fp32, err)), "first token outside the CDF band"
@@ -257,6 +275,16 @@ def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None
             if greedy:
                 assert H.top2_gap(orc.last_draft_logits[j]) < 1e-2, f"block {b}: draft token {j} differs"
                 report["greedy_near_ties"] += 1
+            elif trunc:
+                z = zone(orc.last_draft_logits[j], derr)
+                amb = z["maybe"] & ~z["sure"]
+                if amb[int(g_ids[j])] or amb[int(d_ids[j])]:
+                    report["cut_ambiguous"] += 1
+                else:
+                    assert H.token_within_cdf_band(q[j], orc.last_draft_u[j], int(g_ids[j]),
+                                                   z["rho"] + z["amb"] + 1e-6), \
+                        f"block {b}: draft token {j} = {g_ids[j]} outside the CDF band of {d_ids[j]}"
+                    report["cdf_band_tokens"] += 1
             else:
                 assert H.token_within_cdf_band(q[j], orc.last_draft_u[j], int(g_ids[j]), H.cdf_band(fp32, derr)), \
                     f"block {b}: draft token {j} = {g_ids[j]} outside the CDF band of {d_ids[j]}"
@@ -287,6 +315,17 @@ def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None
                 dist = H.accept_distance(p_x, q_x, orc.last_u[j])
                 if dist < H.ACCEPT_TOL:
                     report["accept_within_tol"] += 1
+                elif trunc:
+                    zp, zq = zone(orc.last_logits[j], verr), zone(orc.last_draft_logits[j], derr)
+                    if (zp["maybe"][x] and not zp["sure"][x]) or (zq["maybe"][x] and not zq["sure"][x]):
+                        report["cut_ambiguous"] += 1
+                    else:
+                        ratio = float(S.accept_prob(p_x, q_x))
+                        explained = ratio * ((1 + zp["rho"]) * (1 + zq["rho"]) - 1) + H.ACCEPT_TOL
+                        assert dist <= explained, \
+                            f"block {b}: accepted {ga} vs oracle {a}; |u - p/q| = {dist:.3e} at test {j} " \
+                            f"(cut zones explain {explained:.3e})"
+                        report["accept_beyond_tol"] += 1
                 else:
                     ratio = float(S.accept_prob(p_x, q_x))
                     explained = ratio * float(np.expm1(2.0 * (verr + derr))) + H.ACCEPT_TOL
@@ -298,14 +337,27 @@ def lockstep(wl, greedy, temperature, n_blocks, logit_tol, std=0.02, gammas=None
                 # same accept decisions; the drawn token may move to a neighbour of the oracle's
                 # when the logits differ: it must stay inside the CDF band
                 p_o = orc.last_p
+                ambiguous = False
                 if a == gamma:
                     w, band = p_o[gamma], H.cdf_band(fp32, verr)
+                    if trunc:
+                        zp = zone(orc.last_logits[gamma], verr)
+                        band = zp["rho"] + zp["amb"] + 1e-6
+                        ambiguous = bool((zp["maybe"] & ~zp["sure"])[[gn, nxt]].any())
                 else:
                     w = np.maximum(F32(0), p_o[a] - q[a])
-                    band = H.cdf_band(fp32, verr, derr, float(w.sum(dtype=np.float64)))
-                assert H.token_within_cdf_band(w, orc.last_u[gamma], gn, band), \
-                    f"block {b}: token {gn} outside the CDF band of the oracle's draw {nxt} (logit err {verr})"
-                report["cdf_band_tokens"] += 1
+                    mass = float(w.sum(dtype=np.float64))
+                    band = H.cdf_band(fp32, verr, derr, mass)
+                    if trunc:
+                        zp, zq = zone(orc.last_logits[a], verr), zone(orc.last_draft_logits[a], derr)
+                        band = (zp["rho"] + zp["amb"] + zq["rho"] + zq["amb"]) / max(mass, 1e-6) + 1e-6
+                        ambiguous = bool(((zp["maybe"] & ~zp["sure"]) | (zq["maybe"] & ~zq["sure"]))[[gn, nxt]].any())
+                if ambiguous:
+                    report["cut_ambiguous"] += 1
+                else:
+                    assert H.token_within_cdf_band(w, orc.last_u[gamma], gn, band), \
+                        f"block {b}: token {gn} outside the CDF band of the oracle's draw {nxt} (logit err {verr})"
+                    report["cdf_band_tokens"] += 1
             report["tolerated"] += 1
         report["blocks"] += 1
         report["accepted"] += a
@@ -451,6 +503,44 @@ def test_lockstep_on_unfiltered_uniforms(shape):
         assert r["blocks"] == 6
     print("unfiltered uniforms", shape, r)
     assert r["skipped_uniforms"] == 0 and r["decisions"] > 0 and r["draws"] > r["blocks"]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("shape,top_k,top_p", [("tiny", 40, 0.0), ("tiny", 0, 0.9), ("tiny", 64, 0.8),
+                                               ("llava7b-2L", 50, 0.9)])
+def test_lockstep_with_top_k_top_p(shape, top_k, top_p):
+    """Truncated sampling inside spd_prefill / spd_draft / spd_verify (spd_cfg.top_k, top_p): both
+    models' rows truncated and renormalised, draft tokens drawn from the truncated rows, the rule
+    on truncated rows -- block by block against the oracle running the same mode."""
+    if shape == "tiny":
+        r = lockstep(synth.tiny_workload(4), False, 1.0, 12, 2e-4, std=0.1, gammas=[4, 7, 2, 5], top_k=top_k,
+                     top_p=top_p)
+        assert r["blocks"] == 12
+    else:
+        wl = synth.llava7b_workload(gamma=5, n_layers=2, draft_layers=2)
+        r = lockstep(wl, False, 1.0, 4, 5e-2, top_k=top_k, top_p=top_p)
+        assert r["blocks"] == 4
+    print("top-k/top-p", shape, top_k, top_p, r)
+    assert r["accepted"] > 0
+
+
+@pytest.mark.gpu
+def test_top_k_one_sampling_reproduces_greedy_decoding():
+    """top_k = 1 leaves a point mass on every row of both models: the sampling path must then emit
+    exactly what greedy speculative decoding emits (which is the target's own greedy continuation,
+    Sec. 4 "Decoding"), through spd_generate's graph replay, for any uniforms."""
+    wl = synth.tiny_workload(4)
+    tw, dw = H.build_weights(wl, 0.2)
+    img, ids = synth.image_embeds(wl), synth.prompt_ids(wl)
+    g = H.make_gpu(wl, tw, dw, 128, 1.0, True)
+    g.prefill(img, ids)
+    want, _ = g.generate(wl.n_new, 4)
+    g.close()
+    t = H.make_gpu(wl, tw, dw, 128, 1.0, False, top_k=1)
+    t.prefill(img, ids, u0=0.6)
+    got, st = t.generate(wl.n_new, 4, synth.uniforms(13, "topk1.gpu", (wl.n_new, 9)))
+    t.close()
+    assert np.array_equal(got, want)
 
 
 # ------------------------------------------------------------------ block loop

@@ -44,3 +44,26 @@ def test_token_within_cdf_band_on_a_four_token_row():
     assert not H.token_within_cdf_band(w, u, 1, 5e-5)
     assert H.token_within_cdf_band(w, u, 1, 2e-4)
     assert not H.token_within_cdf_band(w, u, 3, 2e-4) and not H.token_within_cdf_band(w, u, 0, 2e-4)
+
+
+def test_cut_zone_brackets_every_admissible_kept_set():
+    """Perturb the logits of a row by up to eps many times: the kept set of the perturbed row must
+    contain `sure`, be contained in `maybe`, and every renormalised probability of a sure token
+    must stay within the relative uncertainty rho."""
+    from oracle import warp as W
+    g = np.random.default_rng(0)
+    V, eps = 400, 1e-3
+    for top_k, top_p in ((0, 0.9), (25, 1.0), (40, 0.7)):
+        logits = (g.standard_normal(V) * 1.5).astype(F32)
+        p = S.softmax_t(logits, 1.0)
+        z = H.cut_zone(p, top_k, top_p, eps)
+        base = W.warp_row(p, top_k, top_p)
+        assert z["sure"].sum() > 0 and np.all(z["maybe"][z["sure"]])
+        assert np.all(z["maybe"][base > 0]) and np.all(base[z["sure"]] > 0)
+        for _ in range(200):
+            pert = S.softmax_t(logits + g.uniform(-eps, eps, V).astype(F32), 1.0)
+            row = W.warp_row(pert, top_k, top_p)
+            kept = row > 0
+            assert np.all(kept[z["sure"]]) and not np.any(kept & ~z["maybe"])
+            rel = np.abs(row[z["sure"]] / base[z["sure"]] - 1.0)
+            assert rel.max() <= z["rho"] + 1e-6

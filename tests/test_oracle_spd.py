@@ -123,3 +123,53 @@ def test_draft_rows_given_in_its_own_space_equal_the_linear_adapter_applied_outs
     _, q_with = qa.draft(4, u[0, :4])
     _, q_without = c.draft(4, u[0, :4])
     assert np.abs(np.asarray(q_with[0]) - np.asarray(q_without[0])).max() > 1e-6
+
+
+def test_top_k_one_sampling_equals_greedy_decoding():
+    """top_k = 1 leaves a point mass at the arg-max of every row of both models, so the sampling
+    rule accepts a draft token iff it is the target's arg-max and otherwise emits that arg-max:
+    the whole loop must reproduce greedy speculative decoding (hence the target's own greedy
+    continuation, Sec. 4 "Decoding") whatever the uniforms are."""
+    wl = synth.tiny_workload(4)
+    img, ids = synth.image_embeds(wl), synth.prompt_ids(wl)
+    g = build(wl, greedy=True, std=0.2)
+    g.prefill(img, ids)
+    want = g.generate_target_only(wl.n_new)
+    o = build(wl, greedy=False, std=0.2)
+    o.top_k, o.truncate = 1, True
+    o.prefill(img, ids, u0=0.77)
+    u = synth.uniforms(11, "topk1", (wl.n_new, 9))
+    got, st = o.generate(wl.n_new, 4, u)
+    assert np.array_equal(got, want)
+
+
+def test_truncated_loop_emits_only_tokens_of_the_targets_kept_sets():
+    """With top-k / top-p on, every emitted token has non-zero probability in the target's
+    truncated row at its position (the rule's output law is the truncated target row), the
+    draft's rows handed to the rule are truncated rows (at most k non-zeros, sum 1), and
+    switching truncation off with k >= V and top_p = 1 changes nothing."""
+    from oracle import warp as W, sampling as S
+    wl = synth.tiny_workload(4)
+    img, ids = synth.image_embeds(wl), synth.prompt_ids(wl)
+    o = build(wl, greedy=False, std=0.1)
+    o.top_k, o.top_p, o.truncate = 20, 0.8, True
+    o.prefill(img, ids, u0=0.4)
+    u = synth.uniforms(12, "trunc.loop", (16, 9))
+    for b in range(8):
+        n0 = len(o.seq)
+        d_ids, q = o.draft(4, u[b, :4])
+        assert np.all((q > 0).sum(axis=1) <= 20) and np.allclose(q.sum(axis=1), 1.0, atol=1e-5)
+        assert all(q[j, d_ids[j]] > 0 for j in range(4))
+        a, nxt = o.verify(d_ids, q, u[b, 4:])
+        kept = W.warp_rows(S.softmax_t(o.last_logits, 1.0), 20, 0.8) > 0
+        assert np.array_equal(kept, o.last_p > 0)
+        emitted = o.seq[n0:]
+        assert all(kept[j, tok] for j, tok in enumerate(emitted))
+    full = build(wl, greedy=False, std=0.1)
+    off = build(wl, greedy=False, std=0.1)
+    off.top_k, off.top_p, off.truncate = wl.target.vocab, 1.0, True
+    for m in (full, off):
+        m.prefill(img, ids, u0=0.4)
+    a1, _ = full.generate(12, 4, u)
+    a2, _ = off.generate(12, 4, u)
+    assert np.array_equal(a1, a2)
