@@ -200,6 +200,48 @@ spd_status spd_verify(spd_ctx* ctx, int gamma, const int32_t* draft_ids,
                       const float* draft_probs, const float* uniforms,
                       int32_t* n_accepted, int32_t* next_token);
 
+/* ---- tree blocks (Sec. 5: "recent advancement in SPD algorithm to tree-based decoding can also be
+ * used"; the paper defines no rule).  Built here: several candidates per position, verified in ONE
+ * target call with a tree attention mask, by the multi-candidate rejection rule of the token-tree
+ * systems the paper cites, which keeps Sec. 2.1's guarantee (emitted tokens follow the target's
+ * distribution) when the candidates of a node are drawn independently from the draft's
+ * distribution at that node.  Block rows: 0 = the pending token (root), 1..n = draft nodes,
+ * parents before children; n <= gamma_max <= 7.  Every node gets its own K/V cache row while
+ * siblings share a sequence position; a node attends the committed prefix, its ancestors and
+ * itself.  Rule: starting at the root with cur = p_root, the children of the current node are
+ * tried in row order; child c is accepted iff u[c-1] < min(1, cur(x_c) / q_node(x_c)); on
+ * acceptance the walk descends (cur = p_c); on rejection cur <- max(0, cur - q_node) / sum and the
+ * next child is tried; when no child is left the next token is drawn from cur with u[n].  Greedy:
+ * a child is accepted iff it is the arg-max of p_node, else that arg-max is emitted.  A chain
+ * (one child per node) is exactly spd_draft / spd_verify.  Afterwards the K/V rows of the
+ * accepted nodes are moved to the positions they now hold, in both caches. */
+
+/* Draft tree: every node at depth d-1 gets branching[d-1] children (d = 1..depth), drawn
+ * independently from the draft's softmax(logits / T) at that node (greedy: its branching[d-1] most
+ * probable tokens); the draft runs level by level, each level one tree-masked launch.
+ *   branching    int32 [depth], HOST; the node count n = sum over levels must be <= gamma_max
+ *   uniforms     fp32 [n], host or device: uniforms[i-1] draws node i; may be NULL when greedy
+ *   node_ids     int32 [n], out, host or device, may be NULL (kept internally)
+ *   parent_out   int32 [n+1], out, HOST, may be NULL: parent_out[0] = -1, rows level by level
+ *   draft_probs  fp32 [n+1, vocab], out, DEVICE, may be NULL (kept internally): row r = the draft's
+ *                distribution at block row r (rows of leaves unused); not written when greedy */
+spd_status spd_draft_tree(spd_ctx* ctx, int depth, const int32_t* branching, const float* uniforms,
+                          int32_t* node_ids, int32_t* parent_out, float* draft_probs);
+
+/* Tree verification: one target call on [pending ; node_1..node_n] with the tree mask, the rule
+ * above, commit of the accepted path and the next token, K/V compaction.
+ *   parent       int32 [n+1], HOST, parent[0] = -1, parent[i] in 0..i-1
+ *   node_ids     int32 [n], host or device; NULL = those of the last spd_draft_tree (same shape)
+ *   draft_probs  fp32 [n+1, vocab], DEVICE; NULL = those of the last spd_draft_tree; unused when greedy
+ *   uniforms     fp32 [n+1], host or device: n accept tests, then the one final draw; NULL when greedy
+ *   n_accepted   int32, out: length of the accepted path
+ *   path         int32 [depth of the tree], out: block rows of the accepted nodes, root downwards
+ *   next_token   int32, out
+ * Outputs may be host or device memory or NULL. */
+spd_status spd_verify_tree(spd_ctx* ctx, int n_nodes, const int32_t* parent, const int32_t* node_ids,
+                           const float* draft_probs, const float* uniforms, int32_t* n_accepted, int32_t* path,
+                           int32_t* next_token);
+
 /* Block loop (Fig. 1): repeats draft + verify until n_new tokens exist after the prompt;
  * the pending token (after spd_prefill: the token it produced) is the first of them.
  *   uniforms  fp32 [n_new, 2*gamma+1], host or device: per block gamma draft draws, then

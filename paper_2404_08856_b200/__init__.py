@@ -22,7 +22,7 @@ EXPORTS = ["spd_create", "spd_destroy", "spd_fork", "spd_last_error", "spd_prefi
            "spd_generate", "spd_get_logits", "spd_get_draft_logits", "spd_rollback", "spd_get_state",
            "spd_reject_sample", "spd_skinny_gemm", "spd_verify_bytes", "spd_trace",
            "spd_skinny_gemm_noalloc", "spd_image_adapter", "spd_truncate_probs", "spd_skinny_gemm_status",
-           "spd_wait_selftest"]
+           "spd_wait_selftest", "spd_draft_tree", "spd_verify_tree"]
 
 
 class SpdError(RuntimeError):
@@ -184,6 +184,33 @@ class Spd:
         self._check(lib().spd_verify(self._ctx, gamma, _ptr(ids), _ptr(draft_probs), _ptr(u), C.byref(a),
                                      C.byref(nxt)))
         return a.value, nxt.value
+
+    def draft_tree(self, branching, uniforms=None, probs_out=None):
+        """See spd_draft_tree.  Returns (parent [n+1], node ids [n])."""
+        br = np.ascontiguousarray(branching, dtype=np.int32)
+        n, lvl = 0, 1
+        for b in br:
+            lvl *= int(b)
+            n += lvl
+        ids = np.zeros(max(n, 1), dtype=np.int32)
+        parent = np.zeros(max(n, 1) + 1, dtype=np.int32)
+        u = None if uniforms is None else np.ascontiguousarray(uniforms, dtype=np.float32)
+        self._check(lib().spd_draft_tree(self._ctx, len(br), _ptr(br), _ptr(u), _ptr(ids), _ptr(parent),
+                                         _ptr(probs_out)))
+        return parent[: n + 1], ids[:n]
+
+    def verify_tree(self, parent, uniforms=None, node_ids=None, draft_probs=None):
+        """See spd_verify_tree.  Returns (path, next_token)."""
+        par = np.ascontiguousarray(parent, dtype=np.int32)
+        n = len(par) - 1
+        u = None if uniforms is None else np.ascontiguousarray(uniforms, dtype=np.float32)
+        ids = node_ids if (node_ids is None or hasattr(node_ids, "data_ptr")) \
+            else np.ascontiguousarray(node_ids, dtype=np.int32)
+        a, nxt = C.c_int32(0), C.c_int32(0)
+        path = np.zeros(8, dtype=np.int32)
+        self._check(lib().spd_verify_tree(self._ctx, n, _ptr(par), _ptr(ids), _ptr(draft_probs), _ptr(u),
+                                          C.byref(a), _ptr(path), C.byref(nxt)))
+        return [int(x) for x in path[: a.value]], nxt.value
 
     def draft_async(self, gamma: int, uniforms_dev=None):
         """Enqueue gamma draft steps with device-resident uniforms; nothing is read back."""

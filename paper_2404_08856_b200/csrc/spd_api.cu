@@ -12,6 +12,7 @@
 #include "spd_kernel.cuh"
 #include "spd_prefill.cuh"
 #include "spd_warp.cuh"
+#include "spd_tree.cuh"
 
 using namespace spd;
 
@@ -51,6 +52,11 @@ struct spd_ctx {
   float* qbuf = nullptr;        // [gamma_max][V] draft distributions
   float* prow = nullptr;        // [MAX_M][V] probability rows of the step being sampled (top-k / top-p only)
   bool truncate = false;        // top-k / top-p switched on
+  // tree blocks (spd_draft_tree / spd_verify_tree): scratch allocated on first use
+  float* tree_cur = nullptr;    // [V] renormalised residual between sibling candidates
+  char *tree_stage_t = nullptr, *tree_stage_d = nullptr;   // K/V rows in flight during compaction
+  TreeShape tree_shape{};       // shape of the last spd_draft_tree
+  bool tree_drafted = false;
   float* rows = nullptr;        // prefill rows staging [max_seq][d_max]
   int* ids_dev = nullptr;       // prompt ids [max_seq]
   float* upool = nullptr; size_t upool_cap = 0;
@@ -469,7 +475,7 @@ spd_status launch_forward(spd_ctx* ctx, int M, int dtype, StepArgs a, cudaStream
   // sampling (not greedy): the forward kernel has left logits and per-slice row statistics; two
   // small kernels spread the draw over the whole device and commit the step
   const bool samples = a.mode == MODE_VERIFY || a.mode == MODE_DRAFT || (a.mode == MODE_ROWS && a.want_sample);
-  if (samples && !a.greedy) {
+  if (samples && !a.greedy && !a.tree) {
     if (ctx && ctx->truncate) {
       // top-k / top-p: probability rows -> truncated and renormalised in place -> the rule on rows
       const int nrows = a.mode == MODE_VERIFY ? a.gamma + 1 : 1;
@@ -526,6 +532,29 @@ spd_status copy_out(spd_ctx* ctx, void* dst, const void* src_dev, size_t bytes, 
   return SPD_OK;
 }
 
+// Row tables of the two plain launches (spd_engine.cuh, RowGeom).  Verify: the chain
+// [pending, x_1..x_gamma] from the origin on.  Draft step j: the two rows [token before, token to
+// extend] at slots j-1 and j (slot -1 is the previous token's row, recomputed identically).
+void geom_verify_chain(StepArgs& a, int gamma) {
+  for (int m = 0; m <= gamma; ++m) {
+    a.geo.slot[m] = a.geo.depth[m] = (signed char)m;
+    a.geo.sees[m] = (unsigned char)((2u << m) - 1u);
+    a.geo.src[m] = (signed char)(m - 1);
+  }
+  a.n_slots = gamma + 1;
+  a.stat_r0 = 0; a.stat_n = gamma + 1;
+}
+void geom_draft_step(StepArgs& a, int j) {
+  a.geo.slot[0] = a.geo.depth[0] = (signed char)(j - 1);
+  a.geo.sees[0] = (unsigned char)((1u << j) - 1u);
+  a.geo.src[0] = (signed char)(j == 0 ? -2 : j - 2);
+  a.geo.slot[1] = a.geo.depth[1] = (signed char)j;
+  a.geo.sees[1] = (unsigned char)((2u << j) - 1u);
+  a.geo.src[1] = (signed char)(j - 1);
+  a.n_slots = j + 1;
+  a.stat_r0 = 1; a.stat_n = 1;
+}
+
 StepArgs base_args(spd_ctx* ctx, ModelHost& mh) {
   StepArgs a{};
   a.md = mh.md;
@@ -549,6 +578,7 @@ spd_status feed_rows(spd_ctx* ctx, ModelHost& mh, const float* rows_dev, const i
     a.row_ids = ids_dev ? ids_dev + r : nullptr;
     a.rows_pos0 = pos0 + (r - r0);
     a.want_sample = sample_last && (r + M >= r1);
+    a.stat_r0 = M - 1; a.stat_n = 1;
     a.init_n_text = init_n_text;
     a.init_prev = init_prev;
     a.uniforms = ctx->ubuf + 8;
@@ -718,7 +748,7 @@ spd_status alloc_ctx_buffers(spd_ctx* ctx) {
   if ((s = dalloc(ctx, &ctx->st, 1))) return s;
   if ((s = dalloc(ctx, &ctx->bars, (size_t)32 * BAR_POOL))) return s;
   if ((s = dalloc(ctx, &ctx->ubuf, 16))) return s;
-  if ((s = dalloc(ctx, &ctx->qbuf, (size_t)(cfg->gamma_max > 0 ? cfg->gamma_max : 1) * V))) return s;
+  if ((s = dalloc(ctx, &ctx->qbuf, (size_t)MAX_M * V))) return s;   // chain: gamma rows; tree: one per block row
   ctx->truncate = !cfg->greedy && ((cfg->top_k >= 1 && cfg->top_k < V) || (cfg->top_p > 0.f && cfg->top_p < 1.f));
   if (ctx->truncate) {
     if ((s = dalloc(ctx, &ctx->prow, (size_t)MAX_M * V))) return s;
@@ -959,6 +989,7 @@ spd_status spd_prefill(spd_ctx* ctx, const float* image_embeds, int m, const flo
     CU(cudaMemcpyAsync(tm.md.x, X + (size_t)(Rt - 1) * dt, dt * sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));
     StepArgs a = base_args(ctx, tm);
     a.mode = MODE_ROWS; a.skip_layers = 1; a.want_sample = 1;
+    a.stat_r0 = 0; a.stat_n = 1;
     a.rows = tm.md.x; a.rows_pos0 = Rt - 1;
     a.init_n_text = n; a.init_prev = last_id;
     a.uniforms = ctx->ubuf + 8; a.out_ids = ctx->out_dev;
@@ -1078,6 +1109,7 @@ spd_status spd_draft(spd_ctx* ctx, int gamma, const float* uniforms, int32_t* dr
     StepArgs a = base_args(ctx, dm);
     a.mode = MODE_DRAFT;
     a.gamma = gamma; a.j = j;
+    geom_draft_step(a, j);
     a.uniforms = ctx->ubuf;
     a.q_out = ctx->qbuf;
     a.logits = dm.logits;
@@ -1125,6 +1157,7 @@ spd_status spd_verify(spd_ctx* ctx, int gamma, const int32_t* draft_ids, const f
   StepArgs a = base_args(ctx, tm);
   a.mode = MODE_VERIFY;
   a.gamma = gamma;
+  geom_verify_chain(a, gamma);
   a.uniforms = ctx->ubuf + 8;
   a.q_in = draft_probs ? draft_probs : ctx->qbuf;
   a.out_ids = nullptr;
@@ -1137,6 +1170,181 @@ spd_status spd_verify(spd_ctx* ctx, int gamma, const int32_t* draft_ids, const f
   bool need_sync = false;
   if ((s = copy_out(ctx, n_accepted, &ctx->st->n_acc, sizeof(int32_t), &need_sync))) return s;
   if ((s = copy_out(ctx, next_token, &ctx->st->next, sizeof(int32_t), &need_sync))) return s;
+  if (need_sync) return sync_state(ctx);
+  return SPD_OK;
+}
+
+// ---- tree blocks
+
+static spd_status tree_scratch(spd_ctx* ctx) {
+  if (ctx->tree_cur) return SPD_OK;
+  spd_status s;
+  const ModelHost &tm = ctx->target, &dm = ctx->draft;
+  if ((s = dalloc(ctx, &ctx->tree_stage_t, (size_t)2 * tm.cfg.n_layers * MAX_M * tm.cfg.d_model * tm.esz))) return s;
+  if ((s = dalloc(ctx, &ctx->tree_stage_d, (size_t)2 * dm.cfg.n_layers * MAX_M * dm.cfg.d_model * dm.esz))) return s;
+  if (!ctx->prow && (s = dalloc(ctx, &ctx->prow, (size_t)MAX_M * ctx->cfg.target.vocab))) return s;
+  if ((s = dalloc(ctx, &ctx->tree_cur, (size_t)ctx->cfg.target.vocab))) return s;
+  return SPD_OK;
+}
+
+static spd_status tree_shape_from_parent(spd_ctx* ctx, int n, const int32_t* parent, TreeShape* sh, unsigned char* sees) {
+  if (n < 1 || n > MAX_M - 1 || !parent || parent[0] != -1) return fail(ctx, SPD_EINVAL, "bad tree: 1..7 nodes, parent[0] = -1");
+  sh->n = n; sh->depth_max = 0;
+  sh->parent[0] = -1; sh->depth[0] = 0; sees[0] = 1;
+  for (int i = 1; i <= n; ++i) {
+    if (parent[i] < 0 || parent[i] >= i) return fail(ctx, SPD_EINVAL, "bad tree: parent[i] must lie in 0..i-1");
+    sh->parent[i] = (signed char)parent[i];
+    sh->depth[i] = (signed char)(sh->depth[parent[i]] + 1);
+    sees[i] = (unsigned char)(sees[parent[i]] | (1u << i));
+    if (sh->depth[i] > sh->depth_max) sh->depth_max = sh->depth[i];
+  }
+  for (int i = n + 1; i < MAX_M; ++i) { sh->parent[i] = -1; sh->depth[i] = 0; }
+  return SPD_OK;
+}
+
+// probability rows of the launch's statistic rows (truncated when top-k / top-p is on)
+static spd_status tree_prob_rows(spd_ctx* ctx, const StepArgs& a, cudaStream_t stream) {
+  prob_rows_kernel<<<ctx->n_sm, SAMPLE_THREADS, 0, stream>>>(a, ctx->prow);
+  if (ctx->truncate)
+    truncate_rows_kernel<<<a.stat_n, WARP_THREADS, (size_t)a.md.V * sizeof(float), stream>>>(
+        ctx->prow, ctx->prow, a.md.V, ctx->cfg.top_k, ctx->cfg.top_p > 0.f ? ctx->cfg.top_p : 1.0f);
+  CU(cudaGetLastError());
+  return SPD_OK;
+}
+
+spd_status spd_draft_tree(spd_ctx* ctx, int depth, const int32_t* branching, const float* uniforms,
+                          int32_t* node_ids, int32_t* parent_out, float* draft_probs) {
+  if (!ctx) return SPD_EINVAL;
+  if (!ctx->prefilled) return fail(ctx, SPD_ESTATE, "spd_draft_tree before spd_prefill");
+  if (depth < 1 || depth > MAX_M - 1 || !branching) return fail(ctx, SPD_EINVAL, "bad tree depth / branching");
+  if (!ctx->cfg.greedy && !uniforms) return fail(ctx, SPD_EINVAL, "uniforms required when sampling");
+  if (draft_probs && !is_device_ptr(draft_probs)) return fail(ctx, SPD_EINVAL, "draft_probs must be device memory");
+  // level-order parent table: every node at depth d-1 gets branching[d-1] children
+  int32_t parent[MAX_M + 1];
+  int n = 0, lvl_first = 0, lvl_n = 1;
+  parent[0] = -1;
+  for (int d = 0; d < depth; ++d) {
+    if (branching[d] < 1) return fail(ctx, SPD_EINVAL, "branching must be >= 1");
+    if ((long long)lvl_n * branching[d] + n > MAX_M - 1 || (long long)lvl_n * branching[d] + n > ctx->cfg.gamma_max)
+      return fail(ctx, SPD_EINVAL, "tree has more nodes than gamma_max (at most 7)");
+    const int first_new = n + 1;
+    for (int k = 0; k < lvl_n; ++k)
+      for (int b = 0; b < branching[d]; ++b) parent[++n] = lvl_first + k;
+    lvl_first = first_new; lvl_n = n + 1 - first_new;
+  }
+  TreeShape sh{};
+  unsigned char sees[MAX_M];
+  spd_status s = tree_shape_from_parent(ctx, n, parent, &sh, sees);
+  if (s) return s;
+  if ((s = tree_scratch(ctx))) return s;
+  const int base = ctx->m_image > ctx->draft.pos_base ? ctx->m_image : ctx->draft.pos_base;
+  if (base + ctx->len_ub + n + 1 > ctx->cfg.max_seq) {
+    if ((s = sync_state(ctx))) return s;
+    if (base + ctx->len_ub + n + 1 > ctx->cfg.max_seq) return fail(ctx, SPD_EOVERFLOW, "KV cache full");
+  }
+  if (uniforms) CU(cudaMemcpyAsync(ctx->ubuf, uniforms, n * sizeof(float), cudaMemcpyDefault, ctx->stream));
+  ModelHost& dm = ctx->draft;
+  for (int lev = 0; lev < depth; ++lev) {
+    StepArgs a = base_args(ctx, dm);
+    a.mode = MODE_DRAFT; a.gamma = n; a.j = lev; a.tree = 1;
+    a.uniforms = ctx->ubuf; a.q_out = ctx->qbuf; a.logits = dm.logits;
+    int M;
+    if (lev == 0) {           // the rows the draft has not seen: [previous token, pending token = root]
+      geom_draft_step(a, 0);
+      a.geo.slot[1] = 0;      // (already so: the root is block row 0)
+      M = 2;
+    } else {                  // the nodes of this depth, each attending its ancestors
+      M = 0;
+      for (int i = 1; i <= n; ++i)
+        if (sh.depth[i] == lev) {
+          a.geo.slot[M] = (signed char)i; a.geo.depth[M] = (signed char)lev;
+          a.geo.sees[M] = sees[i]; a.geo.src[M] = (signed char)(i - 1);
+          ++M;
+        }
+      a.n_slots = n + 1;
+      a.stat_r0 = 0; a.stat_n = M;
+    }
+    if ((s = launch_model(ctx, dm, M, a, ctx->stream))) return s;
+    a.fwd_grid = dm.grid; a.sample_r0 = M - 1;
+    if (!ctx->cfg.greedy && (s = tree_prob_rows(ctx, a, ctx->stream))) return s;
+    tree_draw_kernel<<<1, SAMPLE_THREADS, 0, ctx->stream>>>(a, sh, ctx->prow);
+    CU(cudaGetLastError());
+  }
+  ctx->tree_shape = sh;
+  ctx->tree_drafted = true;
+  ctx->drafted_gamma = -1;
+  bool need_sync = false;
+  if (draft_probs && !ctx->cfg.greedy)
+    CU(cudaMemcpyAsync(draft_probs, ctx->qbuf, (size_t)(n + 1) * dm.cfg.vocab * sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));
+  if ((s = copy_out(ctx, node_ids, ctx->st->d_ids, n * sizeof(int32_t), &need_sync))) return s;
+  if (parent_out) memcpy(parent_out, parent, (n + 1) * sizeof(int32_t));
+  if (need_sync) CU(cudaStreamSynchronize(ctx->stream));
+  return SPD_OK;
+}
+
+spd_status spd_verify_tree(spd_ctx* ctx, int n_nodes, const int32_t* parent, const int32_t* node_ids,
+                           const float* draft_probs, const float* uniforms, int32_t* n_accepted, int32_t* path,
+                           int32_t* next_token) {
+  if (!ctx) return SPD_EINVAL;
+  if (!ctx->prefilled) return fail(ctx, SPD_ESTATE, "spd_verify_tree before spd_prefill");
+  if (!ctx->cfg.greedy && !uniforms) return fail(ctx, SPD_EINVAL, "uniforms required when sampling");
+  if (draft_probs && !is_device_ptr(draft_probs)) return fail(ctx, SPD_EINVAL, "draft_probs must be device memory");
+  if (n_nodes > ctx->cfg.gamma_max) return fail(ctx, SPD_EINVAL, "tree has more nodes than gamma_max");
+  TreeShape sh{};
+  unsigned char sees[MAX_M];
+  spd_status s = tree_shape_from_parent(ctx, n_nodes, parent, &sh, sees);
+  if (s) return s;
+  const int n = n_nodes;
+  if ((!node_ids || (!ctx->cfg.greedy && !draft_probs)) &&
+      (!ctx->tree_drafted || ctx->tree_shape.n != n || memcmp(ctx->tree_shape.parent, sh.parent, sizeof(sh.parent))))
+    return fail(ctx, SPD_ESTATE, "spd_verify_tree needs the ids and probabilities of an spd_draft_tree of the same shape");
+  if ((s = tree_scratch(ctx))) return s;
+  if (ctx->m_image + ctx->len_ub + n + 1 > ctx->cfg.max_seq) {
+    if ((s = sync_state(ctx))) return s;
+    if (ctx->m_image + ctx->len_ub + n + 1 > ctx->cfg.max_seq) return fail(ctx, SPD_EOVERFLOW, "KV cache full");
+  }
+  const int V = ctx->cfg.target.vocab;
+  if (node_ids) {
+    if (!is_device_ptr(node_ids))
+      for (int j = 0; j < n; ++j)
+        if (node_ids[j] < 0 || node_ids[j] >= V) return fail(ctx, SPD_EINVAL, "node id out of range");
+    CU(cudaMemcpyAsync(ctx->st->d_ids, node_ids, n * sizeof(int32_t), cudaMemcpyDefault, ctx->stream));
+  }
+  if (uniforms) CU(cudaMemcpyAsync(ctx->ubuf + 8, uniforms, (n + 1) * sizeof(float), cudaMemcpyDefault, ctx->stream));
+  ModelHost &tm = ctx->target, &dm = ctx->draft;
+  StepArgs a = base_args(ctx, tm);
+  a.mode = MODE_VERIFY; a.gamma = n; a.tree = 1;
+  for (int i = 0; i <= n; ++i) {
+    a.geo.slot[i] = (signed char)i; a.geo.depth[i] = sh.depth[i];
+    a.geo.sees[i] = sees[i]; a.geo.src[i] = (signed char)(i - 1);
+  }
+  a.n_slots = n + 1;
+  a.stat_r0 = 0; a.stat_n = n + 1;
+  a.uniforms = ctx->ubuf + 8;
+  a.q_in = draft_probs ? draft_probs : ctx->qbuf;
+  a.out_ids = nullptr;
+  if ((s = launch_model(ctx, tm, n + 1, a, ctx->stream))) return s;
+  a.fwd_grid = tm.grid; a.sample_r0 = n;
+  if (!ctx->cfg.greedy && (s = tree_prob_rows(ctx, a, ctx->stream))) return s;
+  tree_verify_kernel<<<1, SAMPLE_THREADS, 0, ctx->stream>>>(a, sh, ctx->prow, ctx->tree_cur);
+  // accepted rows move up to the positions they now hold, in both caches (the draft was fed the
+  // nodes above the deepest level only)
+  for (int pass = 0; pass < 2; ++pass) {
+    tree_gather_kernel<<<dim3(MAX_M - 1, tm.cfg.n_layers, 2), 256, 0, ctx->stream>>>(
+        ctx->st, tm.md, tm.pos_base, (int)tm.esz, sh.depth_max, ctx->tree_stage_t, pass);
+    if (sh.depth_max > 1)
+      tree_gather_kernel<<<dim3(MAX_M - 1, dm.cfg.n_layers, 2), 256, 0, ctx->stream>>>(
+          ctx->st, dm.md, dm.pos_base, (int)dm.esz, sh.depth_max - 1, ctx->tree_stage_d, pass);
+  }
+  CU(cudaGetLastError());
+  ctx->tree_drafted = false;
+  ctx->drafted_gamma = -1;
+  ctx->len_ub += sh.depth_max + 1;
+  ctx->last_verify_rows = n + 1;
+  bool need_sync = false;
+  if ((s = copy_out(ctx, n_accepted, &ctx->st->n_acc, sizeof(int32_t), &need_sync))) return s;
+  if ((s = copy_out(ctx, next_token, &ctx->st->next, sizeof(int32_t), &need_sync))) return s;
+  if ((s = copy_out(ctx, path, ctx->st->path, sh.depth_max * sizeof(int32_t), &need_sync))) return s;
   if (need_sync) return sync_state(ctx);
   return SPD_OK;
 }
@@ -1181,12 +1389,14 @@ spd_status spd_generate(spd_ctx* ctx, int n_new, int gamma, const float* uniform
     for (int j = 0; j < gamma; ++j) {
       StepArgs a = base_args(ctx, dm);
       a.mode = MODE_DRAFT; a.gamma = gamma; a.j = j;
+      geom_draft_step(a, j);
       a.uniforms = uniforms ? ctx->upool : nullptr; a.u_stride = us; a.u_by_block = 1;
       a.q_out = ctx->qbuf; a.logits = dm.logits;
       if ((r = launch_model(ctx, dm, 2, a, cs))) return r;
     }
     StepArgs a = base_args(ctx, tm);
     a.mode = MODE_VERIFY; a.gamma = gamma;
+    geom_verify_chain(a, gamma);
     a.uniforms = uniforms ? ctx->upool : nullptr; a.u_stride = us; a.u_by_block = 1;
     a.q_in = ctx->qbuf; a.out_ids = ctx->out_dev;
     return launch_model(ctx, tm, gamma + 1, a, cs);

@@ -89,13 +89,38 @@ struct DevState {
   int d_ids[MAX_M];
   int out_cap;
   int pad[3];
+  int path[MAX_M];   // tree blocks: block rows of the accepted nodes, root downwards (n_acc of them)
   // %globaltimer (ns) at the start / end of the last draft steps and verify step
   unsigned long long t_draft0, t_draft1, t_verify0, t_verify1;
 };
 static_assert(sizeof(DevState) <= 256, "the fixed scratch of spd_skinny_gemm_noalloc reserves 256 bytes for it");
 
+// Geometry of the M rows of a decode launch relative to the ORIGIN = sequence position of the
+// pending token (the root of the block).  A plain block is the chain slot = depth = m,
+// sees = {0..m}; a token tree (Sec. 5) gives every node its own cache row (slot) while siblings
+// share a depth, and a node attends its ancestors and itself only.
+struct RowGeom {
+  signed char slot[MAX_M];     // K/V cache row = origin + slot (-1: the row of the previous token)
+  signed char depth[MAX_M];    // rotary position = origin + depth
+  unsigned char sees[MAX_M];   // bit s set: the row attends cache row origin + s; rows below the origin always
+  signed char src[MAX_M];      // token of the row: -2 previous token, -1 pending token, k >= 0 draft token k
+};
+
+// A token tree below the pending token: block row 0 is the root (the pending token itself), rows
+// 1..n are draft nodes in an order in which parents come first.
+struct TreeShape {
+  int n;                       // draft nodes, 1..MAX_M-1
+  int depth_max;               // depth of the deepest node
+  signed char parent[MAX_M];   // parent[i] < i: block row of node i's parent; parent[0] = -1
+  signed char depth[MAX_M];    // depth[0] = 0
+};
+
 struct StepArgs {
   ModelDev md;            // by value: read through the constant bank
+  RowGeom geo;
+  int n_slots;            // cache rows from the origin on that this launch may attend (max slot + 1)
+  int stat_r0, stat_n;    // rows of `logits` whose softmax statistics the kernel leaves for the sampling kernels
+  int tree;               // 1: a tree block -- the rule runs in the tree kernels, never inside this kernel
   DevState* st;
   unsigned* bar;          // grid-barrier counter, zero at launch
   int mode, gamma, j, pos_base, nstage, greedy;
@@ -133,6 +158,9 @@ struct Ctrl {
   float rowmax[MAX_M], rowsum[MAX_M];
   int flag;
   int tok[MAX_M];                   // token ids of the M rows
+  int rowslot[MAX_M];               // absolute K/V cache row of each of the M rows
+  int rowpos[MAX_M];                // rotary position of each row
+  unsigned sees[MAX_M];             // bit s: attends cache row origin + s
   int trace_n;                      // entries written so far (CTA 0 only)
   unsigned long long* trace;        // NULL: tracing off
 };
@@ -387,7 +415,8 @@ struct EpiArgs {
   // QKV
   float* qbuf; void* kc; void* vc;  // cache bases already offset to the layer
   const float *cs, *sn;
-  int pos0, d, dh;
+  const int *rowslot, *rowpos;      // per activation row: cache row to append to, rotary position (shared memory)
+  int d, dh;
 };
 
 __device__ __forceinline__ void cache_store(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
@@ -409,13 +438,14 @@ __device__ __forceinline__ void epilogue_pair(int epi, const EpiArgs& e, int m, 
     stcg(e.out + (size_t)m * e.ldo + (n >> 1), s * b);
   } else {  // EPI_QKV: rows are [q | k | v]; q and k rows are stored pair-interleaved
     const int region = n / e.d, c = n - region * e.d;
-    const int pos = e.pos0 + m;
+    const int slot = e.rowslot[m];
     if (region == 2) {
-      WT* vp = static_cast<WT*>(e.vc) + (size_t)pos * e.d + c;
+      WT* vp = static_cast<WT*>(e.vc) + (size_t)slot * e.d + c;
       cache_store(vp, a);
       cache_store(vp + 1, b);
     } else {
       const int h = c / e.dh, i = (c - h * e.dh) >> 1, half = e.dh >> 1;
+      const int pos = e.rowpos[m];
       const float cs = e.cs[pos * half + i], sn = e.sn[pos * half + i];
       const float ra = a * cs - b * sn, rb = b * cs + a * sn;
       const int c0 = h * e.dh + i;
@@ -423,7 +453,7 @@ __device__ __forceinline__ void epilogue_pair(int epi, const EpiArgs& e, int m, 
         stcg(e.qbuf + (size_t)m * e.d + c0, ra);
         stcg(e.qbuf + (size_t)m * e.d + c0 + half, rb);
       } else {
-        WT* kp = static_cast<WT*>(e.kc) + (size_t)pos * e.d + c0;
+        WT* kp = static_cast<WT*>(e.kc) + (size_t)slot * e.d + c0;
         cache_store(kp, ra);
         cache_store(kp + half, rb);
       }
@@ -781,18 +811,20 @@ __device__ __forceinline__ void frag_from_smem(const char* p, float (&f)[CTraits
   }
 }
 
-// Query row m (position pos0+m) attends cache rows 0..pos0+m.  Work unit = (head, KV
+// Query row m attends every cache row below `origin` and, of the `nslots` rows from the origin
+// on, those named in ctl->sees[m] (a chain: rows origin..origin+m).  Work unit = (head, KV
 // split).  The unit's K and V rows are brought into shared memory with asynchronous
 // 16-byte copies, all in flight at once (one memory latency), in sub-chunks that fit the
 // scratch region, with a running (online) softmax across sub-chunks.  Each unit leaves an
 // unnormalised partial output with its row max and sum; the CTA that finishes a head's
 // last split merges them (no waiting).
 template <int M, typename CT>
-__device__ void attn_phase(const ModelDev& md, int layer, int pos0, int cta, int G, char* xs, int xbytes, Ctrl* ctl) {
+__device__ void attn_phase(const ModelDev& md, int layer, int origin, int nslots, int cta, int G, char* xs, int xbytes,
+                           Ctrl* ctl) {
   constexpr int E = CTraits<CT>::E;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int H = md.H, dh = md.dh, d = md.d;
-  const int len = pos0 + M;
+  const int len = origin + nslots;
   const int nsplit = eff_nsplit(md, len);
   const int Lc = (len + nsplit - 1) / nsplit;
   const int LPP = dh / E, PPI = 32 / LPP;
@@ -860,7 +892,10 @@ __device__ void attn_phase(const ModelDev& md, int layer, int pos0, int cta, int
           for (int m = 0; m < M; ++m) part[m] += __shfl_xor_sync(0xffffffffu, part[m], o);
         if (r < n && li == 0) {
 #pragma unroll
-          for (int m = 0; m < M; ++m) S[m * SC + r] = (c0 + r <= pos0 + m) ? part[m] : -INFINITY;
+          for (int m = 0; m < M; ++m) {
+            const int rel = c0 + r - origin;
+            S[m * SC + r] = (rel < 0 || ((ctl->sees[m] >> rel) & 1u)) ? part[m] : -INFINITY;
+          }
         }
       }
       named_sync(1, CONSUMER_THREADS);
@@ -979,11 +1014,11 @@ __device__ __forceinline__ void split_frag(float2 xa, float2 xb, uint32_t& h0, u
 // ldmatrix) x P^T (B, fp32 probabilities split the same way); warp w owns dims 16w..16w+15,
 // so no cross-warp reduction is needed.  Tile rows are 16-byte-chunk swizzled by position.
 template <int M>
-__device__ void attn_phase_mma(const ModelDev& md, int layer, int pos0, int cta, int G, char* xs, int xbytes,
-                               Ctrl* ctl) {
+__device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int nslots, int cta, int G, char* xs,
+                               int xbytes, Ctrl* ctl) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int H = md.H, dh = md.dh, d = md.d;
-  const int len = pos0 + M;
+  const int len = origin + nslots;
   const int nsplit = eff_nsplit(md, len);
   const int Lc = (len + nsplit - 1) / nsplit;
   const int rowb = dh * 2, cpr = rowb >> 4;
@@ -1052,8 +1087,11 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int pos0, int cta,
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int r = gp * 16 + gq + (j >> 1) * 8, q = 2 * tq + (j & 1);
-          const bool vis = r < n && (c0 + r) <= pos0 + q;
-          if (q < M) S[q * sst + r] = vis ? dsc[j] * md.scale : -INFINITY;
+          if (q < M) {
+            const int rel = c0 + r - origin;
+            const bool vis = r < n && (rel < 0 || ((ctl->sees[q] >> rel) & 1u));
+            S[q * sst + r] = vis ? dsc[j] * md.scale : -INFINITY;
+          }
         }
       }
       named_sync(1, CONSUMER_THREADS);

@@ -136,30 +136,26 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
       const XSrc src{a.gx, (size_t)a.gK, nullptr};
       consume_gemm<M, WT>(g, e, src, nullptr, 0.f, nullptr, nullptr, cta, G, ring, ctl, X, xphase, red, pre_s, zero_addr, stages, err);
     } else {
-      // positions and token ids of the M rows
-      int pos0, pending = 0;
+      // origin = sequence position of the pending token; the launch's row table gives each row its
+      // token, cache row, rotary position and the block rows it attends
+      int origin, pending = 0, nslots;
       int ids[M];
-      if (a.mode == MODE_VERIFY) {
-        pos0 = a.pos_base + st->n_text;
-        pending = st->pending;
-        ids[0] = pending;
+      const bool from_ids = (a.mode != MODE_ROWS) || a.rows == nullptr;
+      if (a.mode == MODE_ROWS) {       // a chunk of prompt rows at absolute positions: a chain from rows_pos0
+        origin = a.rows_pos0;
+        nslots = M;
 #pragma unroll
-        for (int m = 1; m < M; ++m) ids[m] = st->d_ids[m - 1];
-      } else if (a.mode == MODE_DRAFT) {
-        // rows [token before, token to extend]: tokens are prev, pending, x_1, x_2, ...
-        pos0 = a.pos_base + st->n_text - 1 + a.j;
+        for (int m = 0; m < M; ++m) ids[m] = a.row_ids ? a.row_ids[m] : 0;
+      } else {
+        origin = a.pos_base + st->n_text;
+        nslots = a.n_slots;
         pending = st->pending;
 #pragma unroll
         for (int m = 0; m < M; ++m) {
-          const int t = a.j - (M - 1) + m;   // index into [pending, x_1, ...]; -1 = prev
-          ids[m] = t < 0 ? st->prev : (t == 0 ? st->pending : st->d_ids[t - 1]);
+          const int sr = a.geo.src[m];
+          ids[m] = sr == -2 ? st->prev : (sr == -1 ? pending : st->d_ids[sr]);
         }
-      } else {
-        pos0 = a.rows_pos0;
-#pragma unroll
-        for (int m = 0; m < M; ++m) ids[m] = a.row_ids ? a.row_ids[m] : 0;
       }
-      const bool from_ids = (a.mode != MODE_ROWS) || a.rows == nullptr;
 #pragma unroll
       for (int m = 0; m < M; ++m)
         if (from_ids && (ids[m] < 0 || ids[m] >= md.V)) {
@@ -170,7 +166,13 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
       // the ids live in shared memory from here on (embedding rows, sampling rule)
       if (tid == 0) {
 #pragma unroll
-        for (int m = 0; m < M; ++m) ctl->tok[m] = ids[m];
+        for (int m = 0; m < M; ++m) {
+          ctl->tok[m] = ids[m];
+          const bool chain = a.mode == MODE_ROWS;
+          ctl->rowslot[m] = origin + (chain ? m : (int)a.geo.slot[m]);
+          ctl->rowpos[m] = origin + (chain ? m : (int)a.geo.depth[m]);
+          ctl->sees[m] = chain ? ((2u << m) - 1u) : (unsigned)a.geo.sees[m];
+        }
       }
       named_sync(1, CONSUMER_THREADS);
       // bf16 models: every residual epilogue leaves x * (gain of the next RMSNorm) in md.xg and
@@ -200,7 +202,8 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
         } else {
           const LayerDev& ly = layers[l];
           if (which == 0) {          // QKV + RoPE + KV append
-            e.qbuf = md.qbuf; e.d = d; e.dh = md.dh; e.pos0 = pos0; e.cs = md.rope_cos; e.sn = md.rope_sin;
+            e.qbuf = md.qbuf; e.d = d; e.dh = md.dh; e.rowslot = ctl->rowslot; e.rowpos = ctl->rowpos;
+            e.cs = md.rope_cos; e.sn = md.rope_sin;
             e.kc = static_cast<WT*>(md.kcache) + (size_t)l * md.max_seq * d;
             e.vc = static_cast<WT*>(md.vcache) + (size_t)l * md.max_seq * d;
             norm_w = ly.attn_norm;
@@ -227,19 +230,16 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
                             zero_addr, stages, err);
         stamp(3); sync_grid(); stamp(4);
         if (!head && which == 0) {
-          if constexpr (sizeof(WT) == 2) attn_phase_mma<M>(md, l, pos0, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
-          else attn_phase<M, WT>(md, l, pos0, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
+          if constexpr (sizeof(WT) == 2) attn_phase_mma<M>(md, l, origin, nslots, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
+          else attn_phase<M, WT>(md, l, origin, nslots, cta, G, reinterpret_cast<char*>(X), x_bytes(M), ctl);
           stamp(3); sync_grid(); stamp(4);
         }
       }
       if (want_head) {
         // row statistics over vocabulary slices, then CTA 0 applies the sampling rule
-        int r0, nrows;
-        if (a.mode == MODE_VERIFY) { r0 = 0; nrows = a.gamma + 1; }
-        else { r0 = M - 1; nrows = 1; }
-        stats_phase<M>(a.logits, md.V, r0, nrows, a.temperature, cta, G, md.stat_part, ctl);
+        stats_phase<M>(a.logits, md.V, a.stat_r0, a.stat_n, a.temperature, cta, G, md.stat_part, ctl);
         stamp(3); sync_grid(); stamp(4);
-        if (cta == 0 && a.greedy) {
+        if (cta == 0 && a.greedy && !a.tree) {
           if (a.mode == MODE_VERIFY) verify_greedy<M>(a, md, st, ctl, G, 0, a.gamma, ctl->tok + 1, pending);
           else if (a.mode == MODE_DRAFT) draft_greedy<M>(a, md, st, ctl, G);
           else verify_greedy<M>(a, md, st, ctl, G, M - 1, 0, ctl->tok, 0);
@@ -407,13 +407,11 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) sample_pick_kernel(const __gri
 //                       stored as q_j; verify step -> the rule on (prow, q_in), commit; prefill ->
 //                       the first token drawn from the truncated row.
 
-__device__ __forceinline__ int rows_needed(const StepArgs& a) { return a.mode == MODE_VERIFY ? a.gamma + 1 : 1; }
-
 __global__ void __launch_bounds__(SAMPLE_THREADS) prob_rows_kernel(const __grid_constant__ StepArgs a, float* prow) {
   __shared__ SampleShared sh;
   const int cta = blockIdx.x, G = gridDim.x, V = a.md.V;
-  const int nrows = rows_needed(a), r0 = a.mode == MODE_VERIFY ? 0 : a.sample_r0;
-  // the statistics sit at indices 0..nrows-1 (a draft step / a prefill chunk left one row's at index 0)
+  const int nrows = a.stat_n, r0 = a.stat_r0;
+  // the statistics of row r0 + r sit at index r
   merge_stats(a.md.stat_part, a.fwd_grid, nrows, nullptr, sh.rowmax, sh.rowsum, sh.arg);
   const int VS = (V + G - 1) / G;
   const int k0 = cta * VS, k1 = min(V, k0 + VS);

