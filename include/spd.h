@@ -26,7 +26,8 @@
  *     copy of the weights, so the caller may free them afterwards.
  *   - Matrices are row-major [out, in], in the model's dtype (0 = fp32, 1 = bfloat16);
  *     norm gains are fp32 [d_model]; there are no biases.
- *   - One sequence per context (batch 1).
+ *   - One sequence per context; spd_fork gives further sequences on the same weights and
+ *     spd_batch_* runs several of them through one pass over the weights.
  *   - Call order: create -> prefill -> (draft -> verify)* ; anything else is SPD_ESTATE.
  */
 #ifndef SPD_H_
@@ -251,6 +252,49 @@ spd_status spd_verify_tree(spd_ctx* ctx, int n_nodes, const int32_t* parent, con
  * gamma == 0 runs the target alone (the auto-regressive baseline). */
 spd_status spd_generate(spd_ctx* ctx, int n_new, int gamma, const float* uniforms,
                         int32_t* out_ids, spd_stats* stats);
+
+/* ---- several sequences, one pass over the weights ----
+ * The method is stated for one sequence (Sec. 2.1), and its cost argument is that a target call
+ * is bound by streaming the parameters (Sec. 1; Sec. 4 "Metrics": cost proportional to parameter
+ * count).  When B sequences are decoded together the parameters should therefore be streamed
+ * once for all of them.  A batch groups B contexts that share their weights (a context and its
+ * spd_fork's, all on one stream).  A batched step runs the rows of all sequences -- B x (gamma+1)
+ * for the verify step, B x 2 for a draft step, at most 128 -- through every projection as ONE
+ * dense tensor-core GEMM, while rotary embedding, cache append, attention over each sequence's
+ * own cache, the rejection rule and the commit stay per sequence: every sequence keeps its own
+ * length, accepts its own number of tokens and can be rolled back on its own (spd_rollback on its
+ * context).  Prefill stays per sequence (prompts have different lengths).  bf16 models only.
+ * Batched and single-sequence calls may be mixed freely between blocks. */
+typedef struct spd_batch spd_batch;
+
+/* seqs: HOST array of B distinct contexts, all forks of one context (or that context itself);
+ * B x (gamma_max + 1) <= 128.  The contexts must outlive the batch.  Errors are reported on
+ * seqs[0] (spd_last_error(seqs[0])). */
+spd_status spd_batch_create(spd_ctx* const* seqs, int B, spd_batch** out);
+void spd_batch_destroy(spd_batch* batch);
+
+/* gamma draft steps for every sequence (Sec. 2.1), each step one pass over the draft's weights.
+ *   uniforms   fp32 [B, gamma], host or device; may be NULL when greedy
+ *   draft_ids  int32 [B, gamma], out, host or device, may be NULL
+ * The draft distributions are kept inside the batch for spd_batch_verify. */
+spd_status spd_batch_draft(spd_batch* batch, int gamma, const float* uniforms, int32_t* draft_ids);
+
+/* One target call on the B x (gamma+1) rows [pending_b, x_b1..x_b,gamma], then per sequence the
+ * rejection rule (Sec. 2.1, Sec. 3), the commit and the roll-back of its caches to its accepted
+ * length.  gamma must be that of the preceding spd_batch_draft; gamma == 0 is a plain
+ * auto-regressive step of the target for every sequence.
+ *   uniforms    fp32 [B, gamma+1], host or device; may be NULL when greedy
+ *   n_accepted, next_token  int32 [B], out, host or device, may be NULL */
+spd_status spd_batch_verify(spd_batch* batch, int gamma, const float* uniforms, int32_t* n_accepted,
+                            int32_t* next_token);
+
+/* Logits of the last batched call, fp32 [rows, vocab] (row b*(gamma+1)+m after a verify step,
+ * b*2+m after a draft step), host or device.  Test support. */
+spd_status spd_batch_get_logits(spd_batch* batch, float* logits, int rows);
+
+/* Bytes one batched verify step must move: the target's weights once + every sequence's K/V rows
+ * read and written (the figure its roofline is computed from). */
+spd_status spd_batch_verify_bytes(spd_batch* batch, int gamma, double* bytes);
 
 /* ---- test and benchmark support ---- */
 

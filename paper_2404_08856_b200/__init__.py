@@ -22,7 +22,8 @@ EXPORTS = ["spd_create", "spd_destroy", "spd_fork", "spd_last_error", "spd_prefi
            "spd_generate", "spd_get_logits", "spd_get_draft_logits", "spd_rollback", "spd_get_state",
            "spd_reject_sample", "spd_skinny_gemm", "spd_verify_bytes", "spd_trace",
            "spd_skinny_gemm_noalloc", "spd_image_adapter", "spd_truncate_probs", "spd_skinny_gemm_status",
-           "spd_wait_selftest", "spd_draft_tree", "spd_verify_tree"]
+           "spd_wait_selftest", "spd_draft_tree", "spd_verify_tree", "spd_batch_create", "spd_batch_destroy",
+           "spd_batch_draft", "spd_batch_verify", "spd_batch_get_logits", "spd_batch_verify_bytes"]
 
 
 class SpdError(RuntimeError):
@@ -74,8 +75,10 @@ def lib() -> C.CDLL:
         _lib.spd_last_error.argtypes = [C.c_void_p]
         _lib.spd_destroy.restype = None
         _lib.spd_destroy.argtypes = [C.c_void_p]
+        _lib.spd_batch_destroy.restype = None
+        _lib.spd_batch_destroy.argtypes = [C.c_void_p]
         for name in EXPORTS:
-            if name not in ("spd_last_error", "spd_destroy"):
+            if name not in ("spd_last_error", "spd_destroy", "spd_batch_destroy"):
                 getattr(_lib, name).restype = C.c_int
     return _lib
 
@@ -263,6 +266,62 @@ class Spd:
     def verify_bytes(self, gamma: int) -> float:
         b = C.c_double(0)
         self._check(lib().spd_verify_bytes(self._ctx, gamma, C.byref(b)))
+        return b.value
+
+
+class SpdBatch:
+    """Several sequences (contexts that share their weights) decoded with one pass over the weights
+    per step; see spd_batch_create."""
+
+    def __init__(self, seqs):
+        self.seqs = list(seqs)
+        self.B = len(self.seqs)
+        arr = (C.c_void_p * self.B)(*[s._ctx.value for s in self.seqs])
+        self._bt = C.c_void_p(0)
+        st = lib().spd_batch_create(arr, self.B, C.byref(self._bt))
+        if st != SPD_OK:
+            raise SpdError(st, lib().spd_last_error(self.seqs[0]._ctx).decode())
+
+    def _check(self, st: int):
+        if st != SPD_OK:
+            raise SpdError(st, lib().spd_last_error(self.seqs[0]._ctx).decode())
+
+    def close(self):
+        if getattr(self, "_bt", None) and self._bt.value:
+            lib().spd_batch_destroy(self._bt)
+            self._bt = C.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def draft(self, gamma: int, uniforms=None, read_ids: bool = True):
+        """uniforms [B, gamma] (numpy or device tensor).  Returns ids [B, gamma] (or None)."""
+        u = uniforms if (uniforms is None or hasattr(uniforms, "data_ptr")) \
+            else np.ascontiguousarray(uniforms, dtype=np.float32)
+        ids = np.zeros((self.B, gamma), dtype=np.int32) if read_ids else None
+        self._check(lib().spd_batch_draft(self._bt, gamma, _ptr(u), _ptr(ids)))
+        return ids
+
+    def verify(self, gamma: int, uniforms=None, read: bool = True):
+        """uniforms [B, gamma+1].  Returns (n_accepted [B], next_token [B]) (or None)."""
+        u = uniforms if (uniforms is None or hasattr(uniforms, "data_ptr")) \
+            else np.ascontiguousarray(uniforms, dtype=np.float32)
+        a = np.zeros(self.B, dtype=np.int32) if read else None
+        n = np.zeros(self.B, dtype=np.int32) if read else None
+        self._check(lib().spd_batch_verify(self._bt, gamma, _ptr(u), _ptr(a), _ptr(n)))
+        return (a, n) if read else None
+
+    def get_logits(self, rows: int) -> np.ndarray:
+        out = np.zeros((rows, self.seqs[0].vocab), dtype=np.float32)
+        self._check(lib().spd_batch_get_logits(self._bt, _ptr(out), rows))
+        return out
+
+    def verify_bytes(self, gamma: int) -> float:
+        b = C.c_double(0)
+        self._check(lib().spd_batch_verify_bytes(self._bt, gamma, C.byref(b)))
         return b.value
 
 

@@ -13,6 +13,7 @@
 #include "spd_prefill.cuh"
 #include "spd_warp.cuh"
 #include "spd_tree.cuh"
+#include "spd_batch.cuh"
 
 using namespace spd;
 
@@ -33,6 +34,7 @@ struct ModelHost {
   struct RowMajor { __nv_bfloat16 *wqkv, *wo, *wgu, *wd; const float *attn_norm, *ffn_norm; };
   std::vector<RowMajor> rm;
   __nv_bfloat16* adapter_rm = nullptr;
+  __nv_bfloat16* lm_rm = nullptr;   // LM head [V][d], row-major (batched path)
   bool rows_given = false;  // draft only: the image rows arrive already in the draft's space
   int grid = 0;             // CTAs of this model's forward launches (its weights are packed for that count)
   int cluster = 0;          // > 0: those CTAs form one thread-block cluster of this size
@@ -281,6 +283,11 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
     if ((s = put_rows(ctx, rm, c.tied_embeddings ? w->tok_embed : w->lm_head, staging, V, d, esz, 1, 0, 0))) return s;
     if ((s = pack_tiles(ctx, lm, rm, V, d, esz, mh.grid, ctx->stream))) return s;
     md.lm_head = lm;
+    if (esz == 2) {   // natural-order copy for the dense (batched) path
+      if ((s = dalloc(ctx, &mh.lm_rm, (size_t)V * d))) return s;
+      CU(cudaMemcpyAsync(mh.lm_rm, rm, (size_t)V * d * 2, cudaMemcpyDeviceToDevice, ctx->stream));
+      CU(cudaStreamSynchronize(ctx->stream));
+    }
   }
   float* fn = nullptr;
   if ((s = dalloc(ctx, &fn, (size_t)d))) return s;
@@ -1346,6 +1353,288 @@ spd_status spd_verify_tree(spd_ctx* ctx, int n_nodes, const int32_t* parent, con
   if ((s = copy_out(ctx, next_token, &ctx->st->next, sizeof(int32_t), &need_sync))) return s;
   if ((s = copy_out(ctx, path, ctx->st->path, sh.depth_max * sizeof(int32_t), &need_sync))) return s;
   if (need_sync) return sync_state(ctx);
+  return SPD_OK;
+}
+
+// ---- several sequences in one pass over the weights
+
+}  // extern "C"
+
+struct spd_batch {
+  std::vector<spd_ctx*> seqs;
+  spd_ctx* lead = nullptr;      // stream, error word and GEMM scratch of the batch
+  int B = 0;
+  BatchSeq* seqs_dev = nullptr;
+  ModelDev *mds_t = nullptr, *mds_d = nullptr;
+  int *rowslot = nullptr, *origins = nullptr, *out_acc = nullptr, *out_next = nullptr;
+  float *X = nullptr, *logits = nullptr, *probs = nullptr, *q_all = nullptr, *u_draft = nullptr, *u_verify = nullptr;
+  int drafted_gamma = -1;
+  int last_rows = 0;
+  std::vector<void*> allocs;
+};
+
+namespace {
+
+template <typename T>
+spd_status balloc(spd_batch* bt, T** p, size_t n) {
+  spd_ctx* ctx = bt->lead;
+  void* q = nullptr;
+  CU(cudaMalloc(&q, n * sizeof(T) + 256));
+  CU(cudaMemsetAsync(q, 0, n * sizeof(T) + 256, ctx->stream));
+  bt->allocs.push_back(q);
+  *p = static_cast<T*>(q);
+  return SPD_OK;
+}
+
+constexpr int BATCH_ATTN_SCRATCH = 200 * 1024;
+
+template <int M>
+spd_status launch_batch_attn(spd_ctx* ctx, const ModelDev* mds, const int* origins, int B, int layer, int chain0) {
+  static bool attr[MAX_DEV];
+  const size_t smem = CTRL_BYTES + BATCH_ATTN_SCRATCH;
+  if (!attr[ctx->device]) {
+    CU(cudaFuncSetAttribute((const void*)batch_attn_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attr[ctx->device] = true;
+  }
+  batch_attn_kernel<M><<<ctx->n_sm, CONSUMER_THREADS, smem, ctx->stream>>>(mds, origins, B, layer, chain0,
+                                                                          BATCH_ATTN_SCRATCH);
+  CU(cudaGetLastError());
+  return SPD_OK;
+}
+
+spd_status batch_attn(spd_ctx* ctx, int M, const ModelDev* mds, const int* origins, int B, int layer, int chain0) {
+  switch (M) {
+    case 1: return launch_batch_attn<1>(ctx, mds, origins, B, layer, chain0);
+    case 2: return launch_batch_attn<2>(ctx, mds, origins, B, layer, chain0);
+    case 3: return launch_batch_attn<3>(ctx, mds, origins, B, layer, chain0);
+    case 4: return launch_batch_attn<4>(ctx, mds, origins, B, layer, chain0);
+    case 5: return launch_batch_attn<5>(ctx, mds, origins, B, layer, chain0);
+    case 6: return launch_batch_attn<6>(ctx, mds, origins, B, layer, chain0);
+    case 7: return launch_batch_attn<7>(ctx, mds, origins, B, layer, chain0);
+    default: return launch_batch_attn<8>(ctx, mds, origins, B, layer, chain0);
+  }
+}
+
+// Dense forward of the B x M rows of a batched step through every layer and the LM head of one
+// model: logits land in bt->logits [B*M][V]; each sequence's K/V rows are appended to its own cache.
+spd_status batch_forward(spd_batch* bt, bool draft, int M, int j) {
+  spd_ctx* ctx = bt->lead;
+  ModelHost& mh = draft ? ctx->draft : ctx->target;
+  const int B = bt->B, R = B * M;
+  const int d = mh.cfg.d_model, f = mh.cfg.d_ffn, H = mh.cfg.n_heads, dh = d / H, L = mh.cfg.n_layers, V = mh.cfg.vocab;
+  spd_status s;
+  if ((s = prefill_scratch(ctx, R))) return s;
+  auto& pf = ctx->pf;
+  cudaStream_t cs = ctx->stream;
+  float* X = bt->X;
+  const ModelDev* mds = draft ? bt->mds_d : bt->mds_t;
+  batch_embed_kernel<<<R, 128, 0, cs>>>(bt->seqs_dev, B, M, draft ? 1 : 0, j, mh.md.embed, d, V, X, bt->rowslot,
+                                        bt->origins, &ctx->st->err);
+  const Operand h_hi{pf.h_hi, d, R, 1, (size_t)d * 2, (size_t)R * d * 2}, h_lo{pf.h_lo, d, R, 1, (size_t)d * 2, (size_t)R * d * 2};
+  for (int l = 0; l < L; ++l) {
+    const ModelHost::RowMajor& w = mh.rm[l];
+    TcArgs a{};
+    rms_split_kernel<<<R, 256, 0, cs>>>(X, w.attn_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
+    a = TcArgs{}; a.M = R; a.N = 3 * d; a.K = d; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = pf.wide; a.ldo = 3 * d;
+    if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wqkv, d, 3 * d, 1, (size_t)d * 2, (size_t)3 * d * d * 2}, a))) return s;
+    batch_rope_append_kernel<<<296, 256, 0, cs>>>(pf.wide, R, M, d, dh, bt->rowslot, mh.md.rope_cos, mh.md.rope_sin, mds, l);
+    if ((s = batch_attn(ctx, M, mds, bt->origins, B, l, draft ? j - 1 : 0))) return s;
+    batch_gather_split_kernel<<<296, 256, 0, cs>>>(mds, R, M, d, pf.h_hi, pf.h_lo);
+    a = TcArgs{}; a.M = R; a.N = d; a.K = d; a.mode = TC_OUT_F32_ADD; a.alpha = 1.f; a.out_f32 = X; a.ldo = d;
+    if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wo, d, d, 1, (size_t)d * 2, (size_t)d * d * 2}, a))) return s;
+    rms_split_kernel<<<R, 256, 0, cs>>>(X, w.ffn_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
+    a = TcArgs{}; a.M = R; a.N = 2 * f; a.K = d; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = pf.wide; a.ldo = 2 * f;
+    if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wgu, d, 2 * f, 1, (size_t)d * 2, (size_t)2 * f * d * 2}, a))) return s;
+    swiglu_split_kernel<<<296, 256, 0, cs>>>(pf.wide, R, f, pf.h_hi, pf.h_lo);
+    a = TcArgs{}; a.M = R; a.N = d; a.K = f; a.mode = TC_OUT_F32_ADD; a.alpha = 1.f; a.out_f32 = X; a.ldo = d;
+    if ((s = tc_gemm(ctx, {pf.h_hi, f, R, 1, (size_t)f * 2, (size_t)R * f * 2}, {pf.h_lo, f, R, 1, (size_t)f * 2, (size_t)R * f * 2},
+                     {w.wd, f, d, 1, (size_t)f * 2, (size_t)d * f * 2}, a))) return s;
+  }
+  rms_split_kernel<<<R, 256, 0, cs>>>(X, mh.md.final_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
+  TcArgs a{}; a.M = R; a.N = V; a.K = d; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = bt->logits; a.ldo = V;
+  if ((s = tc_gemm(ctx, h_hi, h_lo, {mh.lm_rm, d, V, 1, (size_t)d * 2, (size_t)V * d * 2}, a))) return s;
+  CU(cudaGetLastError());
+  bt->last_rows = R;
+  return SPD_OK;
+}
+
+// softmax rows of bt->logits -> bt->probs, truncated when top-k / top-p is on
+spd_status batch_probs(spd_batch* bt, int R) {
+  spd_ctx* ctx = bt->lead;
+  const int V = ctx->cfg.target.vocab;
+  batch_softmax_kernel<<<R, SAMPLE_THREADS, 0, ctx->stream>>>(bt->logits, V, ctx->cfg.temperature, bt->probs);
+  if (ctx->truncate)
+    truncate_rows_kernel<<<R, WARP_THREADS, (size_t)V * sizeof(float), ctx->stream>>>(
+        bt->probs, bt->probs, V, ctx->cfg.top_k, ctx->cfg.top_p > 0.f ? ctx->cfg.top_p : 1.0f);
+  CU(cudaGetLastError());
+  return SPD_OK;
+}
+
+spd_status batch_room(spd_batch* bt, int rows, bool draft) {
+  for (spd_ctx* c : bt->seqs) {
+    const int base = draft ? (c->m_image > c->draft.pos_base ? c->m_image : c->draft.pos_base) : c->m_image;
+    if (base + c->len_ub + rows > c->cfg.max_seq) {
+      spd_status s = sync_state(c);
+      if (s) return s;
+      if (base + c->len_ub + rows > c->cfg.max_seq) return fail(bt->lead, SPD_EOVERFLOW, "KV cache of a sequence is full");
+    }
+  }
+  return SPD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+void spd_batch_destroy(spd_batch* bt) {
+  if (!bt) return;
+  if (bt->lead) cudaStreamSynchronize(bt->lead->stream);
+  for (void* p : bt->allocs) cudaFree(p);
+  delete bt;
+}
+
+spd_status spd_batch_create(spd_ctx* const* seqs, int B, spd_batch** out) {
+  if (out) *out = nullptr;
+  if (!seqs || !out || B < 1) return SPD_EINVAL;
+  spd_ctx* ctx = seqs[0];
+  if (!ctx) return SPD_EINVAL;
+  const int gm = ctx->cfg.gamma_max > 0 ? ctx->cfg.gamma_max : 1;
+  if (B * (gm + 1) > BATCH_ROWS_MAX || B * 2 > BATCH_ROWS_MAX)
+    return fail(ctx, SPD_EINVAL, "batch x (gamma_max + 1) rows must fit one 128-row tile");
+  if (ctx->cfg.target.dtype != 1 || ctx->cfg.draft.dtype != 1)
+    return fail(ctx, SPD_EINVAL, "the batched path needs bf16 models (tensor-core GEMMs)");
+  const spd_ctx* origin0 = ctx->origin ? ctx->origin : ctx;
+  for (int b = 0; b < B; ++b) {
+    spd_ctx* c = seqs[b];
+    if (!c) return fail(ctx, SPD_EINVAL, "null sequence in the batch");
+    if ((c->origin ? c->origin : c) != origin0 || c->stream != ctx->stream)
+      return fail(ctx, SPD_EINVAL, "the sequences of a batch must be forks of one context (shared weights and stream)");
+    for (int k = 0; k < b; ++k)
+      if (seqs[k] == c) return fail(ctx, SPD_EINVAL, "a sequence appears twice in the batch");
+  }
+  spd_batch* bt = new (std::nothrow) spd_batch();
+  if (!bt) return SPD_ENOMEM;
+  bt->lead = ctx; bt->B = B;
+  bt->seqs.assign(seqs, seqs + B);
+  const int V = ctx->cfg.target.vocab;
+  const size_t dmax = ctx->cfg.target.d_model > ctx->cfg.draft.d_model ? ctx->cfg.target.d_model : ctx->cfg.draft.d_model;
+  spd_status s = SPD_OK;
+  if (!s) s = balloc(bt, &bt->seqs_dev, (size_t)B);
+  if (!s) s = balloc(bt, &bt->mds_t, (size_t)B);
+  if (!s) s = balloc(bt, &bt->mds_d, (size_t)B);
+  if (!s) s = balloc(bt, &bt->rowslot, (size_t)BATCH_ROWS_MAX);
+  if (!s) s = balloc(bt, &bt->origins, (size_t)B);
+  if (!s) s = balloc(bt, &bt->out_acc, (size_t)B);
+  if (!s) s = balloc(bt, &bt->out_next, (size_t)B);
+  if (!s) s = balloc(bt, &bt->X, (size_t)BATCH_ROWS_MAX * dmax);
+  if (!s) s = balloc(bt, &bt->logits, (size_t)BATCH_ROWS_MAX * V);
+  if (!s) s = balloc(bt, &bt->probs, (size_t)BATCH_ROWS_MAX * V);
+  if (!s) s = balloc(bt, &bt->q_all, (size_t)B * gm * V);
+  if (!s) s = balloc(bt, &bt->u_draft, (size_t)B * MAX_M);
+  if (!s) s = balloc(bt, &bt->u_verify, (size_t)B * MAX_M);
+  if (!s && ctx->truncate &&
+      cudaFuncSetAttribute((const void*)truncate_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)((size_t)V * sizeof(float))) != cudaSuccess)
+    s = fail(ctx, SPD_ECUDA, "cannot size the truncation kernel's shared memory");
+  if (s) { spd_batch_destroy(bt); return s; }
+  *out = bt;
+  return SPD_OK;
+}
+
+// (re)reads each sequence's descriptors: a prefill changes the rows in front of the text
+static spd_status batch_refresh(spd_batch* bt) {
+  spd_ctx* ctx = bt->lead;
+  std::vector<BatchSeq> hs(bt->B);
+  std::vector<ModelDev> ht(bt->B), hd(bt->B);
+  for (int b = 0; b < bt->B; ++b) {
+    spd_ctx* c = bt->seqs[b];
+    if (!c->prefilled) return fail(ctx, SPD_ESTATE, "a sequence of the batch has not been prefilled");
+    hs[b] = BatchSeq{c->st, c->target.pos_base, c->draft.pos_base};
+    ht[b] = c->target.md;
+    hd[b] = c->draft.md;
+  }
+  CU(cudaMemcpyAsync(bt->seqs_dev, hs.data(), hs.size() * sizeof(BatchSeq), cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaMemcpyAsync(bt->mds_t, ht.data(), ht.size() * sizeof(ModelDev), cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaMemcpyAsync(bt->mds_d, hd.data(), hd.size() * sizeof(ModelDev), cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));   // the host vectors go out of scope
+  return SPD_OK;
+}
+
+spd_status spd_batch_draft(spd_batch* bt, int gamma, const float* uniforms, int32_t* draft_ids) {
+  if (!bt) return SPD_EINVAL;
+  spd_ctx* ctx = bt->lead;
+  if (gamma < 1 || gamma > ctx->cfg.gamma_max) return fail(ctx, SPD_EINVAL, "gamma out of range");
+  if (!ctx->cfg.greedy && !uniforms) return fail(ctx, SPD_EINVAL, "uniforms required when sampling");
+  spd_status s;
+  if ((s = batch_refresh(bt))) return s;
+  if ((s = batch_room(bt, gamma + 1, true))) return s;
+  const int B = bt->B, V = ctx->cfg.target.vocab;
+  if (uniforms) CU(cudaMemcpyAsync(bt->u_draft, uniforms, (size_t)B * gamma * sizeof(float), cudaMemcpyDefault, ctx->stream));
+  for (int j = 0; j < gamma; ++j) {
+    if ((s = batch_forward(bt, true, 2, j))) return s;
+    if (!ctx->cfg.greedy && (s = batch_probs(bt, 2 * B))) return s;
+    batch_draft_sample_kernel<<<B, SAMPLE_THREADS, 0, ctx->stream>>>(bt->seqs_dev, ctx->cfg.greedy ? bt->logits : bt->probs,
+                                                                      V, gamma, j, ctx->cfg.greedy, bt->u_draft, bt->q_all);
+    CU(cudaGetLastError());
+  }
+  bt->drafted_gamma = gamma;
+  for (spd_ctx* c : bt->seqs) { c->drafted_gamma = -1; c->tree_drafted = false; }
+  if (draft_ids) {
+    const bool host = !is_device_ptr(draft_ids);
+    for (int b = 0; b < B; ++b)
+      CU(cudaMemcpyAsync(draft_ids + (size_t)b * gamma, bt->seqs[b]->st->d_ids, gamma * sizeof(int32_t), cudaMemcpyDefault, ctx->stream));
+    if (host) CU(cudaStreamSynchronize(ctx->stream));
+  }
+  return SPD_OK;
+}
+
+spd_status spd_batch_verify(spd_batch* bt, int gamma, const float* uniforms, int32_t* n_accepted, int32_t* next_token) {
+  if (!bt) return SPD_EINVAL;
+  spd_ctx* ctx = bt->lead;
+  if (gamma < 0 || gamma > ctx->cfg.gamma_max) return fail(ctx, SPD_EINVAL, "gamma out of range");
+  if (gamma > 0 && bt->drafted_gamma != gamma) return fail(ctx, SPD_ESTATE, "spd_batch_verify needs an spd_batch_draft with the same gamma");
+  if (!ctx->cfg.greedy && !uniforms) return fail(ctx, SPD_EINVAL, "uniforms required when sampling");
+  spd_status s;
+  if ((s = batch_refresh(bt))) return s;
+  if ((s = batch_room(bt, gamma + 1, false))) return s;
+  const int B = bt->B, V = ctx->cfg.target.vocab, M = gamma + 1;
+  if (uniforms) CU(cudaMemcpyAsync(bt->u_verify, uniforms, (size_t)B * M * sizeof(float), cudaMemcpyDefault, ctx->stream));
+  if ((s = batch_forward(bt, false, M, 0))) return s;
+  if (!ctx->cfg.greedy && (s = batch_probs(bt, B * M))) return s;
+  batch_verify_kernel<<<B, SAMPLE_THREADS, 0, ctx->stream>>>(bt->seqs_dev, ctx->cfg.greedy ? bt->logits : bt->probs, bt->q_all,
+                                                              ctx->cfg.greedy ? nullptr : bt->u_verify, gamma, V,
+                                                              ctx->cfg.greedy, bt->out_acc, bt->out_next);
+  CU(cudaGetLastError());
+  bt->drafted_gamma = -1;
+  for (spd_ctx* c : bt->seqs) { c->len_ub += M; c->drafted_gamma = -1; c->last_verify_rows = 0; }
+  bool need_sync = false;
+  if ((s = copy_out(ctx, n_accepted, bt->out_acc, B * sizeof(int32_t), &need_sync))) return s;
+  if ((s = copy_out(ctx, next_token, bt->out_next, B * sizeof(int32_t), &need_sync))) return s;
+  if (need_sync) return sync_state(ctx);   // also reports a device-side error (bad id, a wait that ran out)
+  return SPD_OK;
+}
+
+spd_status spd_batch_get_logits(spd_batch* bt, float* logits, int rows) {
+  if (!bt || !logits) return SPD_EINVAL;
+  spd_ctx* ctx = bt->lead;
+  if (rows < 1 || rows > bt->last_rows) return fail(ctx, SPD_EINVAL, "rows exceed the last batched call");
+  CU(cudaMemcpyAsync(logits, bt->logits, (size_t)rows * ctx->cfg.target.vocab * sizeof(float), cudaMemcpyDefault, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  return SPD_OK;
+}
+
+spd_status spd_batch_verify_bytes(spd_batch* bt, int gamma, double* bytes) {
+  if (!bt || !bytes) return SPD_EINVAL;
+  spd_ctx* ctx = bt->lead;
+  double kv = 0.0;
+  for (spd_ctx* c : bt->seqs) {
+    spd_status s = sync_state(c);
+    if (s) return s;
+    const double C = c->m_image + c->st_host->n_text;
+    const double kv_row = 2.0 * c->target.cfg.n_layers * c->target.cfg.d_model * c->target.esz;
+    kv += kv_row * (C + gamma + 1) + kv_row * (gamma + 1);
+  }
+  *bytes = (double)ctx->target.wbytes + kv;
   return SPD_OK;
 }
 
