@@ -557,10 +557,11 @@ def run_gpu(args, rank, world):
 
 
 def run_batched(args):
-    """The batched KV-heavy workload on forked sequences: B sequences (default 16), each with
-    576 image rows + 1024 prompt ids in its bf16 KV cache, gamma = 5, temperature 1, one block per
-    sequence per step.  Sequences share the weights (spd_fork) but are NOT batched into one weight
-    pass: every draft and verify call streams the weights once.  Prints one JSON line; not the
+    """The batched KV-heavy workload: B sequences (default 16), each with 576 image rows + 1024
+    prompt ids in its bf16 KV cache, gamma = 5, temperature 1, one speculative block per sequence
+    per step.  `--batched-mode pass` (default) runs the rows of all sequences through ONE pass over
+    the weights per draft / verify step (spd_batch_*); `forked` drives the sequences one after the
+    other (each call streams the weights again) for comparison.  Prints one JSON line; not the
     default benchmark."""
     import torch
     import paper_2404_08856_b200 as spd
@@ -568,10 +569,11 @@ def run_batched(args):
     torch.cuda.set_device(0)
     build.build()
     B, n_prompt, steps = args.batch, 1024, args.steps
+    warm = max(args.warmup, 1)
     wl = synth.llava7b_workload(gamma=GAMMA, n_layers=args.layers, draft_layers=args.draft_layers, n_prompt=n_prompt)
     tw = synth.Weights(wl.target, wl.seeds["weights"], "target")
     dw = synth.Weights(wl.draft, wl.seeds["weights"], "draft")
-    max_seq = wl.n_image + n_prompt + (GAMMA + 1) * (steps + max(args.warmup, 1) + 2) + 64
+    max_seq = wl.n_image + n_prompt + (GAMMA + 1) * (steps + warm + 2) + 64
     seqs = [spd.Spd(wl.target, wl.draft, tw.stored, dw.stored, max_seq, GAMMA, 1.0, False)]
     del tw, dw
     seqs += [seqs[0].fork() for _ in range(B - 1)]
@@ -583,31 +585,57 @@ def run_batched(args):
         g.prefill(synth.image_embeds(w2), synth.prompt_ids(w2), u0=0.5)
     torch.cuda.synchronize()
     t_prefill = time.time() - t0
-    u = torch.from_numpy(synth.uniforms(3, "batched", (steps + args.warmup + 1, B, 2 * GAMMA + 1))).cuda()
+    u = torch.from_numpy(synth.uniforms(3, "batched", (steps + warm + 1, B, 2 * GAMMA + 1))).cuda()
+    one_pass = args.batched_mode == "pass"
+    bt = spd.SpdBatch(seqs) if one_pass else None
+    ev = []
 
     def step(i):
-        for k, g in enumerate(seqs):
-            g.draft_async(GAMMA, u[i, k, :GAMMA])
-            g.verify_async(GAMMA, u[i, k, GAMMA:])
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record(stream)
+        if one_pass:
+            bt.draft(GAMMA, u[i, :, :GAMMA].contiguous(), read_ids=False)
+            e[1].record(stream)
+            bt.verify(GAMMA, u[i, :, GAMMA:].contiguous(), read=False)
+        else:
+            for k, g in enumerate(seqs):
+                g.draft_async(GAMMA, u[i, k, :GAMMA])
+            e[1].record(stream)
+            for k, g in enumerate(seqs):
+                g.verify_async(GAMMA, u[i, k, GAMMA:])
+        e[2].record(stream)
+        ev.append(e)
 
-    for i in range(max(args.warmup, 1)):
+    for i in range(warm):
         step(i)
     torch.cuda.synchronize()
+    ev.clear()
     n0 = [g.get_state()[0] for g in seqs]
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(steps):
-        step(max(args.warmup, 1) + i)
-    e1.record(stream)
-    torch.cuda.synchronize()
+    bytes_step = bt.verify_bytes(GAMMA) if one_pass else None
+    with ClockSampler(0) as cs:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(steps):
+            step(warm + i)
+        e1.record(stream)
+        torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
     tokens = sum(g.get_state()[0] - a for g, a in zip(seqs, n0))
-    bytes_step = seqs[0].verify_bytes(GAMMA)
-    line = {"workload": "batched KV-heavy verify on forked sequences (weights shared, not batched)", "batch": B,
-            "kv_rows_per_sequence": wl.n_image + n_prompt, "gamma": GAMMA, "temperature": 1.0, "steps": steps,
-            "ms_per_step": ms / steps, "tokens_per_s": tokens / (ms * 1e-3), "tau": tokens / (steps * B),
-            "verify_bytes_per_sequence": bytes_step, "prefill_s_total": t_prefill,
-            "truncated_layers": args.layers}
+    draft_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+    verify_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
+    peak, peak_kind = measured_peak()
+    line = {"workload": "batched KV-heavy verify: " + ("one pass over the weights per step for all sequences"
+                                                      if one_pass else "forked sequences, one call each"),
+            "batch": B, "kv_rows_per_sequence": wl.n_image + n_prompt, "gamma": GAMMA, "temperature": 1.0,
+            "steps": steps, "ms_per_step": ms / steps, "draft_ms_per_step": draft_ms, "verify_ms_per_step": verify_ms,
+            "tokens_per_s": tokens / (ms * 1e-3), "tau": tokens / (steps * B), "prefill_s_total": t_prefill,
+            "truncated_layers": args.layers, "clocks": cs.summary()}
+    if one_pass:
+        achieved = bytes_step / (verify_ms * 1e-3) / 1e9
+        line["roofline"] = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                            "peak_kind": peak_kind, "bytes_per_launch": bytes_step, "ms_per_launch": verify_ms,
+                            "kernel": "batched verify step (weights once + every sequence's K/V)", "traffic": None}
+        bt.close()
     for g in seqs[1:]:
         g.close()
     seqs[0].close()
@@ -663,6 +691,8 @@ def main():
     ap.add_argument("--workload", default="bs1", choices=["bs1", "batched"],
                     help="batched: B forked sequences with 1600 cached rows each (informational line)")
     ap.add_argument("--batch", type=int, default=16)
+    ap.add_argument("--batched-mode", default="pass", choices=["pass", "forked"],
+                    help="batched workload: one weight pass per step for all sequences, or one call per sequence")
     ap.add_argument("--M", type=int, default=6)
     ap.add_argument("--N", type=int, default=32768)
     ap.add_argument("--K", type=int, default=4096)

@@ -1371,6 +1371,14 @@ struct spd_batch {
   int drafted_gamma = -1;
   int last_rows = 0;
   std::vector<void*> allocs;
+  // One step (forward + probability rows + sampling / rule kernels) is a fixed sequence of ~10 small
+  // launches per layer whose arguments never change (lengths and tokens live on the device), so it
+  // is captured once as a CUDA graph per (model, rows per sequence, draft step) and replayed.
+  cudaStream_t cap_stream = nullptr;
+  struct StepGraph { cudaGraphExec_t exec = nullptr; int seen = 0; };
+  StepGraph g_draft[MAX_M][MAX_M];   // [gamma][j]
+  StepGraph g_verify[MAX_M + 1];     // [gamma]
+  bool graphs_ok = true;
 };
 
 namespace {
@@ -1482,6 +1490,40 @@ spd_status batch_room(spd_batch* bt, int rows, bool draft) {
   return SPD_OK;
 }
 
+// Runs `enqueue` (which issues its launches on ctx->stream) either directly or, from its second use
+// on, as a replay of the graph captured from it.  The first use runs eagerly so that one-time set-up
+// (scratch growth, kernel attributes) happens outside any capture.
+template <class F>
+spd_status run_step_graph(spd_batch* bt, spd_batch::StepGraph& g, F enqueue) {
+  spd_ctx* ctx = bt->lead;
+  if (!bt->graphs_ok || g.seen == 0) { g.seen = 1; return enqueue(); }
+  if (!g.exec) {
+    if (!bt->cap_stream && cudaStreamCreateWithFlags(&bt->cap_stream, cudaStreamNonBlocking) != cudaSuccess) {
+      cudaGetLastError(); bt->graphs_ok = false; return enqueue();
+    }
+    cudaStream_t user = ctx->stream;
+    cudaGraph_t graph = nullptr;
+    bool ok = cudaStreamBeginCapture(bt->cap_stream, cudaStreamCaptureModeRelaxed) == cudaSuccess;
+    spd_status r = SPD_OK;
+    if (ok) {
+      ctx->stream = bt->cap_stream;          // the step's launches go to the capturing stream
+      r = enqueue();
+      ctx->stream = user;
+      ok = cudaStreamEndCapture(bt->cap_stream, &graph) == cudaSuccess && r == SPD_OK && graph != nullptr;
+    }
+    if (ok) ok = cudaGraphInstantiate(&g.exec, graph, 0) == cudaSuccess;
+    if (graph) cudaGraphDestroy(graph);
+    if (!ok) {                               // capture not available: plain launches from now on
+      cudaGetLastError();
+      g.exec = nullptr;
+      bt->graphs_ok = false;
+      return enqueue();
+    }
+  }
+  CU(cudaGraphLaunch(g.exec, ctx->stream));
+  return SPD_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -1489,6 +1531,12 @@ extern "C" {
 void spd_batch_destroy(spd_batch* bt) {
   if (!bt) return;
   if (bt->lead) cudaStreamSynchronize(bt->lead->stream);
+  for (auto& row : bt->g_draft)
+    for (auto& g : row)
+      if (g.exec) cudaGraphExecDestroy(g.exec);
+  for (auto& g : bt->g_verify)
+    if (g.exec) cudaGraphExecDestroy(g.exec);
+  if (bt->cap_stream) cudaStreamDestroy(bt->cap_stream);
   for (void* p : bt->allocs) cudaFree(p);
   delete bt;
 }
@@ -1571,12 +1619,18 @@ spd_status spd_batch_draft(spd_batch* bt, int gamma, const float* uniforms, int3
   const int B = bt->B, V = ctx->cfg.target.vocab;
   if (uniforms) CU(cudaMemcpyAsync(bt->u_draft, uniforms, (size_t)B * gamma * sizeof(float), cudaMemcpyDefault, ctx->stream));
   for (int j = 0; j < gamma; ++j) {
-    if ((s = batch_forward(bt, true, 2, j))) return s;
-    if (!ctx->cfg.greedy && (s = batch_probs(bt, 2 * B))) return s;
-    batch_draft_sample_kernel<<<B, SAMPLE_THREADS, 0, ctx->stream>>>(bt->seqs_dev, ctx->cfg.greedy ? bt->logits : bt->probs,
-                                                                      V, gamma, j, ctx->cfg.greedy, bt->u_draft, bt->q_all);
-    CU(cudaGetLastError());
+    auto step = [&]() -> spd_status {
+      spd_status r;
+      if ((r = batch_forward(bt, true, 2, j))) return r;
+      if (!ctx->cfg.greedy && (r = batch_probs(bt, 2 * B))) return r;
+      batch_draft_sample_kernel<<<B, SAMPLE_THREADS, 0, ctx->stream>>>(
+          bt->seqs_dev, ctx->cfg.greedy ? bt->logits : bt->probs, V, gamma, j, ctx->cfg.greedy, bt->u_draft, bt->q_all);
+      CU(cudaGetLastError());
+      return SPD_OK;
+    };
+    if ((s = run_step_graph(bt, bt->g_draft[gamma][j], step))) return s;
   }
+  bt->last_rows = 2 * B;
   bt->drafted_gamma = gamma;
   for (spd_ctx* c : bt->seqs) { c->drafted_gamma = -1; c->tree_drafted = false; }
   if (draft_ids) {
@@ -1599,12 +1653,18 @@ spd_status spd_batch_verify(spd_batch* bt, int gamma, const float* uniforms, int
   if ((s = batch_room(bt, gamma + 1, false))) return s;
   const int B = bt->B, V = ctx->cfg.target.vocab, M = gamma + 1;
   if (uniforms) CU(cudaMemcpyAsync(bt->u_verify, uniforms, (size_t)B * M * sizeof(float), cudaMemcpyDefault, ctx->stream));
-  if ((s = batch_forward(bt, false, M, 0))) return s;
-  if (!ctx->cfg.greedy && (s = batch_probs(bt, B * M))) return s;
-  batch_verify_kernel<<<B, SAMPLE_THREADS, 0, ctx->stream>>>(bt->seqs_dev, ctx->cfg.greedy ? bt->logits : bt->probs, bt->q_all,
-                                                              ctx->cfg.greedy ? nullptr : bt->u_verify, gamma, V,
-                                                              ctx->cfg.greedy, bt->out_acc, bt->out_next);
-  CU(cudaGetLastError());
+  auto step = [&]() -> spd_status {
+    spd_status r;
+    if ((r = batch_forward(bt, false, M, 0))) return r;
+    if (!ctx->cfg.greedy && (r = batch_probs(bt, B * M))) return r;
+    batch_verify_kernel<<<B, SAMPLE_THREADS, 0, ctx->stream>>>(bt->seqs_dev, ctx->cfg.greedy ? bt->logits : bt->probs,
+                                                                bt->q_all, ctx->cfg.greedy ? nullptr : bt->u_verify, gamma,
+                                                                V, ctx->cfg.greedy, bt->out_acc, bt->out_next);
+    CU(cudaGetLastError());
+    return SPD_OK;
+  };
+  if ((s = run_step_graph(bt, bt->g_verify[gamma], step))) return s;
+  bt->last_rows = B * M;
   bt->drafted_gamma = -1;
   for (spd_ctx* c : bt->seqs) { c->len_ub += M; c->drafted_gamma = -1; c->last_verify_rows = 0; }
   bool need_sync = false;

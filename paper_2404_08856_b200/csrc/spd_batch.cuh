@@ -74,28 +74,31 @@ __global__ void batch_rope_append_kernel(const float* qkv, int R, int M, int d, 
   }
 }
 
-// Attention of every sequence's M rows over its own cache: the single-sequence phase
-// (attn_phase_mma: units = head x KV split, partial results merged by the CTA that finishes a
-// head's last split) run for one sequence after the other by a grid of persistent CTAs, the unit
-// assignment rotated per sequence so that all CTAs stay busy.  No CTA waits for another.
-// `chain0`: block-row offset of row 0 (verify: 0; draft step j: j - 1); row m attends the rows
-// from the origin up to its own.
+// Attention of every sequence's M rows over its own cache.  Work unit = (sequence, head, KV split),
+// the single-sequence unit of attn_phase_mma (partial results of a head merged by the CTA that
+// finishes its last split); the units of ALL sequences form one list that a grid of persistent CTAs
+// walks with stride gridDim.x, so a CTA's next unit usually belongs to another sequence and no CTA
+// waits for another.  `chain0`: block-row offset of row 0 (verify: 0; draft step j: j - 1); row m
+// attends the rows from the origin up to its own.
 template <int M>
 __global__ void __launch_bounds__(CONSUMER_THREADS) batch_attn_kernel(const ModelDev* mds, const int* origins, int B,
                                                                       int layer, int chain0, int xbytes) {
   extern __shared__ __align__(1024) char bsm[];
   Ctrl* ctl = reinterpret_cast<Ctrl*>(bsm);
   char* xs = bsm + CTRL_BYTES;
-  const int G = gridDim.x;
   if (threadIdx.x < M) {
     const int top = chain0 + (int)threadIdx.x;          // highest block row this row attends (-1: none)
     ctl->sees[threadIdx.x] = top < 0 ? 0u : ((2u << top) - 1u);
   }
   __syncthreads();
-  for (int b = 0; b < B; ++b) {
+  const int umax = mds[0].H * mds[0].nsplit;            // most units a sequence can have
+  for (int g = blockIdx.x; g < B * umax; g += gridDim.x) {
+    const int b = g / umax, u = g - b * umax;
     const ModelDev md = mds[b];
-    const int cta = (int)((blockIdx.x + (unsigned)b * 37u) % (unsigned)G);
-    attn_phase_mma<M>(md, layer, origins[b], chain0 + M, cta, G, xs, xbytes, ctl);
+    const int units = md.H * eff_nsplit(md, origins[b] + chain0 + M);
+    if (u >= units) continue;
+    // one unit: the phase's own loop runs once for "CTA u of a grid of `units`"
+    attn_phase_mma<M>(md, layer, origins[b], chain0 + M, u, units, xs, xbytes, ctl);
     named_sync(1, CONSUMER_THREADS);
   }
 }
