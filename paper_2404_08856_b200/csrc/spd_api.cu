@@ -633,8 +633,11 @@ spd_status make_map(spd_ctx* ctx, CUtensorMap* m, const void* ptr, int inner, in
 
 struct Operand { const void* ptr; int inner, rows, batch; size_t row_stride, batch_stride; };
 
+// stream_ksplit = 0: the prefill form (3 stages, two CTAs per SM).  > 0: few rows against a large
+// weight matrix -- 6 stages, one CTA per SM, and the K loop cut into that many slices so that
+// enough CTAs stream; the slices' partial products go to `ws` and are summed in slice order.
 spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const Operand& b, TcArgs args,
-                   bool gelu = false) {
+                   bool gelu = false, int stream_ksplit = 0, float* ws = nullptr) {
   CUtensorMap ma, ml, mb;
   spd_status s;
   if ((s = make_map(ctx, &ma, a_hi.ptr, a_hi.inner, a_hi.rows, a_hi.batch, a_hi.row_stride, a_hi.batch_stride))) return s;
@@ -643,15 +646,34 @@ spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const
   static bool attr_set[MAX_DEV];
   if (ctx->device < 0 || ctx->device >= MAX_DEV) return fail(ctx, SPD_ECUDA, "device index out of range");
   if (!attr_set[ctx->device]) {
-    CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
-    CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
+    CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel<false, TC_STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
+    CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel<true, TC_STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
+    CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel<false, TC_STAGES_STREAM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                            tc_smem_bytes(TC_STAGES_STREAM)));
     attr_set[ctx->device] = true;
   }
   args.split = 1;
   args.err = &ctx->st->err;
+  args.ksplit = 1;
+  if (stream_ksplit > 0) {
+    if (gelu || a_hi.batch != 1 || args.mode == TC_OUT_SPLIT) return fail(ctx, SPD_EINVAL, "streaming GEMM: plain fp32 output only");
+    const int mode = args.mode;
+    float* dest = args.out_f32;
+    const long long ldo = args.ldo;
+    if (stream_ksplit > 1) {
+      if (!ws || ldo != args.N) return fail(ctx, SPD_EINVAL, "split GEMM needs a workspace and a dense output");
+      args.ksplit = stream_ksplit; args.out_f32 = ws; args.mode = TC_OUT_F32;
+    }
+    dim3 grid((args.N + TC_BN - 1) / TC_BN, (args.M + TC_BM - 1) / TC_BM, stream_ksplit);
+    tc_gemm_kernel<false, TC_STAGES_STREAM><<<grid, 128, tc_smem_bytes(TC_STAGES_STREAM), ctx->stream>>>(ma, ml, mb, args);
+    if (stream_ksplit > 1)
+      tc_reduce_kernel<<<148, 256, 0, ctx->stream>>>(ws, stream_ksplit, (size_t)args.M * args.N, dest, mode == TC_OUT_F32_ADD);
+    CU(cudaGetLastError());
+    return SPD_OK;
+  }
   dim3 grid((args.N + TC_BN - 1) / TC_BN, (args.M + TC_BM - 1) / TC_BM, a_hi.batch);
-  if (gelu) tc_gemm_kernel<true><<<grid, 128, TC_SMEM_BYTES, ctx->stream>>>(ma, ml, mb, args);
-  else tc_gemm_kernel<false><<<grid, 128, TC_SMEM_BYTES, ctx->stream>>>(ma, ml, mb, args);
+  if (gelu) tc_gemm_kernel<true, TC_STAGES><<<grid, 128, TC_SMEM_BYTES, ctx->stream>>>(ma, ml, mb, args);
+  else tc_gemm_kernel<false, TC_STAGES><<<grid, 128, TC_SMEM_BYTES, ctx->stream>>>(ma, ml, mb, args);
   CU(cudaGetLastError());
   return SPD_OK;
 }
@@ -1368,6 +1390,7 @@ struct spd_batch {
   ModelDev *mds_t = nullptr, *mds_d = nullptr;
   int *rowslot = nullptr, *origins = nullptr, *out_acc = nullptr, *out_next = nullptr;
   float *X = nullptr, *logits = nullptr, *probs = nullptr, *q_all = nullptr, *u_draft = nullptr, *u_verify = nullptr;
+  float* gemm_ws = nullptr;     // partial products of K-sliced GEMMs
   int drafted_gamma = -1;
   int last_rows = 0;
   std::vector<void*> allocs;
@@ -1395,9 +1418,11 @@ spd_status balloc(spd_batch* bt, T** p, size_t n) {
 }
 
 constexpr int BATCH_ATTN_SCRATCH = 200 * 1024;
+constexpr int BATCH_KSPLIT_MAX = 8;
 
 template <int M>
-spd_status launch_batch_attn(spd_ctx* ctx, const ModelDev* mds, const int* origins, int B, int layer, int chain0) {
+spd_status launch_batch_attn(spd_ctx* ctx, const ModelDev* mds, const int* origins, int B, int layer, int chain0,
+                             int max_split) {
   static bool attr[MAX_DEV];
   const size_t smem = CTRL_BYTES + BATCH_ATTN_SCRATCH;
   if (!attr[ctx->device]) {
@@ -1405,21 +1430,22 @@ spd_status launch_batch_attn(spd_ctx* ctx, const ModelDev* mds, const int* origi
     attr[ctx->device] = true;
   }
   batch_attn_kernel<M><<<ctx->n_sm, CONSUMER_THREADS, smem, ctx->stream>>>(mds, origins, B, layer, chain0,
-                                                                          BATCH_ATTN_SCRATCH);
+                                                                          BATCH_ATTN_SCRATCH, max_split);
   CU(cudaGetLastError());
   return SPD_OK;
 }
 
-spd_status batch_attn(spd_ctx* ctx, int M, const ModelDev* mds, const int* origins, int B, int layer, int chain0) {
+spd_status batch_attn(spd_ctx* ctx, int M, const ModelDev* mds, const int* origins, int B, int layer, int chain0,
+                      int max_split) {
   switch (M) {
-    case 1: return launch_batch_attn<1>(ctx, mds, origins, B, layer, chain0);
-    case 2: return launch_batch_attn<2>(ctx, mds, origins, B, layer, chain0);
-    case 3: return launch_batch_attn<3>(ctx, mds, origins, B, layer, chain0);
-    case 4: return launch_batch_attn<4>(ctx, mds, origins, B, layer, chain0);
-    case 5: return launch_batch_attn<5>(ctx, mds, origins, B, layer, chain0);
-    case 6: return launch_batch_attn<6>(ctx, mds, origins, B, layer, chain0);
-    case 7: return launch_batch_attn<7>(ctx, mds, origins, B, layer, chain0);
-    default: return launch_batch_attn<8>(ctx, mds, origins, B, layer, chain0);
+    case 1: return launch_batch_attn<1>(ctx, mds, origins, B, layer, chain0, max_split);
+    case 2: return launch_batch_attn<2>(ctx, mds, origins, B, layer, chain0, max_split);
+    case 3: return launch_batch_attn<3>(ctx, mds, origins, B, layer, chain0, max_split);
+    case 4: return launch_batch_attn<4>(ctx, mds, origins, B, layer, chain0, max_split);
+    case 5: return launch_batch_attn<5>(ctx, mds, origins, B, layer, chain0, max_split);
+    case 6: return launch_batch_attn<6>(ctx, mds, origins, B, layer, chain0, max_split);
+    case 7: return launch_batch_attn<7>(ctx, mds, origins, B, layer, chain0, max_split);
+    default: return launch_batch_attn<8>(ctx, mds, origins, B, layer, chain0, max_split);
   }
 }
 
@@ -1439,28 +1465,42 @@ spd_status batch_forward(spd_batch* bt, bool draft, int M, int j) {
   batch_embed_kernel<<<R, 128, 0, cs>>>(bt->seqs_dev, B, M, draft ? 1 : 0, j, mh.md.embed, d, V, X, bt->rowslot,
                                         bt->origins, &ctx->st->err);
   const Operand h_hi{pf.h_hi, d, R, 1, (size_t)d * 2, (size_t)R * d * 2}, h_lo{pf.h_lo, d, R, 1, (size_t)d * 2, (size_t)R * d * 2};
+  // KV splits per head: about two (sequence, head, split) units per SM, never more than a single sequence would use
+  int attn_split = (2 * ctx->n_sm + B * H - 1) / (B * H);
+  if (attn_split > mh.md.nsplit) attn_split = mh.md.nsplit;
+  if (attn_split < 1) attn_split = 1;
+  // every GEMM here is a few rows against a large weight matrix: cut K so that about one CTA per SM streams
+  auto ksplit = [&](int N, int K) {
+    const int tiles = (N + TC_BN - 1) / TC_BN, kb = (K + TC_BK - 1) / TC_BK;
+    int sp = (ctx->n_sm + tiles - 1) / tiles;
+    if (sp > BATCH_KSPLIT_MAX) sp = BATCH_KSPLIT_MAX;
+    if (sp > kb / 8) sp = kb / 8 > 0 ? kb / 8 : 1;       // at least 8 K blocks per slice
+    return sp < 1 ? 1 : sp;
+  };
   for (int l = 0; l < L; ++l) {
     const ModelHost::RowMajor& w = mh.rm[l];
     TcArgs a{};
     rms_split_kernel<<<R, 256, 0, cs>>>(X, w.attn_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
     a = TcArgs{}; a.M = R; a.N = 3 * d; a.K = d; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = pf.wide; a.ldo = 3 * d;
-    if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wqkv, d, 3 * d, 1, (size_t)d * 2, (size_t)3 * d * d * 2}, a))) return s;
+    if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wqkv, d, 3 * d, 1, (size_t)d * 2, (size_t)3 * d * d * 2}, a, false,
+                     ksplit(3 * d, d), bt->gemm_ws))) return s;
     batch_rope_append_kernel<<<296, 256, 0, cs>>>(pf.wide, R, M, d, dh, bt->rowslot, mh.md.rope_cos, mh.md.rope_sin, mds, l);
-    if ((s = batch_attn(ctx, M, mds, bt->origins, B, l, draft ? j - 1 : 0))) return s;
+    if ((s = batch_attn(ctx, M, mds, bt->origins, B, l, draft ? j - 1 : 0, attn_split))) return s;
     batch_gather_split_kernel<<<296, 256, 0, cs>>>(mds, R, M, d, pf.h_hi, pf.h_lo);
     a = TcArgs{}; a.M = R; a.N = d; a.K = d; a.mode = TC_OUT_F32_ADD; a.alpha = 1.f; a.out_f32 = X; a.ldo = d;
-    if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wo, d, d, 1, (size_t)d * 2, (size_t)d * d * 2}, a))) return s;
+    if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wo, d, d, 1, (size_t)d * 2, (size_t)d * d * 2}, a, false, ksplit(d, d), bt->gemm_ws))) return s;
     rms_split_kernel<<<R, 256, 0, cs>>>(X, w.ffn_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
     a = TcArgs{}; a.M = R; a.N = 2 * f; a.K = d; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = pf.wide; a.ldo = 2 * f;
-    if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wgu, d, 2 * f, 1, (size_t)d * 2, (size_t)2 * f * d * 2}, a))) return s;
+    if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wgu, d, 2 * f, 1, (size_t)d * 2, (size_t)2 * f * d * 2}, a, false,
+                     ksplit(2 * f, d), bt->gemm_ws))) return s;
     swiglu_split_kernel<<<296, 256, 0, cs>>>(pf.wide, R, f, pf.h_hi, pf.h_lo);
     a = TcArgs{}; a.M = R; a.N = d; a.K = f; a.mode = TC_OUT_F32_ADD; a.alpha = 1.f; a.out_f32 = X; a.ldo = d;
     if ((s = tc_gemm(ctx, {pf.h_hi, f, R, 1, (size_t)f * 2, (size_t)R * f * 2}, {pf.h_lo, f, R, 1, (size_t)f * 2, (size_t)R * f * 2},
-                     {w.wd, f, d, 1, (size_t)f * 2, (size_t)d * f * 2}, a))) return s;
+                     {w.wd, f, d, 1, (size_t)f * 2, (size_t)d * f * 2}, a, false, ksplit(d, f), bt->gemm_ws))) return s;
   }
   rms_split_kernel<<<R, 256, 0, cs>>>(X, mh.md.final_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
   TcArgs a{}; a.M = R; a.N = V; a.K = d; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = bt->logits; a.ldo = V;
-  if ((s = tc_gemm(ctx, h_hi, h_lo, {mh.lm_rm, d, V, 1, (size_t)d * 2, (size_t)V * d * 2}, a))) return s;
+  if ((s = tc_gemm(ctx, h_hi, h_lo, {mh.lm_rm, d, V, 1, (size_t)d * 2, (size_t)V * d * 2}, a, false, ksplit(V, d), bt->gemm_ws))) return s;
   CU(cudaGetLastError());
   bt->last_rows = R;
   return SPD_OK;
@@ -1580,6 +1620,14 @@ spd_status spd_batch_create(spd_ctx* const* seqs, int B, spd_batch** out) {
   if (!s) s = balloc(bt, &bt->q_all, (size_t)B * gm * V);
   if (!s) s = balloc(bt, &bt->u_draft, (size_t)B * MAX_M);
   if (!s) s = balloc(bt, &bt->u_verify, (size_t)B * MAX_M);
+  {   // widest split output: [slices][128 rows][max(3 d, 2 f, V)]
+    size_t wide = (size_t)V;
+    for (const spd_model_cfg* c : {&ctx->cfg.target, &ctx->cfg.draft}) {
+      if ((size_t)3 * c->d_model > wide) wide = (size_t)3 * c->d_model;
+      if ((size_t)2 * c->d_ffn > wide) wide = (size_t)2 * c->d_ffn;
+    }
+    if (!s) s = balloc(bt, &bt->gemm_ws, (size_t)BATCH_KSPLIT_MAX * BATCH_ROWS_MAX * wide);
+  }
   if (!s && ctx->truncate &&
       cudaFuncSetAttribute((const void*)truncate_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)((size_t)V * sizeof(float))) != cudaSuccess)

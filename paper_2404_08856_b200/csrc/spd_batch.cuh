@@ -80,9 +80,11 @@ __global__ void batch_rope_append_kernel(const float* qkv, int R, int M, int d, 
 // walks with stride gridDim.x, so a CTA's next unit usually belongs to another sequence and no CTA
 // waits for another.  `chain0`: block-row offset of row 0 (verify: 0; draft step j: j - 1); row m
 // attends the rows from the origin up to its own.
+// `max_split`: KV splits per head at most -- with B sequences there are enough (sequence, head) pairs
+// to fill the grid, so heads are cut no further than needed (fewer partial results to merge).
 template <int M>
 __global__ void __launch_bounds__(CONSUMER_THREADS) batch_attn_kernel(const ModelDev* mds, const int* origins, int B,
-                                                                      int layer, int chain0, int xbytes) {
+                                                                      int layer, int chain0, int xbytes, int max_split) {
   extern __shared__ __align__(1024) char bsm[];
   Ctrl* ctl = reinterpret_cast<Ctrl*>(bsm);
   char* xs = bsm + CTRL_BYTES;
@@ -91,14 +93,15 @@ __global__ void __launch_bounds__(CONSUMER_THREADS) batch_attn_kernel(const Mode
     ctl->sees[threadIdx.x] = top < 0 ? 0u : ((2u << top) - 1u);
   }
   __syncthreads();
-  const int umax = mds[0].H * mds[0].nsplit;            // most units a sequence can have
+  const int umax = mds[0].H * max_split;                // most units a sequence can have
   for (int g = blockIdx.x; g < B * umax; g += gridDim.x) {
     const int b = g / umax, u = g - b * umax;
-    const ModelDev md = mds[b];
+    ModelDev md = mds[b];
+    md.nsplit = max_split;
     const int units = md.H * eff_nsplit(md, origins[b] + chain0 + M);
     if (u >= units) continue;
     // one unit: the phase's own loop runs once for "CTA u of a grid of `units`"
-    attn_phase_mma<M>(md, layer, origins[b], chain0 + M, u, units, xs, xbytes, ctl);
+    attn_phase_mma<M, true>(md, layer, origins[b], chain0 + M, u, units, xs, xbytes, ctl);
     named_sync(1, CONSUMER_THREADS);
   }
 }

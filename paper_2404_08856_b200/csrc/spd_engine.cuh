@@ -1013,7 +1013,9 @@ __device__ __forceinline__ void split_frag(float2 xa, float2 xb, uint32_t& h0, u
 // fp32 q split into bf16 hi + lo).  Output: D[16 dims x 8 queries] = V^T (A, transposing
 // ldmatrix) x P^T (B, fp32 probabilities split the same way); warp w owns dims 16w..16w+15,
 // so no cross-warp reduction is needed.  Tile rows are 16-byte-chunk swizzled by position.
-template <int M>
+// PIPE (the batched kernel, where a unit spans several sub-chunks): two K/V tile buffers, the
+// next sub-chunk's rows are requested before the current one is computed.
+template <int M, bool PIPE = false>
 __device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int nslots, int cta, int G, char* xs,
                                int xbytes, Ctrl* ctl) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -1024,19 +1026,38 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int ns
   const int rowb = dh * 2, cpr = rowb >> 4;
   const int gq = lane >> 2, tq = lane & 3, mat = lane >> 3, rr = lane & 7;
   const int qst = dh + 8;                                    // padded fp32 row of q
-  // scratch: q [M][dh+8] fp32 | K tile [SC][rowb] | V tile [SC][rowb] | S [M][SC+8] fp32
-  int SC = ((xbytes - M * qst * 4 - M * 8 * 4) / (2 * rowb + M * 4)) & ~15;
+  const char* Kl = static_cast<const char*>(md.kcache) + (size_t)layer * md.max_seq * d * 2;
+  const char* Vl = static_cast<const char*>(md.vcache) + (size_t)layer * md.max_seq * d * 2;
+  // scratch: q [M][dh+8] fp32 | NB x (K tile [SC][rowb] | V tile [SC][rowb]) | S [M][SC+8] fp32
+  constexpr int NB = PIPE ? 2 : 1;
+  int SC = ((xbytes - M * qst * 4 - M * 8 * 4) / (2 * NB * rowb + M * 4)) & ~15;
   {  // equal sub-chunks instead of full ones plus a sliver
     const int nsub = (Lc + SC - 1) / SC;
     SC = min(SC, (((Lc + nsub - 1) / nsub) + 15) & ~15);
   }
   const int sst = SC + 8;
   float* qs = reinterpret_cast<float*>(xs);
-  char* Kt = xs + M * qst * 4;
-  char* Vt = Kt + (size_t)SC * rowb;
-  float* S = reinterpret_cast<float*>(Vt + (size_t)SC * rowb);
-  const char* Kl = static_cast<const char*>(md.kcache) + (size_t)layer * md.max_seq * d * 2;
-  const char* Vl = static_cast<const char*>(md.vcache) + (size_t)layer * md.max_seq * d * 2;
+  char* const Kt0 = xs + M * qst * 4;
+  const size_t tileb = (size_t)SC * rowb;
+  float* S = reinterpret_cast<float*>(Kt0 + 2 * NB * tileb);
+  // request rows [c0, c0 + n) of the head's K and V into tile buffer `buf`
+  auto request = [&](int h, int c0, int n, int buf) {
+    char* Kt = Kt0 + (size_t)buf * 2 * tileb;
+    char* Vt = Kt + tileb;
+    const int n16 = (n + 15) & ~15;
+    for (int i = tid; i < n16 * cpr; i += CONSUMER_THREADS) {
+      const int r = i / cpr, cc = i - r * cpr;
+      const int dst = r * rowb + ((cc ^ (r & 7)) << 4);
+      if (r < n) {
+        const size_t g = ((size_t)(c0 + r) * d + h * dh) * 2 + (size_t)cc * 16;
+        cp_async16(Kt + dst, Kl + g);
+        cp_async16(Vt + dst, Vl + g);
+      } else {   // rows past the end must not hold NaN patterns: P is 0 there
+        *reinterpret_cast<uint4*>(Vt + dst) = make_uint4(0, 0, 0, 0);
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
   const int nkd = dh >> 4;                                   // 16-wide slices of the head dim
 
   for (int unit = cta; unit < H * nsplit; unit += G) {
@@ -1049,20 +1070,24 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int ns
     }
     if (tid < M) { ctl->rowmax[tid] = -INFINITY; ctl->rowsum[tid] = 0.f; }
     float oacc[4] = {0.f, 0.f, 0.f, 0.f};
+    int buf = 0;
+    if (PIPE) request(h, p0, min(SC, p1 - p0), 0);
     for (int c0 = p0; c0 < p1; c0 += SC) {
       const int n = min(SC, p1 - c0), n16 = (n + 15) & ~15;
-      for (int i = tid; i < n16 * cpr; i += CONSUMER_THREADS) {
-        const int r = i / cpr, cc = i - r * cpr;
-        const int dst = r * rowb + ((cc ^ (r & 7)) << 4);
-        if (r < n) {
-          const size_t g = ((size_t)(c0 + r) * d + h * dh) * 2 + (size_t)cc * 16;
-          cp_async16(Kt + dst, Kl + g);
-          cp_async16(Vt + dst, Vl + g);
-        } else {   // rows past the end must not hold NaN patterns: P is 0 there
-          *reinterpret_cast<uint4*>(Vt + dst) = make_uint4(0, 0, 0, 0);
+      if (PIPE) {
+        const int c1 = c0 + SC;
+        if (c1 < p1) {
+          request(h, c1, min(SC, p1 - c1), buf ^ 1);
+          asm volatile("cp.async.wait_group 1;" ::: "memory");
+        } else {
+          asm volatile("cp.async.wait_group 0;" ::: "memory");
         }
+      } else {
+        request(h, c0, n, 0);
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
       }
-      cp_async_wait_all();
+      char* Kt = Kt0 + (size_t)buf * 2 * tileb;
+      char* Vt = Kt + tileb;
       named_sync(1, CONSUMER_THREADS);
       // ---- scores: warp takes 16-position groups
       for (int gp = warp; gp * 16 < n; gp += 8) {
@@ -1143,6 +1168,7 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int ns
         }
       }
       named_sync(1, CONSUMER_THREADS);   // tiles and S are free again
+      if (PIPE) buf ^= 1;
     }
     // oacc[0,1]: dim 16w+gq, queries 2tq, 2tq+1; oacc[2,3]: dim +8
     if (nsplit == 1) {   // the whole context was here: normalise and finish the head
@@ -1177,7 +1203,7 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int ns
       __threadfence();
     }
     named_sync(1, CONSUMER_THREADS);
-    if (ctl->flag) merge_head<M>(md, h, nsplit, reinterpret_cast<float*>(Kt));
+    if (ctl->flag) merge_head<M>(md, h, nsplit, reinterpret_cast<float*>(Kt0));
     named_sync(1, CONSUMER_THREADS);
   }
 }

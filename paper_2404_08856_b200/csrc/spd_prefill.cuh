@@ -15,10 +15,13 @@
 
 namespace spd {
 
-constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64, TC_STAGES = 3;   // 3 stages: two CTAs per SM
+constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64;
+constexpr int TC_STAGES = 3;          // prefill (compute-bound, many tiles): 3 stages, two CTAs per SM
+constexpr int TC_STAGES_STREAM = 6;   // few rows against large weights (HBM-bound): 6 stages, one CTA per SM
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2, TC_B_BYTES = TC_BN * TC_BK * 2;
 constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;                  // 32 KB
-constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 + 256;   // + alignment slack + barriers
+__host__ __device__ constexpr int tc_smem_bytes(int stages) { return stages * TC_STAGE_BYTES + 1024 + 256; }   // + alignment slack + barriers
+constexpr int TC_SMEM_BYTES = tc_smem_bytes(TC_STAGES);
 constexpr int TC_TMEM_COLS = 128;
 
 enum : int { TC_OUT_F32 = 0, TC_OUT_F32_ADD = 1, TC_OUT_SPLIT = 2 };
@@ -32,6 +35,8 @@ struct TcArgs {
   __nv_bfloat16 *out_hi, *out_lo;
   long long ldo, out_batch; // output row stride and per-batch offset, in elements
   int* err;                 // sticky error word (DEV_TIMEOUT_*)
+  int ksplit;               // > 1: blockIdx.z is a slice of the K loop (not a batch index); slice s stores its
+                            // partial product (alpha applied) at out_f32 + s * M * ldo, summed by tc_reduce_kernel
 };
 
 __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
@@ -82,22 +87,24 @@ __device__ __forceinline__ float gelu_exact(float x) { return 0.5f * x * (1.0f +
 // grid = (N tiles, M tiles, batch); 128 threads: thread 0 feeds TMA, thread 32 issues the MMAs,
 // all four warps read the accumulator back (warp w owns TMEM lanes 32w..32w+31 = tile rows).
 // GELU: the hi/lo output (TC_OUT_SPLIT) is gelu(alpha * accumulator) instead of alpha * accumulator.
-template <bool GELU>
-__global__ void __launch_bounds__(128, 2)
+template <bool GELU, int STAGES>
+__global__ void __launch_bounds__(128, STAGES <= 3 ? 2 : 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
                const __grid_constant__ CUtensorMap map_b, const TcArgs a) {
   extern __shared__ uint8_t tc_smem_raw[];
   uint8_t* stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full = reinterpret_cast<uint64_t*>(stages + TC_STAGES * TC_STAGE_BYTES);
-  uint64_t* empty = full + TC_STAGES;
-  uint64_t* accum = empty + TC_STAGES;
+  uint64_t* full = reinterpret_cast<uint64_t*>(stages + STAGES * TC_STAGE_BYTES);
+  uint64_t* empty = full + STAGES;
+  uint64_t* accum = empty + STAGES;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
   volatile int* err = a.err;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int tile_n = blockIdx.x, tile_m = blockIdx.y, z = blockIdx.z;
+  const int tile_n = blockIdx.x, tile_m = blockIdx.y;
+  const int z = a.ksplit > 1 ? 0 : (int)blockIdx.z;           // batch index
+  const int slice = a.ksplit > 1 ? (int)blockIdx.z : 0;       // slice of the K loop
 
   if (tid == 0) {
-    for (int i = 0; i < TC_STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     mbar_init(accum, 1);
     mbar_fence_init();
   }
@@ -112,16 +119,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
-  const int k_blocks = (a.K + TC_BK - 1) / TC_BK;
+  const int k_all = (a.K + TC_BK - 1) / TC_BK;
+  const int k_per = a.ksplit > 1 ? (k_all + a.ksplit - 1) / a.ksplit : k_all;
+  const int k_first = slice * k_per;
+  const int k_blocks = max(0, min(k_all, k_first + k_per) - k_first);
   const int total = k_blocks * (a.split ? 2 : 1);
   if (tid == 0) {
     // ---- TMA producer
     for (int it = 0; it < total; ++it) {
-      const int s = it % TC_STAGES;
-      const unsigned ph = (it / TC_STAGES) & 1;
+      const int s = it % STAGES;
+      const unsigned ph = (it / STAGES) & 1;
       if (!mbar_wait(&empty[s], ph ^ 1u, err, DEV_TIMEOUT_EMPTY)) break;
       mbar_arrive_expect_tx(&full[s], TC_STAGE_BYTES);
-      const int kb = it % k_blocks;
+      const int kb = k_first + it % k_blocks;
       const CUtensorMap* ma = (it >= k_blocks) ? &map_a_lo : &map_a_hi;
       tma_load_3d(stages + s * TC_STAGE_BYTES, ma, kb * TC_BK, tile_m * TC_BM, z, &full[s]);
       tma_load_3d(stages + s * TC_STAGE_BYTES + TC_A_BYTES, &map_b, kb * TC_BK, tile_n * TC_BN, z, &full[s]);
@@ -130,8 +140,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
     // ---- MMA issuer
     bool ok = true;
     for (int it = 0; it < total && ok; ++it) {
-      const int s = it % TC_STAGES;
-      const unsigned ph = (it / TC_STAGES) & 1;
+      const int s = it % STAGES;
+      const unsigned ph = (it / STAGES) & 1;
       ok = mbar_wait(&full[s], ph, err, DEV_TIMEOUT_FULL);
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -146,17 +156,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
   }
   __syncwarp();
   // ---- epilogue
-  const bool done = mbar_wait(accum, 0u, err, DEV_TIMEOUT_FULL);
+  // (a K slice that got no block -- more slices than blocks -- has nothing to wait for and stores zeros)
+  const bool done = total == 0 ? true : mbar_wait(accum, 0u, err, DEV_TIMEOUT_FULL);
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const int row = tile_m * TC_BM + warp * 32 + lane;
   if (done) {
 #pragma unroll 1
     for (int c0 = 0; c0 < TC_BN; c0 += 32) {
       uint32_t v[32];
-      tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+      if (total == 0) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = 0u;
+      } else {
+        tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+      }
       const int col0 = tile_n * TC_BN + c0;
       if (row < a.M && col0 < a.N) {
-        const long long off = (long long)z * a.out_batch + (long long)row * a.ldo + col0;
+        const long long off = (long long)z * a.out_batch + (long long)slice * a.M * a.ldo + (long long)row * a.ldo + col0;
         const int nv = min(32, a.N - col0);
         // a thread owns 32 consecutive columns of its row: 16-byte stores where the row start
         // and the width allow it (ldo and out_batch multiples of 8, all 32 columns present)
@@ -223,6 +239,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
   if (warp == 0) {
     if (!done) for (int i = 0; i < 200; ++i) __nanosleep(1000);   // let copies in flight land
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
+  }
+}
+
+// Sum of the K slices of a split GEMM, in slice order (deterministic): out (+)= sum_s part[s].
+__global__ void tc_reduce_kernel(const float* part, int slices, size_t n, float* out, int add) {
+  for (size_t i = (blockIdx.x * (size_t)blockDim.x + threadIdx.x) * 4; i < n; i += (size_t)gridDim.x * blockDim.x * 4) {
+    float4 acc = add ? *reinterpret_cast<const float4*>(out + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < slices; ++s) {
+      const float4 p = *reinterpret_cast<const float4*>(part + (size_t)s * n + i);
+      acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+    }
+    *reinterpret_cast<float4*>(out + i) = acc;
   }
 }
 
