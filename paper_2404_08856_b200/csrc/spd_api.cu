@@ -388,20 +388,24 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
 
 using KernelFn = void (*)(const StepArgs);
 
-template <typename WT>
+template <typename WT, bool TRACE>
 KernelFn pick_m(int M) {
   switch (M) {
-    case 1: return forward_kernel<1, WT>;
-    case 2: return forward_kernel<2, WT>;
-    case 3: return forward_kernel<3, WT>;
-    case 4: return forward_kernel<4, WT>;
-    case 5: return forward_kernel<5, WT>;
-    case 6: return forward_kernel<6, WT>;
-    case 7: return forward_kernel<7, WT>;
-    default: return forward_kernel<8, WT>;
+    case 1: return forward_kernel<1, WT, TRACE>;
+    case 2: return forward_kernel<2, WT, TRACE>;
+    case 3: return forward_kernel<3, WT, TRACE>;
+    case 4: return forward_kernel<4, WT, TRACE>;
+    case 5: return forward_kernel<5, WT, TRACE>;
+    case 6: return forward_kernel<6, WT, TRACE>;
+    case 7: return forward_kernel<7, WT, TRACE>;
+    default: return forward_kernel<8, WT, TRACE>;
   }
 }
-KernelFn pick_kernel(int M, int dtype) { return dtype == 1 ? pick_m<__nv_bfloat16>(M) : pick_m<float>(M); }
+// trace: the instantiation with phase timestamps (spd_trace); the plain one carries none
+KernelFn pick_kernel(int M, int dtype, bool trace = false) {
+  if (trace) return dtype == 1 ? pick_m<__nv_bfloat16, true>(M) : pick_m<float, true>(M);
+  return dtype == 1 ? pick_m<__nv_bfloat16, false>(M) : pick_m<float, false>(M);
+}
 
 struct LaunchCfg { int nstage; size_t smem; };
 
@@ -410,13 +414,13 @@ constexpr int MAX_DEV = 64;   // devices per process that the per-device tables 
 spd_status launch_cfg(spd_ctx* ctx, KernelFn fn, int M, int n_sm, int smem_optin, LaunchCfg* lc) {
   // per device and kernel variant; filled on first use (the shared-memory attribute of a kernel
   // belongs to the device it was set on)
-  static LaunchCfg cache_all[MAX_DEV][2 * (MAX_M + 1)];
-  static KernelFn cache_fn_all[MAX_DEV][2 * (MAX_M + 1)];
+  static LaunchCfg cache_all[MAX_DEV][4 * (MAX_M + 1)];
+  static KernelFn cache_fn_all[MAX_DEV][4 * (MAX_M + 1)];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEV) return fail(ctx, SPD_ECUDA, "no current device");
   LaunchCfg* cache = cache_all[dev];
   KernelFn* cache_fn = cache_fn_all[dev];
-  for (int i = 0; i < 2 * (MAX_M + 1); ++i)
+  for (int i = 0; i < 4 * (MAX_M + 1); ++i)
     if (cache_fn[i] == fn) { *lc = cache[i]; return SPD_OK; }
   cudaFuncAttributes fa{};
   CU(cudaFuncGetAttributes(&fa, (const void*)fn));
@@ -429,7 +433,7 @@ spd_status launch_cfg(spd_ctx* ctx, KernelFn fn, int M, int n_sm, int smem_optin
   lc->smem = fixed + (size_t)ns * STAGE_BYTES;
   CU(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lc->smem));
   (void)n_sm;
-  for (int i = 0; i < 2 * (MAX_M + 1); ++i)
+  for (int i = 0; i < 4 * (MAX_M + 1); ++i)
     if (!cache_fn[i]) { cache[i] = *lc; cache_fn[i] = fn; break; }
   return SPD_OK;
 }
@@ -457,7 +461,7 @@ bool cluster_fits(KernelFn fn, int cs, size_t smem) {
 // and synchronise inside it, otherwise it is a cooperative launch with the barrier word `bar`.
 spd_status launch_forward(spd_ctx* ctx, int M, int dtype, StepArgs a, cudaStream_t stream, int grid, int cluster,
                           int smem_optin, unsigned* bar, int n_sm_sampling) {
-  KernelFn fn = pick_kernel(M, dtype);
+  KernelFn fn = pick_kernel(M, dtype, a.trace != nullptr);
   LaunchCfg lc{};
   spd_status s = launch_cfg(ctx, fn, M, grid, smem_optin, &lc);
   if (s) return s;

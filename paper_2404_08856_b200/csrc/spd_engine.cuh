@@ -510,7 +510,7 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
 }
 
 // This CTA's share of one projection.  src gives the M activation rows (fp32).
-template <int M, typename WT>
+template <int M, typename WT, bool TRACE>
 __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, const XSrc& src, const float* norm_w, float eps,
                              float* copy_out, const float* ssq_in, int cta, int G, Ring& ring, Ctrl* ctl, float* X,
                              unsigned& xphase, float* red, float* pre_s, uint32_t zero_addr, const char* stages, volatile int* err) {
@@ -541,7 +541,7 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, const XSrc& src, c
     else
       load_x<M, false>(X, kcl, g.K, src, 0, nullptr, eps, g.K, ctl, xphase, nullptr, err, prenorm ? ssq_in : nullptr, G);
   }
-  trace_stamp(ctl, 1);
+  if constexpr (TRACE) trace_stamp(ctl, 1);
   const int gq = lane >> 2, tq = lane & 3;
   float ssq_acc = 0.f;    // threads 0..7: this CTA's sum of x^2 of activation row tid (bf16 RESID with xg)
   for (int t = 0; t * 32 < rows; ++t) {
@@ -625,7 +625,7 @@ __device__ void consume_gemm(const Gemm& g, const EpiArgs& e, const XSrc& src, c
         ring.advance();
       }
     }
-    if (t * 32 + 32 >= rows) trace_stamp(ctl, 2);
+    if constexpr (TRACE) { if (t * 32 + 32 >= rows) trace_stamp(ctl, 2); }
     if constexpr (!BF) {
       // 4*M sums per warp, value index m*4 + r
       float v[4 * M];
