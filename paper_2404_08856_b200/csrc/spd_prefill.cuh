@@ -6,8 +6,10 @@
 //
 // Precision: B operands are exact bf16 data (weights, cached K and V).  The A operand
 // (activations, probabilities) is fp32 upstream and is fed as TWO bf16 matrices hi + lo
-// (x = hi + lo up to 2^-17 |x|), i.e. the K loop runs twice.  Prefill results therefore
-// match an fp32 reference to ~1e-5 relative, like the M <= 8 path, at twice the tensor work.
+// (x = hi + lo up to 2^-17 |x|): a stage holds the hi tile, the lo tile and ONE B tile of a K
+// block, and both products accumulate into the same tensor-memory columns.  Prefill results
+// therefore match an fp32 reference to ~1e-5 relative, like the M <= 8 path, at twice the
+// tensor work but with every B tile loaded once.
 #pragma once
 #include <cuda.h>
 
@@ -16,10 +18,10 @@
 namespace spd {
 
 constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64;
-constexpr int TC_STAGES = 3;          // prefill (compute-bound, many tiles): 3 stages, two CTAs per SM
-constexpr int TC_STAGES_STREAM = 6;   // few rows against large weights (HBM-bound): 6 stages, one CTA per SM
+constexpr int TC_STAGES = 2;          // prefill (compute-bound, many tiles): 2 stages, two CTAs per SM
+constexpr int TC_STAGES_STREAM = 4;   // few rows against large weights (HBM-bound): 4 stages, one CTA per SM
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2, TC_B_BYTES = TC_BN * TC_BK * 2;
-constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;                  // 32 KB
+constexpr int TC_STAGE_BYTES = 2 * TC_A_BYTES + TC_B_BYTES;              // A hi | A lo | B = 48 KB
 __host__ __device__ constexpr int tc_smem_bytes(int stages) { return stages * TC_STAGE_BYTES + 1024 + 256; }   // + alignment slack + barriers
 constexpr int TC_SMEM_BYTES = tc_smem_bytes(TC_STAGES);
 constexpr int TC_TMEM_COLS = 128;
@@ -28,7 +30,7 @@ enum : int { TC_OUT_F32 = 0, TC_OUT_F32_ADD = 1, TC_OUT_SPLIT = 2 };
 
 struct TcArgs {
   int M, N, K;              // A rows, B rows (= output columns), inner dimension
-  int split;                // 1: A is given as hi and lo maps
+  int split;                // (always 1: A is given as hi and lo maps)
   int mode;                 // TC_OUT_*
   float alpha;              // result scale
   float* out_f32;
@@ -123,7 +125,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
   const int k_per = a.ksplit > 1 ? (k_all + a.ksplit - 1) / a.ksplit : k_all;
   const int k_first = slice * k_per;
   const int k_blocks = max(0, min(k_all, k_first + k_per) - k_first);
-  const int total = k_blocks * (a.split ? 2 : 1);
+  const int total = k_blocks;
   if (tid == 0) {
     // ---- TMA producer
     for (int it = 0; it < total; ++it) {
@@ -131,10 +133,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
       const unsigned ph = (it / STAGES) & 1;
       if (!mbar_wait(&empty[s], ph ^ 1u, err, DEV_TIMEOUT_EMPTY)) break;
       mbar_arrive_expect_tx(&full[s], TC_STAGE_BYTES);
-      const int kb = k_first + it % k_blocks;
-      const CUtensorMap* ma = (it >= k_blocks) ? &map_a_lo : &map_a_hi;
-      tma_load_3d(stages + s * TC_STAGE_BYTES, ma, kb * TC_BK, tile_m * TC_BM, z, &full[s]);
-      tma_load_3d(stages + s * TC_STAGE_BYTES + TC_A_BYTES, &map_b, kb * TC_BK, tile_n * TC_BN, z, &full[s]);
+      const int kb = k_first + it;
+      tma_load_3d(stages + s * TC_STAGE_BYTES, &map_a_hi, kb * TC_BK, tile_m * TC_BM, z, &full[s]);
+      tma_load_3d(stages + s * TC_STAGE_BYTES + TC_A_BYTES, &map_a_lo, kb * TC_BK, tile_m * TC_BM, z, &full[s]);
+      tma_load_3d(stages + s * TC_STAGE_BYTES + 2 * TC_A_BYTES, &map_b, kb * TC_BK, tile_n * TC_BN, z, &full[s]);
     }
   } else if (tid == 32) {
     // ---- MMA issuer
@@ -145,11 +147,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
       ok = mbar_wait(&full[s], ph, err, DEV_TIMEOUT_FULL);
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint64_t ad = umma_desc(smem_u32(stages + s * TC_STAGE_BYTES));
-      const uint64_t bd = umma_desc(smem_u32(stages + s * TC_STAGE_BYTES + TC_A_BYTES));
+      const uint64_t ah = umma_desc(smem_u32(stages + s * TC_STAGE_BYTES));
+      const uint64_t al = umma_desc(smem_u32(stages + s * TC_STAGE_BYTES + TC_A_BYTES));
+      const uint64_t bd = umma_desc(smem_u32(stages + s * TC_STAGE_BYTES + 2 * TC_A_BYTES));
 #pragma unroll
-      for (int k = 0; k < TC_BK / 16; ++k)   // 32 bytes further along K inside the swizzle atom
-        umma_bf16(tmem_base, ad + 2 * k, bd + 2 * k, (it > 0 || k > 0) ? 1u : 0u);
+      for (int k = 0; k < TC_BK / 16; ++k) {   // 32 bytes further along K inside the swizzle atom
+        umma_bf16(tmem_base, ah + 2 * k, bd + 2 * k, (it > 0 || k > 0) ? 1u : 0u);
+        umma_bf16(tmem_base, al + 2 * k, bd + 2 * k, 1u);
+      }
       umma_commit(&empty[s]);   // the stage is free once these MMAs have read it
     }
     umma_commit(accum);         // arrives when every MMA above has completed
