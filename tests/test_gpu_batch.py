@@ -19,11 +19,14 @@ def _inputs(wl, k, extra_prompt):
     return synth.image_embeds(w2), synth.prompt_ids(w2)
 
 
-def run_batch_lockstep(wl, B, gamma, n_blocks, greedy, logit_tol, std, extra_prompt=3, max_seq=None):
+def run_batch_lockstep(wl, B, gamma, n_blocks, greedy, logit_tol, std, extra_prompt=3, max_seq=None, top_k=0):
+    """top_k = 1 (sampling mode): every row is a point mass at its arg-max, so the sampling kernels of
+    the batched path must reproduce greedy decoding whatever the uniforms are; the oracle then runs
+    greedy."""
     spd = _lib()
     tw, dw = H.build_weights(wl, std)
     max_seq = max_seq or (wl.n_image + wl.n_prompt + extra_prompt * B + 8 * (n_blocks + 2) + 16)
-    seqs = [H.make_gpu(wl, tw, dw, max_seq, 1.0, greedy)]
+    seqs = [H.make_gpu(wl, tw, dw, max_seq, 1.0, greedy and not top_k, top_k=top_k)]
     seqs += [seqs[0].fork() for _ in range(B - 1)]
     inputs = [_inputs(wl, k, extra_prompt) for k in range(B)]
     orcs = [H.make_oracle(wl, tw, dw, max_seq, 1.0, greedy) for _ in range(B)]
@@ -33,7 +36,7 @@ def run_batch_lockstep(wl, B, gamma, n_blocks, greedy, logit_tol, std, extra_pro
         img, ids = inputs[k]
         if greedy:
             x0 = orcs[k].prefill(img, ids)
-            g0 = seqs[k].prefill(img, ids)
+            g0 = seqs[k].prefill(img, ids, u0=0.37 if top_k else None)
         else:
             probe = H.make_oracle(wl, tw, dw, max_seq, 1.0, greedy)
             probe.prefill(img, ids, u0=0.5)
@@ -51,7 +54,8 @@ def run_batch_lockstep(wl, B, gamma, n_blocks, greedy, logit_tol, std, extra_pro
         for k in range(B):
             d_ids, q = orcs[k].draft(gamma, None if greedy else su.draft_hook)
             d_all.append(d_ids); q_all.append(q); u_d.append(orcs[k].last_draft_u)
-        g_ids = bt.draft(gamma, None if greedy else np.stack(u_d))
+        any_u = synth.uniforms(8, f"batch.any.{blk}", (B, 2 * gamma + 1))     # top_k = 1: the values do not matter
+        g_ids = bt.draft(gamma, (any_u[:, :gamma].copy() if top_k else None) if greedy else np.stack(u_d))
         dl = bt.get_logits(2 * B).reshape(B, 2, V)[:, 1]          # last draft step's rows
         for k in range(B):
             derr = float(np.abs(dl[k] - orcs[k].last_draft_logits[gamma - 1]).max()) \
@@ -74,7 +78,7 @@ def run_batch_lockstep(wl, B, gamma, n_blocks, greedy, logit_tol, std, extra_pro
                         assert H.token_within_cdf_band(q_all[k][j], u_d[k][j], int(g_ids[k][j]), H.cdf_band(False, 2e-3))
             rep["tolerated"] += 1
         else:
-            ga, gn = bt.verify(gamma, None if greedy else np.stack(u_v))
+            ga, gn = bt.verify(gamma, (any_u[:, gamma:].copy() if top_k else None) if greedy else np.stack(u_v))
             lg = bt.get_logits(B * (gamma + 1)).reshape(B, gamma + 1, V)
             for k in range(B):
                 verr = float(np.abs(lg[k] - orcs[k].last_logits).max())
@@ -99,7 +103,8 @@ def run_batch_lockstep(wl, B, gamma, n_blocks, greedy, logit_tol, std, extra_pro
         for k in range(B):
             if not same[k] or not all(same):
                 img, _ = inputs[k]
-                seqs[k].prefill(img, np.asarray(orcs[k].seq[:-1], dtype=np.int32), u0=None if greedy else 0.5)
+                seqs[k].prefill(img, np.asarray(orcs[k].seq[:-1], dtype=np.int32),
+                                u0=0.5 if (top_k or not greedy) else None)
                 seqs[k].rollback(len(orcs[k].seq) - 1, orcs[k].seq[-2], orcs[k].seq[-1])
         rep["blocks"] += 1
     bt.close()
@@ -122,6 +127,18 @@ def test_three_ragged_sequences_small_bf16(greedy):
     assert r["blocks"] == 8
     if not greedy:
         assert sum(r["accepted"]) > 0 and len(set(r["accepted"])) > 1      # sequences advance at their own pace
+
+
+@pytest.mark.gpu
+def test_batched_sampling_kernels_with_top_k_one_reproduce_greedy():
+    """The probability-row path of the batched steps (softmax rows, truncation, per-sequence draw
+    and rule) with top_k = 1: the output must be the greedy one for any uniforms."""
+    t = synth.ModelCfg(2, 256, 4, 688, 1024, False, dtype="bf16")
+    d = synth.ModelCfg(1, 128, 2, 344, 1024, False, dtype="bf16")
+    wl = synth.Workload("tiny-bf16-batch", t, d, 16, 16, 4, 32)
+    r = run_batch_lockstep(wl, 3, 4, 6, True, 5e-2, 0.15, extra_prompt=5, top_k=1)
+    print("batch of 3, top_k = 1", r)
+    assert r["blocks"] == 6
 
 
 @pytest.mark.gpu

@@ -781,6 +781,16 @@ def test_llava7b_full_size_sampling_blocks_match_oracle():
 
 
 @pytest.mark.gpu
+def test_llava7b_full_size_top_k_top_p_blocks_match_oracle():
+    """Truncated sampling (top-k 50, top-p 0.9) at full depth against the oracle running the same
+    mode: 3 blocks with gamma = 5, 3, 7."""
+    wl = synth.llava7b_workload(gamma=5)
+    r = lockstep(wl, False, 1.0, 3, 5e-2, gammas=[5, 3, 7], top_k=50, top_p=0.9)
+    print("full-size top-k/top-p report", r)
+    assert r["blocks"] == 3 and r["max_logit_err"] < 4e-2
+
+
+@pytest.mark.gpu
 def test_llava7b_shaped_two_layer_with_draft_adapter():
     """The draft with an image adapter at LLaVA-7B shapes: 576 features of width 1024 projected
     by one linear layer to the draft's width and prepended to its input (bf16, tensor-core

@@ -137,6 +137,17 @@ def test_llava7b_shaped_two_layer_tree_lockstep():
 
 
 @pytest.mark.gpu
+def test_llava7b_full_size_tree_blocks_match_oracle():
+    """Tree blocks at full depth (32 target layers, 12 draft layers, 576 image rows + 64 prompt ids),
+    temperature 1: draft nodes, the target's logits for every node under the tree mask, accepted
+    paths and next tokens against the oracle for the shapes [2, 2], [3, 1] and [2, 1, 1]."""
+    wl = synth.llava7b_workload(gamma=5)
+    r = lockstep_tree(wl, False, [[2, 2], [3, 1], [2, 1, 1]], 3, 5e-2)
+    print("full-size tree", r)
+    assert r["blocks"] == 3 and r["max_logit_err"] < 4e-2
+
+
+@pytest.mark.gpu
 def test_chain_shaped_tree_equals_the_plain_block_on_the_device():
     """branching [1, 1, 1, 1] is a plain block of gamma = 4: spd_draft_tree / spd_verify_tree must
     return the ids, the accepted count and the next token of spd_draft / spd_verify, block after
