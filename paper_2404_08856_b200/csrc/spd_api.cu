@@ -744,11 +744,11 @@ spd_status prefill_tc(spd_ctx* ctx, ModelHost& mh, float* X, int R) {
     if ((s = tc_gemm(ctx, {pf.h_hi, d, R, 1, (size_t)d * 2, (size_t)R * d * 2}, {pf.h_lo, d, R, 1, (size_t)d * 2, (size_t)R * d * 2},
                      {w.wqkv, d, 3 * d, 1, (size_t)d * 2, (size_t)3 * d * d * 2}, a))) return s;
     rope_kv_kernel<<<592, 256, 0, cs>>>(pf.wide, R, d, dh, 0, mh.md.rope_cos, mh.md.rope_sin, pf.q_hi, pf.q_lo, kc, vc,
-                                        pf.vT, rp);
+                                        pf.vT, rp, (int)max_seq);
     a = TcArgs{}; a.M = R; a.N = R; a.K = dh; a.mode = TC_OUT_F32; a.alpha = mh.md.scale; a.out_f32 = pf.S; a.ldo = rp;
     a.out_batch = (long long)R * rp;
     if ((s = tc_gemm(ctx, {pf.q_hi, dh, R, H, (size_t)d * 2, (size_t)dh * 2}, {pf.q_lo, dh, R, H, (size_t)d * 2, (size_t)dh * 2},
-                     {kc, dh, R, H, (size_t)d * 2, (size_t)dh * 2}, a))) return s;
+                     {kc, dh, R, H, (size_t)dh * 2, max_seq * dh * 2}, a))) return s;   // a head's cached rows are contiguous
     softmax_causal_split_kernel<<<H * R, 256, 0, cs>>>(pf.S, R, rp, pf.p_hi, pf.p_lo);
     a = TcArgs{}; a.M = R; a.N = dh; a.K = rp; a.mode = TC_OUT_SPLIT; a.alpha = 1.f; a.out_hi = pf.h_hi; a.out_lo = pf.h_lo;
     a.ldo = d; a.out_batch = dh;

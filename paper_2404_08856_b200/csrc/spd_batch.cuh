@@ -65,12 +65,13 @@ __global__ void batch_rope_append_kernel(const float* qkv, int R, int M, int d, 
     float* q = md.qbuf + (size_t)m * d;
     q[c0] = qa * c - qb * s;
     q[c1] = qb * c + qa * s;
-    __nv_bfloat16* kc = static_cast<__nv_bfloat16*>(md.kcache) + ((size_t)layer * md.max_seq + pos) * d;
-    __nv_bfloat16* vc = static_cast<__nv_bfloat16*>(md.vcache) + ((size_t)layer * md.max_seq + pos) * d;
-    kc[c0] = __float2bfloat16_rn(ka * c - kb * s);
-    kc[c1] = __float2bfloat16_rn(kb * c + ka * s);
-    vc[c0] = __float2bfloat16_rn(row[2 * d + c0]);
-    vc[c1] = __float2bfloat16_rn(row[2 * d + c1]);
+    const size_t crow = (((size_t)layer * md.H + h) * md.max_seq + pos) * dh;   // cache: [L][H][max_seq][dh]
+    __nv_bfloat16* kc = static_cast<__nv_bfloat16*>(md.kcache) + crow;
+    __nv_bfloat16* vc = static_cast<__nv_bfloat16*>(md.vcache) + crow;
+    kc[jj] = __float2bfloat16_rn(ka * c - kb * s);
+    kc[jj + half] = __float2bfloat16_rn(kb * c + ka * s);
+    vc[jj] = __float2bfloat16_rn(row[2 * d + c0]);
+    vc[jj + half] = __float2bfloat16_rn(row[2 * d + c1]);
   }
 }
 

@@ -67,7 +67,7 @@ struct ModelDev {
   const void* lm_head;
   const float* final_norm;
   const float *rope_cos, *rope_sin;   // [max_seq][dh/2]
-  void *kcache, *vcache;              // [L][max_seq][d]
+  void *kcache, *vcache;              // [L][H][max_seq][dh]: a head's rows are contiguous (one stream per attention unit)
   float *x, *qbuf, *attn, *act;       // [8][d], [8][d], [8][d], [8][f]
   float *xg;                          // [8][d]: residual stream times the gain of the next RMSNorm
   float *ssq;                         // [grid][8]: per-CTA partial sums of x^2 of the residual stream rows
@@ -416,7 +416,7 @@ struct EpiArgs {
   float* qbuf; void* kc; void* vc;  // cache bases already offset to the layer
   const float *cs, *sn;
   const int *rowslot, *rowpos;      // per activation row: cache row to append to, rotary position (shared memory)
-  int d, dh;
+  int d, dh, max_seq;
 };
 
 __device__ __forceinline__ void cache_store(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
@@ -440,7 +440,8 @@ __device__ __forceinline__ void epilogue_pair(int epi, const EpiArgs& e, int m, 
     const int region = n / e.d, c = n - region * e.d;
     const int slot = e.rowslot[m];
     if (region == 2) {
-      WT* vp = static_cast<WT*>(e.vc) + (size_t)slot * e.d + c;
+      const int hv = c / e.dh;
+      WT* vp = static_cast<WT*>(e.vc) + ((size_t)hv * e.max_seq + slot) * e.dh + (c - hv * e.dh);
       cache_store(vp, a);
       cache_store(vp + 1, b);
     } else {
@@ -453,7 +454,7 @@ __device__ __forceinline__ void epilogue_pair(int epi, const EpiArgs& e, int m, 
         stcg(e.qbuf + (size_t)m * e.d + c0, ra);
         stcg(e.qbuf + (size_t)m * e.d + c0 + half, rb);
       } else {
-        WT* kp = static_cast<WT*>(e.kc) + (size_t)slot * e.d + c0;
+        WT* kp = static_cast<WT*>(e.kc) + ((size_t)h * e.max_seq + slot) * e.dh + i;
         cache_store(kp, ra);
         cache_store(kp + half, rb);
       }
@@ -866,7 +867,7 @@ __device__ void attn_phase(const ModelDev& md, int layer, int origin, int nslots
       const int n = min(SC, p1 - c0);
       for (int i = tid; i < n * cpr; i += CONSUMER_THREADS) {
         const int r = i / cpr, cc = i - r * cpr;
-        const size_t g = ((size_t)(c0 + r) * d + h * dh) * sizeof(CT) + (size_t)cc * 16;
+        const size_t g = (((size_t)h * md.max_seq + c0 + r) * dh) * sizeof(CT) + (size_t)cc * 16;
         cp_async16(Kt + (size_t)r * rowb + cc * 16, reinterpret_cast<const char*>(Kl) + g);
         cp_async16(Vt + (size_t)r * rowb + cc * 16, reinterpret_cast<const char*>(Vl) + g);
       }
@@ -1049,7 +1050,7 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int ns
       const int r = i / cpr, cc = i - r * cpr;
       const int dst = r * rowb + ((cc ^ (r & 7)) << 4);
       if (r < n) {
-        const size_t g = ((size_t)(c0 + r) * d + h * dh) * 2 + (size_t)cc * 16;
+        const size_t g = (((size_t)h * md.max_seq + c0 + r) * dh) * 2 + (size_t)cc * 16;
         cp_async16(Kt + dst, Kl + g);
         cp_async16(Vt + dst, Vl + g);
       } else {   // rows past the end must not hold NaN patterns: P is 0 there

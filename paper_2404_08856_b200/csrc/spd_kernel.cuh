@@ -205,7 +205,7 @@ __global__ void __launch_bounds__(ENGINE_THREADS, 1) forward_kernel(const __grid
         } else {
           const LayerDev& ly = layers[l];
           if (which == 0) {          // QKV + RoPE + KV append
-            e.qbuf = md.qbuf; e.d = d; e.dh = md.dh; e.rowslot = ctl->rowslot; e.rowpos = ctl->rowpos;
+            e.qbuf = md.qbuf; e.d = d; e.dh = md.dh; e.max_seq = md.max_seq; e.rowslot = ctl->rowslot; e.rowpos = ctl->rowpos;
             e.cs = md.rope_cos; e.sn = md.rope_sin;
             e.kc = static_cast<WT*>(md.kcache) + (size_t)l * md.max_seq * d;
             e.vc = static_cast<WT*>(md.vcache) + (size_t)l * md.max_seq * d;

@@ -293,10 +293,11 @@ __global__ void __launch_bounds__(256) rms_split_kernel(const float* x, const fl
 }
 
 // qkv fp32 [R][3d] (natural row order) -> rotary on q and k (pairs (i, i + dh/2)), q split into
-// hi/lo [R][d], k and v appended to the cache rows pos0.., v also transposed to vT [H][dh][rpad].
+// hi/lo [R][d], k and v appended to the cache rows pos0.. (cache of one layer: [H][max_seq][dh]),
+// v also transposed to vT [H][dh][rpad].
 __global__ void rope_kv_kernel(const float* qkv, int R, int d, int dh, int pos0, const float* cs, const float* sn,
                                __nv_bfloat16* q_hi, __nv_bfloat16* q_lo, __nv_bfloat16* kc, __nv_bfloat16* vc,
-                               __nv_bfloat16* vT, int rpad) {
+                               __nv_bfloat16* vT, int rpad, int max_seq) {
   const int half = dh >> 1, pairs = d >> 1;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < (size_t)R * pairs;
        i += (size_t)gridDim.x * blockDim.x) {
@@ -308,11 +309,12 @@ __global__ void rope_kv_kernel(const float* qkv, int R, int d, int dh, int pos0,
     const float qa = row[c0], qb = row[c1], ka = row[d + c0], kb = row[d + c1];
     store_split(q_hi, q_lo, (size_t)r * d + c0, qa * c - qb * s);
     store_split(q_hi, q_lo, (size_t)r * d + c1, qb * c + qa * s);
-    kc[(size_t)(pos0 + r) * d + c0] = __float2bfloat16_rn(ka * c - kb * s);
-    kc[(size_t)(pos0 + r) * d + c1] = __float2bfloat16_rn(kb * c + ka * s);
+    const size_t crow = ((size_t)h * max_seq + pos0 + r) * dh;
+    kc[crow + j] = __float2bfloat16_rn(ka * c - kb * s);
+    kc[crow + j + half] = __float2bfloat16_rn(kb * c + ka * s);
     const __nv_bfloat16 v0 = __float2bfloat16_rn(row[2 * d + c0]), v1 = __float2bfloat16_rn(row[2 * d + c1]);
-    vc[(size_t)(pos0 + r) * d + c0] = v0;
-    vc[(size_t)(pos0 + r) * d + c1] = v1;
+    vc[crow + j] = v0;
+    vc[crow + j + half] = v1;
     vT[((size_t)h * dh + j) * rpad + r] = v0;
     vT[((size_t)h * dh + j + half) * rpad + r] = v1;
   }

@@ -154,12 +154,18 @@ __global__ void tree_gather_kernel(const DevState* st, const ModelDev md, int po
   const int node = st->path[j - 1];
   if (node == j) return;                                // already in place
   const int origin = pos_base + st->n_text - (a + 1);
-  const size_t rowb = (size_t)md.d * esz;
-  char* cache = static_cast<char*>(kv ? md.vcache : md.kcache) + (size_t)l * md.max_seq * rowb;
+  const size_t rowb = (size_t)md.d * esz, headb = (size_t)md.dh * esz;      // a node's row = H pieces of dh
+  char* cache = static_cast<char*>(kv ? md.vcache : md.kcache) + (size_t)l * md.max_seq * rowb;   // [H][max_seq][dh]
   char* stg = staging + (((size_t)kv * md.L + l) * MAX_M + j) * rowb;
-  const uint4* src = reinterpret_cast<const uint4*>(scatter ? stg : cache + (size_t)(origin + node) * rowb);
-  uint4* dst = reinterpret_cast<uint4*>(scatter ? cache + (size_t)(origin + j) * rowb : stg);
-  for (int i = threadIdx.x; i < (int)(rowb >> 4); i += blockDim.x) dst[i] = src[i];
+  const int per_head = (int)(headb >> 4);
+  for (int i = threadIdx.x; i < (int)(rowb >> 4); i += blockDim.x) {
+    const int h = i / per_head, c = i - h * per_head;
+    uint4* in_stage = reinterpret_cast<uint4*>(stg + (size_t)h * headb) + c;
+    if (scatter)
+      reinterpret_cast<uint4*>(cache + ((size_t)h * md.max_seq + origin + j) * headb)[c] = *in_stage;
+    else
+      *in_stage = reinterpret_cast<const uint4*>(cache + ((size_t)h * md.max_seq + origin + node) * headb)[c];
+  }
 }
 
 }  // namespace spd
