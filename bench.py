@@ -39,7 +39,7 @@ import synth  # noqa: E402
 # algorithmic bytes (profiles/forward_kernel_verify_llava7b_2layer_ncu_full.md).  Weights dominate and grow
 # in proportion to the layer count, so the full launch's traffic is this ratio times its algorithmic
 # bytes.  Set to None when the kernel has changed since.
-VERIFY_TRAFFIC_RATIO = (1.092901e9 + 3.390720e6) / 1.093107712e9
+VERIFY_TRAFFIC_RATIO = (1.092909e9 + 3.516672e6) / 1.093107712e9
 GAMMA = 5   # block size of the benchmark's workload; --gamma overrides it for sweeps
 SAMPLING = False   # --sampling: temperature-1 rejection sampling instead of greedy acceptance
 DRAFT = "115m"   # "table1": the draft shape printed in the paper's Table 1 (informational run)
