@@ -621,12 +621,12 @@ EncodeTiledFn encode_tiled_fn() {
 
 // bf16 operand view [batch][rows][inner] with byte strides; box = 64 inner x 128 rows x 1.
 spd_status make_map(spd_ctx* ctx, CUtensorMap* m, const void* ptr, int inner, int rows, int batch, size_t row_stride,
-                    size_t batch_stride) {
+                    size_t batch_stride, int box_rows = TC_BM) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return fail(ctx, SPD_ECUDA, "cuTensorMapEncodeTiled not available");
   const cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)batch};
   const cuuint64_t strides[2] = {(cuuint64_t)row_stride, (cuuint64_t)batch_stride};
-  const cuuint32_t box[3] = {(cuuint32_t)TC_BK, (cuuint32_t)TC_BM, 1};
+  const cuuint32_t box[3] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -640,13 +640,16 @@ struct Operand { const void* ptr; int inner, rows, batch; size_t row_stride, bat
 // stream_ksplit = 0: the prefill form (3 stages, two CTAs per SM).  > 0: few rows against a large
 // weight matrix -- 6 stages, one CTA per SM, and the K loop cut into that many slices so that
 // enough CTAs stream; the slices' partial products go to `ws` and are summed in slice order.
+// `wide`: the streaming form with 256-row weight tiles (one activation tile per two weight tiles).
 spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const Operand& b, TcArgs args,
-                   bool gelu = false, int stream_ksplit = 0, float* ws = nullptr) {
+                   bool gelu = false, int stream_ksplit = 0, float* ws = nullptr, bool wide = false,
+                   bool leave_slices = false) {
   CUtensorMap ma, ml, mb;
   spd_status s;
   if ((s = make_map(ctx, &ma, a_hi.ptr, a_hi.inner, a_hi.rows, a_hi.batch, a_hi.row_stride, a_hi.batch_stride))) return s;
   if ((s = make_map(ctx, &ml, a_lo.ptr, a_lo.inner, a_lo.rows, a_lo.batch, a_lo.row_stride, a_lo.batch_stride))) return s;
-  if ((s = make_map(ctx, &mb, b.ptr, b.inner, b.rows, b.batch, b.row_stride, b.batch_stride))) return s;
+  if ((s = make_map(ctx, &mb, b.ptr, b.inner, b.rows, b.batch, b.row_stride, b.batch_stride,
+                    wide && stream_ksplit > 0 ? TC_BN_WIDE : TC_BN))) return s;
   static bool attr_set[MAX_DEV];
   if (ctx->device < 0 || ctx->device >= MAX_DEV) return fail(ctx, SPD_ECUDA, "device index out of range");
   if (!attr_set[ctx->device]) {
@@ -654,6 +657,8 @@ spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const
     CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel<true, TC_STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
     CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel<false, TC_STAGES_STREAM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                             tc_smem_bytes(TC_STAGES_STREAM)));
+    CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel<false, TC_STAGES_WIDE, TC_BN_WIDE>,
+                            cudaFuncAttributeMaxDynamicSharedMemorySize, tc_smem_bytes(TC_STAGES_WIDE, TC_BN_WIDE)));
     attr_set[ctx->device] = true;
   }
   args.split = 1;
@@ -668,9 +673,13 @@ spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const
       if (!ws || ldo != args.N) return fail(ctx, SPD_EINVAL, "split GEMM needs a workspace and a dense output");
       args.ksplit = stream_ksplit; args.out_f32 = ws; args.mode = TC_OUT_F32;
     }
-    dim3 grid((args.N + TC_BN - 1) / TC_BN, (args.M + TC_BM - 1) / TC_BM, stream_ksplit);
-    tc_gemm_kernel<false, TC_STAGES_STREAM><<<grid, 128, tc_smem_bytes(TC_STAGES_STREAM), ctx->stream>>>(ma, ml, mb, args);
-    if (stream_ksplit > 1)
+    const int bn = wide ? TC_BN_WIDE : TC_BN;
+    dim3 grid((args.N + bn - 1) / bn, (args.M + TC_BM - 1) / TC_BM, stream_ksplit);
+    if (wide)
+      tc_gemm_kernel<false, TC_STAGES_WIDE, TC_BN_WIDE><<<grid, 128, tc_smem_bytes(TC_STAGES_WIDE, TC_BN_WIDE), ctx->stream>>>(ma, ml, mb, args);
+    else
+      tc_gemm_kernel<false, TC_STAGES_STREAM><<<grid, 128, tc_smem_bytes(TC_STAGES_STREAM), ctx->stream>>>(ma, ml, mb, args);
+    if (stream_ksplit > 1 && !leave_slices)   // (leave_slices: the caller's next kernel adds them up)
       tc_reduce_kernel<<<148, 256, 0, ctx->stream>>>(ws, stream_ksplit, (size_t)args.M * args.N, dest, mode == TC_OUT_F32_ADD);
     CU(cudaGetLastError());
     return SPD_OK;
@@ -1421,7 +1430,7 @@ spd_status balloc(spd_batch* bt, T** p, size_t n) {
   return SPD_OK;
 }
 
-constexpr int BATCH_ATTN_SCRATCH = 200 * 1024;
+constexpr int BATCH_ATTN_SCRATCH = 100 * 1024;   // two CTAs per SM: 16 warps hide each other's dependency stalls
 constexpr int BATCH_KSPLIT_MAX = 8;
 
 template <int M>
@@ -1433,7 +1442,7 @@ spd_status launch_batch_attn(spd_ctx* ctx, const ModelDev* mds, const int* origi
     CU(cudaFuncSetAttribute((const void*)batch_attn_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     attr[ctx->device] = true;
   }
-  batch_attn_kernel<M><<<ctx->n_sm, CONSUMER_THREADS, smem, ctx->stream>>>(mds, origins, B, layer, chain0,
+  batch_attn_kernel<M><<<2 * ctx->n_sm, CONSUMER_THREADS, smem, ctx->stream>>>(mds, origins, B, layer, chain0,
                                                                           BATCH_ATTN_SCRATCH, max_split);
   CU(cudaGetLastError());
   return SPD_OK;
@@ -1477,37 +1486,55 @@ spd_status batch_forward(spd_batch* bt, bool draft, int M, int j) {
   if (attn_split > mh.md.nsplit) attn_split = mh.md.nsplit;
   if (attn_split < 1) attn_split = 1;
   // every GEMM here is a few rows against a large weight matrix: cut K so that about one CTA per SM streams
-  auto ksplit = [&](int N, int K) {
-    const int tiles = (N + TC_BN - 1) / TC_BN, kb = (K + TC_BK - 1) / TC_BK;
-    int sp = (ctx->n_sm + tiles - 1) / tiles;
+  // K slices: up to one CTA per SM, never a second wave, at least 8 K blocks per slice.  256-row weight
+  // tiles (half the activation re-reads of 128-row ones) wherever they still give half the SMs a CTA.
+  auto slices = [&](int N, int K, int bn) {
+    const int tiles = (N + bn - 1) / bn, kb = (K + TC_BK - 1) / TC_BK;
+    int sp = ctx->n_sm / tiles;
     if (sp > BATCH_KSPLIT_MAX) sp = BATCH_KSPLIT_MAX;
-    if (sp > kb / 8) sp = kb / 8 > 0 ? kb / 8 : 1;       // at least 8 K blocks per slice
+    if (sp > kb / 8) sp = kb / 8;
     return sp < 1 ? 1 : sp;
   };
+  auto wide = [&](int N, int K) {
+    return ((N + TC_BN_WIDE - 1) / TC_BN_WIDE) * slices(N, K, TC_BN_WIDE) * 2 >= ctx->n_sm;
+  };
+  auto ksplit = [&](int N, int K) { return slices(N, K, wide(N, K) ? TC_BN_WIDE : TC_BN); };
+  // Where a projection is cut into K slices, the kernel that reads its result adds the slices up
+  // (in slice order): the rotary / cache-append kernel for QKV, the fused residual + RMSNorm + split
+  // kernel for the output and down projections.
+  const size_t xs = (size_t)R * d;
+  rms_split_kernel<<<R, 256, 0, cs>>>(X, mh.rm[0].attn_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
   for (int l = 0; l < L; ++l) {
     const ModelHost::RowMajor& w = mh.rm[l];
     TcArgs a{};
-    rms_split_kernel<<<R, 256, 0, cs>>>(X, w.attn_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
     a = TcArgs{}; a.M = R; a.N = 3 * d; a.K = d; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = pf.wide; a.ldo = 3 * d;
-    if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wqkv, d, 3 * d, 1, (size_t)d * 2, (size_t)3 * d * d * 2}, a, false,
-                     ksplit(3 * d, d), bt->gemm_ws))) return s;
-    batch_rope_append_kernel<<<296, 256, 0, cs>>>(pf.wide, R, M, d, dh, bt->rowslot, mh.md.rope_cos, mh.md.rope_sin, mds, l);
+    const int sq = ksplit(3 * d, d);
+    if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wqkv, d, 3 * d, 1, (size_t)d * 2, (size_t)3 * d * d * 2}, a, false, sq, bt->gemm_ws,
+                     wide(3 * d, d), true))) return s;
+    batch_rope_append_kernel<<<1184, 256, 0, cs>>>(sq > 1 ? bt->gemm_ws : pf.wide, sq, R, M, d, dh, bt->rowslot,
+                                                 mh.md.rope_cos, mh.md.rope_sin, mds, l);
     if ((s = batch_attn(ctx, M, mds, bt->origins, B, l, draft ? j - 1 : 0, attn_split))) return s;
     batch_gather_split_kernel<<<296, 256, 0, cs>>>(mds, R, M, d, pf.h_hi, pf.h_lo);
     a = TcArgs{}; a.M = R; a.N = d; a.K = d; a.mode = TC_OUT_F32_ADD; a.alpha = 1.f; a.out_f32 = X; a.ldo = d;
-    if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wo, d, d, 1, (size_t)d * 2, (size_t)d * d * 2}, a, false, ksplit(d, d), bt->gemm_ws))) return s;
-    rms_split_kernel<<<R, 256, 0, cs>>>(X, w.ffn_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
+    const int so = ksplit(d, d);
+    if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wo, d, d, 1, (size_t)d * 2, (size_t)d * d * 2}, a, false, so, bt->gemm_ws, wide(d, d),
+                     true))) return s;
+    resid_rms_split_kernel<<<R, 256, 0, cs>>>(X, bt->gemm_ws, so > 1 ? so : 0, xs, w.ffn_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
     a = TcArgs{}; a.M = R; a.N = 2 * f; a.K = d; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = pf.wide; a.ldo = 2 * f;
     if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wgu, d, 2 * f, 1, (size_t)d * 2, (size_t)2 * f * d * 2}, a, false,
-                     ksplit(2 * f, d), bt->gemm_ws))) return s;
+                     ksplit(2 * f, d), bt->gemm_ws, wide(2 * f, d)))) return s;
     swiglu_split_kernel<<<296, 256, 0, cs>>>(pf.wide, R, f, pf.h_hi, pf.h_lo);
     a = TcArgs{}; a.M = R; a.N = d; a.K = f; a.mode = TC_OUT_F32_ADD; a.alpha = 1.f; a.out_f32 = X; a.ldo = d;
+    const int sd = ksplit(d, f);
     if ((s = tc_gemm(ctx, {pf.h_hi, f, R, 1, (size_t)f * 2, (size_t)R * f * 2}, {pf.h_lo, f, R, 1, (size_t)f * 2, (size_t)R * f * 2},
-                     {w.wd, f, d, 1, (size_t)f * 2, (size_t)d * f * 2}, a, false, ksplit(d, f), bt->gemm_ws))) return s;
+                     {w.wd, f, d, 1, (size_t)f * 2, (size_t)d * f * 2}, a, false, sd, bt->gemm_ws, wide(d, f), true))) return s;
+    // the norm in front of the next layer (or of the LM head) rides on the residual update
+    resid_rms_split_kernel<<<R, 256, 0, cs>>>(X, bt->gemm_ws, sd > 1 ? sd : 0, xs,
+                                              l + 1 < L ? mh.rm[l + 1].attn_norm : mh.md.final_norm, mh.cfg.rms_eps, d,
+                                              pf.h_hi, pf.h_lo);
   }
-  rms_split_kernel<<<R, 256, 0, cs>>>(X, mh.md.final_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
   TcArgs a{}; a.M = R; a.N = V; a.K = d; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = bt->logits; a.ldo = V;
-  if ((s = tc_gemm(ctx, h_hi, h_lo, {mh.lm_rm, d, V, 1, (size_t)d * 2, (size_t)V * d * 2}, a, false, ksplit(V, d), bt->gemm_ws))) return s;
+  if ((s = tc_gemm(ctx, h_hi, h_lo, {mh.lm_rm, d, V, 1, (size_t)d * 2, (size_t)V * d * 2}, a, false, ksplit(V, d), bt->gemm_ws, wide(V, d)))) return s;
   CU(cudaGetLastError());
   bt->last_rows = R;
   return SPD_OK;

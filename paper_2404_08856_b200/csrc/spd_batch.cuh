@@ -48,8 +48,16 @@ __global__ void batch_embed_kernel(const BatchSeq* seqs, int B, int M, int draft
 // qkv fp32 [R][3d] (natural row order) -> rotary embedding on q and k at each row's own position
 // (pairs (i, i + dh/2)); q goes to its sequence's query rows [M][d] (fp32), k and v are appended
 // to its sequence's cache at the row's cache row.
-__global__ void batch_rope_append_kernel(const float* qkv, int R, int M, int d, int dh, const int* rowslot,
+// `qkv` may be the sum of `slices` partial products [slices][R][3d] (K slices of the projection, added in
+// slice order as tc_reduce_kernel does).
+__global__ void batch_rope_append_kernel(const float* qkv, int slices, int R, int M, int d, int dh, const int* rowslot,
                                          const float* cs, const float* sn, const ModelDev* mds, int layer) {
+  const size_t sstride = (size_t)R * 3 * d;
+  auto at = [&](const float* p) {
+    float v = 0.f;
+    for (int s = 0; s < slices; ++s) v += p[(size_t)s * sstride];
+    return v;
+  };
   const int half = dh >> 1, pairs = d >> 1;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < (size_t)R * pairs;
        i += (size_t)gridDim.x * blockDim.x) {
@@ -60,7 +68,7 @@ __global__ void batch_rope_append_kernel(const float* qkv, int R, int M, int d, 
     const int pos = rowslot[r];
     const float* row = qkv + (size_t)r * 3 * d;
     const float c = cs[(size_t)pos * half + jj], s = sn[(size_t)pos * half + jj];
-    const float qa = row[c0], qb = row[c1], ka = row[d + c0], kb = row[d + c1];
+    const float qa = at(row + c0), qb = at(row + c1), ka = at(row + d + c0), kb = at(row + d + c1);
     const ModelDev& md = mds[b];
     float* q = md.qbuf + (size_t)m * d;
     q[c0] = qa * c - qb * s;
@@ -70,8 +78,8 @@ __global__ void batch_rope_append_kernel(const float* qkv, int R, int M, int d, 
     __nv_bfloat16* vc = static_cast<__nv_bfloat16*>(md.vcache) + crow;
     kc[jj] = __float2bfloat16_rn(ka * c - kb * s);
     kc[jj + half] = __float2bfloat16_rn(kb * c + ka * s);
-    vc[jj] = __float2bfloat16_rn(row[2 * d + c0]);
-    vc[jj + half] = __float2bfloat16_rn(row[2 * d + c1]);
+    vc[jj] = __float2bfloat16_rn(at(row + 2 * d + c0));
+    vc[jj + half] = __float2bfloat16_rn(at(row + 2 * d + c1));
   }
 }
 
@@ -84,7 +92,7 @@ __global__ void batch_rope_append_kernel(const float* qkv, int R, int M, int d, 
 // `max_split`: KV splits per head at most -- with B sequences there are enough (sequence, head) pairs
 // to fill the grid, so heads are cut no further than needed (fewer partial results to merge).
 template <int M>
-__global__ void __launch_bounds__(CONSUMER_THREADS) batch_attn_kernel(const ModelDev* mds, const int* origins, int B,
+__global__ void __launch_bounds__(CONSUMER_THREADS, 2) batch_attn_kernel(const ModelDev* mds, const int* origins, int B,
                                                                       int layer, int chain0, int xbytes, int max_split) {
   extern __shared__ __align__(1024) char bsm[];
   Ctrl* ctl = reinterpret_cast<Ctrl*>(bsm);

@@ -22,9 +22,11 @@ constexpr int TC_STAGES = 2;          // prefill (compute-bound, many tiles): 2 
 constexpr int TC_STAGES_STREAM = 4;   // few rows against large weights (HBM-bound): 4 stages, one CTA per SM
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2, TC_B_BYTES = TC_BN * TC_BK * 2;
 constexpr int TC_STAGE_BYTES = 2 * TC_A_BYTES + TC_B_BYTES;              // A hi | A lo | B = 48 KB
-__host__ __device__ constexpr int tc_smem_bytes(int stages) { return stages * TC_STAGE_BYTES + 1024 + 256; }   // + alignment slack + barriers
+__host__ __device__ constexpr int tc_stage_bytes(int bn) { return 2 * TC_A_BYTES + bn * TC_BK * 2; }          // A hi | A lo | B (bn rows)
+__host__ __device__ constexpr int tc_smem_bytes(int stages, int bn = TC_BN) { return stages * tc_stage_bytes(bn) + 1024 + 256; }   // + alignment slack + barriers
+constexpr int TC_BN_WIDE = 256;       // streaming form: two weight tiles per activation tile (half the activation re-reads)
+constexpr int TC_STAGES_WIDE = 3;     // 3 x 64 KB
 constexpr int TC_SMEM_BYTES = tc_smem_bytes(TC_STAGES);
-constexpr int TC_TMEM_COLS = 128;
 
 enum : int { TC_OUT_F32 = 0, TC_OUT_F32_ADD = 1, TC_OUT_SPLIT = 2 };
 
@@ -53,15 +55,17 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, i
 __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
   return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
-// kind::f16: D = fp32, A = B = bf16, both K-major, M = 128, N = 128.
-constexpr uint32_t TC_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TC_BN >> 3) << 17) |
-                              ((uint32_t)(TC_BM >> 4) << 24);
+// kind::f16: D = fp32, A = B = bf16, both K-major, M = 128, N = bn.
+__host__ __device__ constexpr uint32_t tc_idesc(int bn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+}
 
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(TC_IDESC), "r"(accumulate)
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
@@ -89,13 +93,14 @@ __device__ __forceinline__ float gelu_exact(float x) { return 0.5f * x * (1.0f +
 // grid = (N tiles, M tiles, batch); 128 threads: thread 0 feeds TMA, thread 32 issues the MMAs,
 // all four warps read the accumulator back (warp w owns TMEM lanes 32w..32w+31 = tile rows).
 // GELU: the hi/lo output (TC_OUT_SPLIT) is gelu(alpha * accumulator) instead of alpha * accumulator.
-template <bool GELU, int STAGES>
-__global__ void __launch_bounds__(128, STAGES <= 3 ? 2 : 1)
+template <bool GELU, int STAGES, int BN = TC_BN>
+__global__ void __launch_bounds__(128, (STAGES <= 3 && BN == TC_BN) ? 2 : 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
                const __grid_constant__ CUtensorMap map_b, const TcArgs a) {
+  constexpr int STAGE_B = tc_stage_bytes(BN);     // bytes of one ring stage
   extern __shared__ uint8_t tc_smem_raw[];
   uint8_t* stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full = reinterpret_cast<uint64_t*>(stages + STAGES * TC_STAGE_BYTES);
+  uint64_t* full = reinterpret_cast<uint64_t*>(stages + STAGES * STAGE_B);
   uint64_t* empty = full + STAGES;
   uint64_t* accum = empty + STAGES;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
@@ -112,7 +117,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(TC_TMEM_COLS)
+                 "r"(BN)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -132,11 +137,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
       const int s = it % STAGES;
       const unsigned ph = (it / STAGES) & 1;
       if (!mbar_wait(&empty[s], ph ^ 1u, err, DEV_TIMEOUT_EMPTY)) break;
-      mbar_arrive_expect_tx(&full[s], TC_STAGE_BYTES);
+      mbar_arrive_expect_tx(&full[s], STAGE_B);
       const int kb = k_first + it;
-      tma_load_3d(stages + s * TC_STAGE_BYTES, &map_a_hi, kb * TC_BK, tile_m * TC_BM, z, &full[s]);
-      tma_load_3d(stages + s * TC_STAGE_BYTES + TC_A_BYTES, &map_a_lo, kb * TC_BK, tile_m * TC_BM, z, &full[s]);
-      tma_load_3d(stages + s * TC_STAGE_BYTES + 2 * TC_A_BYTES, &map_b, kb * TC_BK, tile_n * TC_BN, z, &full[s]);
+      tma_load_3d(stages + s * STAGE_B, &map_a_hi, kb * TC_BK, tile_m * TC_BM, z, &full[s]);
+      tma_load_3d(stages + s * STAGE_B + TC_A_BYTES, &map_a_lo, kb * TC_BK, tile_m * TC_BM, z, &full[s]);
+      tma_load_3d(stages + s * STAGE_B + 2 * TC_A_BYTES, &map_b, kb * TC_BK, tile_n * BN, z, &full[s]);
     }
   } else if (tid == 32) {
     // ---- MMA issuer
@@ -147,13 +152,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
       ok = mbar_wait(&full[s], ph, err, DEV_TIMEOUT_FULL);
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint64_t ah = umma_desc(smem_u32(stages + s * TC_STAGE_BYTES));
-      const uint64_t al = umma_desc(smem_u32(stages + s * TC_STAGE_BYTES + TC_A_BYTES));
-      const uint64_t bd = umma_desc(smem_u32(stages + s * TC_STAGE_BYTES + 2 * TC_A_BYTES));
+      const uint64_t ah = umma_desc(smem_u32(stages + s * STAGE_B));
+      const uint64_t al = umma_desc(smem_u32(stages + s * STAGE_B + TC_A_BYTES));
+      const uint64_t bd = umma_desc(smem_u32(stages + s * STAGE_B + 2 * TC_A_BYTES));
 #pragma unroll
       for (int k = 0; k < TC_BK / 16; ++k) {   // 32 bytes further along K inside the swizzle atom
-        umma_bf16(tmem_base, ah + 2 * k, bd + 2 * k, (it > 0 || k > 0) ? 1u : 0u);
-        umma_bf16(tmem_base, al + 2 * k, bd + 2 * k, 1u);
+        umma_bf16(tmem_base, ah + 2 * k, bd + 2 * k, tc_idesc(BN), (it > 0 || k > 0) ? 1u : 0u);
+        umma_bf16(tmem_base, al + 2 * k, bd + 2 * k, tc_idesc(BN), 1u);
       }
       umma_commit(&empty[s]);   // the stage is free once these MMAs have read it
     }
@@ -167,7 +172,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
   const int row = tile_m * TC_BM + warp * 32 + lane;
   if (done) {
 #pragma unroll 1
-    for (int c0 = 0; c0 < TC_BN; c0 += 32) {
+    for (int c0 = 0; c0 < BN; c0 += 32) {
       uint32_t v[32];
       if (total == 0) {
 #pragma unroll
@@ -175,7 +180,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
       } else {
         tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
       }
-      const int col0 = tile_n * TC_BN + c0;
+      const int col0 = tile_n * BN + c0;
       if (row < a.M && col0 < a.N) {
         const long long off = (long long)z * a.out_batch + (long long)slice * a.M * a.ldo + (long long)row * a.ldo + col0;
         const int nv = min(32, a.N - col0);
@@ -243,7 +248,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
   __syncthreads();
   if (warp == 0) {
     if (!done) for (int i = 0; i < 200; ++i) __nanosleep(1000);   // let copies in flight land
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
   }
 }
 
@@ -290,6 +295,58 @@ __global__ void __launch_bounds__(256) rms_split_kernel(const float* x, const fl
   const float inv = 1.0f / sqrtf(tot / (float)d + eps);
   for (int k = threadIdx.x; k < d; k += 256)
     store_split(hi, lo, (size_t)blockIdx.x * d + k, (row[k] * inv) * gain[k]);
+}
+
+// x[row] += sum over the K slices of a projection's partial products (slice order, as
+// tc_reduce_kernel adds them), then the RMSNorm of the updated row with `gain`, split into hi/lo
+// bf16: one launch instead of the slice sum and the norm.  slices = 0: the residual is already in x.
+__global__ void __launch_bounds__(256) resid_rms_split_kernel(float* x, const float* part, int slices, size_t slice_stride,
+                                                              const float* gain, float eps, int d, __nv_bfloat16* hi,
+                                                              __nv_bfloat16* lo) {
+  __shared__ float red[8];
+  constexpr int PER = 4096 / 4 / 256;     // float4 per thread: rows of up to 4096 columns stay in registers
+  float* row = x + (size_t)blockIdx.x * d;
+  const float* prow = part + (size_t)blockIdx.x * d;
+  const int d4 = d >> 2;
+  float4 v[PER];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < PER; ++i) {
+    const int k4 = threadIdx.x + i * 256;
+    v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (k4 < d4) {
+      v[i] = reinterpret_cast<const float4*>(row)[k4];
+      float4 p[8];   // all slices of this piece travel together, then they are added in slice order
+#pragma unroll
+      for (int s = 0; s < 8; ++s)
+        if (s < slices) p[s] = reinterpret_cast<const float4*>(prow + (size_t)s * slice_stride)[k4];
+#pragma unroll
+      for (int s = 0; s < 8; ++s)
+        if (s < slices) { v[i].x += p[s].x; v[i].y += p[s].y; v[i].z += p[s].z; v[i].w += p[s].w; }
+      if (slices > 0) reinterpret_cast<float4*>(row)[k4] = v[i];
+      ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) tot += red[w];
+  const float inv = 1.0f / sqrtf(tot / (float)d + eps);
+#pragma unroll
+  for (int i = 0; i < PER; ++i) {
+    const int k4 = threadIdx.x + i * 256;
+    if (k4 < d4) {
+      const float4 g = reinterpret_cast<const float4*>(gain)[k4];
+      const size_t o = (size_t)blockIdx.x * d + (size_t)k4 * 4;
+      store_split(hi, lo, o, (v[i].x * inv) * g.x);
+      store_split(hi, lo, o + 1, (v[i].y * inv) * g.y);
+      store_split(hi, lo, o + 2, (v[i].z * inv) * g.z);
+      store_split(hi, lo, o + 3, (v[i].w * inv) * g.w);
+    }
+  }
 }
 
 // qkv fp32 [R][3d] (natural row order) -> rotary on q and k (pairs (i, i + dh/2)), q split into
