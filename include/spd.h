@@ -120,7 +120,7 @@ typedef struct {
 
 /* Validates cfg, copies and repacks the weights, allocates KV caches and workspaces,
  * builds the rotary table.  Shapes must satisfy: d_model <= 4096 and a multiple of 32,
- * d_head = d_model / n_heads in {32, 64, 128}, d_ffn a multiple of 8, gamma_max <= 7, max_seq >= 16,
+ * d_head = d_model / n_heads in {32, 64, 128} (bf16 models: 64 or 128), d_ffn a multiple of 8, gamma_max <= 7, max_seq >= 16,
  * equal vocab for both models.  *out is NULL on failure. */
 spd_status spd_create(const spd_weights* target_w, const spd_weights* draft_w,
                       const spd_cfg* cfg, spd_ctx** out);

@@ -214,6 +214,9 @@ spd_status check_model(spd_ctx* ctx, const spd_model_cfg& c, const char* who) {
   if (c.d_model % c.n_heads) return bad("d_model not divisible by n_heads");
   const int dh = c.d_model / c.n_heads;
   if (dh != 32 && dh != 64 && dh != 128) return bad("d_head must be 32, 64 or 128");
+  // the tensor-core attention tiles swizzle the eight 16-byte pieces of a 128-byte row segment: a
+  // bf16 row needs at least eight pieces
+  if (c.dtype == 1 && dh == 32) return bad("bf16 models need d_head 64 or 128");
   if (c.d_model > KC_MAX) return bad("d_model > 4096 not supported");
   if (c.d_model % 32 || c.d_ffn % 8) return bad("d_model must be a multiple of 32 and d_ffn of 8");
   if (c.dtype != 0 && c.dtype != 1) return bad("dtype must be 0 (fp32) or 1 (bf16)");

@@ -623,6 +623,12 @@ def test_state_and_overflow_errors():
     bad = synth.ModelCfg(2, 100, 3, 64, 64, dtype="fp32")   # d_model not divisible by heads
     with pytest.raises(spd.SpdError):
         H.make_gpu(synth.Workload("bad", bad, bad, 0, 4, 1, 4), tw, tw, 48)
+    # bf16 with d_head 32: the tensor-core attention tiles need rows of at least 128 bytes
+    narrow = synth.ModelCfg(1, 128, 4, 344, 1024, False, dtype="bf16")
+    nw = synth.Weights(narrow, 3, "narrow")
+    with pytest.raises(spd.SpdError) as e:
+        H.make_gpu(synth.Workload("narrow", narrow, narrow, 0, 4, 1, 4), nw, nw, 48)
+    assert e.value.status == spd.SPD_EINVAL
 
 
 @pytest.mark.gpu
