@@ -76,6 +76,7 @@ struct spd_ctx {
     size_t cap_rows = 0;
     __nv_bfloat16 *h_hi = nullptr, *h_lo = nullptr, *q_hi = nullptr, *q_lo = nullptr, *vT = nullptr;
     __nv_bfloat16 *p_hi = nullptr, *p_lo = nullptr;
+    __nv_bfloat16 *g_hi = nullptr, *g_lo = nullptr;   // silu(gate) * up [rows][d_ffn]
     float *wide = nullptr, *S = nullptr;
   } pf;
   // scratch of spd_image_adapter, grown on demand
@@ -345,8 +346,9 @@ spd_status build_model(spd_ctx* ctx, ModelHost& mh, const spd_model_cfg& c, cons
       CU(cudaMemcpyAsync(r.wqkv + (size_t)d * d, w->wk[l], (size_t)d * d * 2, cudaMemcpyDefault, ctx->stream));
       CU(cudaMemcpyAsync(r.wqkv + (size_t)2 * d * d, w->wv[l], (size_t)d * d * 2, cudaMemcpyDefault, ctx->stream));
       CU(cudaMemcpyAsync(r.wo, w->wo[l], (size_t)d * d * 2, cudaMemcpyDefault, ctx->stream));
-      CU(cudaMemcpyAsync(r.wgu, w->w_gate[l], (size_t)f * d * 2, cudaMemcpyDefault, ctx->stream));
-      CU(cudaMemcpyAsync(r.wgu + (size_t)f * d, w->w_up[l], (size_t)f * d * 2, cudaMemcpyDefault, ctx->stream));
+      // gate and up rows interleaved (gate_0, up_0, gate_1, ...): the GEMM's epilogue pairs them
+      if ((s = put_rows(ctx, r.wgu, w->w_gate[l], staging, f, d, esz, 2, 0, 0))) return s;
+      if ((s = put_rows(ctx, r.wgu, w->w_up[l], staging, f, d, esz, 2, 1, 0))) return s;
       CU(cudaMemcpyAsync(r.wd, w->w_down[l], (size_t)d * f * 2, cudaMemcpyDefault, ctx->stream));
       CU(cudaStreamSynchronize(ctx->stream));
       r.attn_norm = an; r.ffn_norm = fnw;
@@ -668,7 +670,8 @@ spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const
   args.err = &ctx->st->err;
   args.ksplit = 1;
   if (stream_ksplit > 0) {
-    if (gelu || a_hi.batch != 1 || args.mode == TC_OUT_SPLIT) return fail(ctx, SPD_EINVAL, "streaming GEMM: plain fp32 output only");
+    if (gelu || a_hi.batch != 1 || args.mode == TC_OUT_SPLIT || (args.mode == TC_OUT_SWIGLU && stream_ksplit > 1))
+      return fail(ctx, SPD_EINVAL, "streaming GEMM: fp32 output, or the SwiGLU epilogue on an unsliced K");
     const int mode = args.mode;
     float* dest = args.out_f32;
     const long long ldo = args.ldo;
@@ -730,6 +733,8 @@ spd_status prefill_scratch(spd_ctx* ctx, int R) {
   if ((s = dalloc(ctx, &ctx->pf.S, hm * rp * rp))) return s;
   if ((s = dalloc(ctx, &ctx->pf.p_hi, hm * rp * rp))) return s;
   if ((s = dalloc(ctx, &ctx->pf.p_lo, hm * rp * rp))) return s;
+  if ((s = dalloc(ctx, &ctx->pf.g_hi, rp * fm))) return s;
+  if ((s = dalloc(ctx, &ctx->pf.g_lo, rp * fm))) return s;
   ctx->pf.cap_rows = rp;
   return SPD_OK;
 }
@@ -771,12 +776,12 @@ spd_status prefill_tc(spd_ctx* ctx, ModelHost& mh, float* X, int R) {
                      {w.wo, d, d, 1, (size_t)d * 2, (size_t)d * d * 2}, a))) return s;
     // feed-forward block
     rms_split_kernel<<<R, 256, 0, cs>>>(X, w.ffn_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
-    a = TcArgs{}; a.M = R; a.N = 2 * f; a.K = d; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = pf.wide; a.ldo = 2 * f;
+    // gate/up with SwiGLU in the epilogue (interleaved gate/up rows): hi/lo [R][f] straight out of the GEMM
+    a = TcArgs{}; a.M = R; a.N = 2 * f; a.K = d; a.mode = TC_OUT_SWIGLU; a.alpha = 1.f; a.out_hi = pf.g_hi; a.out_lo = pf.g_lo; a.ldo = f;
     if ((s = tc_gemm(ctx, {pf.h_hi, d, R, 1, (size_t)d * 2, (size_t)R * d * 2}, {pf.h_lo, d, R, 1, (size_t)d * 2, (size_t)R * d * 2},
                      {w.wgu, d, 2 * f, 1, (size_t)d * 2, (size_t)2 * f * d * 2}, a))) return s;
-    swiglu_split_kernel<<<592, 256, 0, cs>>>(pf.wide, R, f, pf.h_hi, pf.h_lo);
     a = TcArgs{}; a.M = R; a.N = d; a.K = f; a.mode = TC_OUT_F32_ADD; a.alpha = 1.f; a.out_f32 = X; a.ldo = d;
-    if ((s = tc_gemm(ctx, {pf.h_hi, f, R, 1, (size_t)f * 2, (size_t)R * f * 2}, {pf.h_lo, f, R, 1, (size_t)f * 2, (size_t)R * f * 2},
+    if ((s = tc_gemm(ctx, {pf.g_hi, f, R, 1, (size_t)f * 2, (size_t)R * f * 2}, {pf.g_lo, f, R, 1, (size_t)f * 2, (size_t)R * f * 2},
                      {w.wd, f, d, 1, (size_t)f * 2, (size_t)d * f * 2}, a))) return s;
     CU(cudaGetLastError());
   }
@@ -1523,13 +1528,20 @@ spd_status batch_forward(spd_batch* bt, bool draft, int M, int j) {
     if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wo, d, d, 1, (size_t)d * 2, (size_t)d * d * 2}, a, false, so, bt->gemm_ws, wide(d, d),
                      true))) return s;
     resid_rms_split_kernel<<<R, 256, 0, cs>>>(X, bt->gemm_ws, so > 1 ? so : 0, xs, w.ffn_norm, mh.cfg.rms_eps, d, pf.h_hi, pf.h_lo);
-    a = TcArgs{}; a.M = R; a.N = 2 * f; a.K = d; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = pf.wide; a.ldo = 2 * f;
-    if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wgu, d, 2 * f, 1, (size_t)d * 2, (size_t)2 * f * d * 2}, a, false,
-                     ksplit(2 * f, d), bt->gemm_ws, wide(2 * f, d)))) return s;
-    swiglu_split_kernel<<<296, 256, 0, cs>>>(pf.wide, R, f, pf.h_hi, pf.h_lo);
+    const int sg = ksplit(2 * f, d);
+    if (sg == 1) {   // SwiGLU in the GEMM's epilogue
+      a = TcArgs{}; a.M = R; a.N = 2 * f; a.K = d; a.mode = TC_OUT_SWIGLU; a.alpha = 1.f; a.out_hi = pf.g_hi; a.out_lo = pf.g_lo; a.ldo = f;
+      if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wgu, d, 2 * f, 1, (size_t)d * 2, (size_t)2 * f * d * 2}, a, false, 1, bt->gemm_ws,
+                       wide(2 * f, d)))) return s;
+    } else {
+      a = TcArgs{}; a.M = R; a.N = 2 * f; a.K = d; a.mode = TC_OUT_F32; a.alpha = 1.f; a.out_f32 = pf.wide; a.ldo = 2 * f;
+      if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wgu, d, 2 * f, 1, (size_t)d * 2, (size_t)2 * f * d * 2}, a, false, sg, bt->gemm_ws,
+                       wide(2 * f, d)))) return s;
+      swiglu_split_kernel<<<296, 256, 0, cs>>>(pf.wide, R, f, pf.g_hi, pf.g_lo);
+    }
     a = TcArgs{}; a.M = R; a.N = d; a.K = f; a.mode = TC_OUT_F32_ADD; a.alpha = 1.f; a.out_f32 = X; a.ldo = d;
     const int sd = ksplit(d, f);
-    if ((s = tc_gemm(ctx, {pf.h_hi, f, R, 1, (size_t)f * 2, (size_t)R * f * 2}, {pf.h_lo, f, R, 1, (size_t)f * 2, (size_t)R * f * 2},
+    if ((s = tc_gemm(ctx, {pf.g_hi, f, R, 1, (size_t)f * 2, (size_t)R * f * 2}, {pf.g_lo, f, R, 1, (size_t)f * 2, (size_t)R * f * 2},
                      {w.wd, f, d, 1, (size_t)f * 2, (size_t)d * f * 2}, a, false, sd, bt->gemm_ws, wide(d, f), true))) return s;
     // the norm in front of the next layer (or of the LM head) rides on the residual update
     resid_rms_split_kernel<<<R, 256, 0, cs>>>(X, bt->gemm_ws, sd > 1 ? sd : 0, xs,

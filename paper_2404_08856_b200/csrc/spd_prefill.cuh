@@ -28,7 +28,9 @@ constexpr int TC_BN_WIDE = 256;       // streaming form: two weight tiles per ac
 constexpr int TC_STAGES_WIDE = 3;     // 3 x 64 KB
 constexpr int TC_SMEM_BYTES = tc_smem_bytes(TC_STAGES);
 
-enum : int { TC_OUT_F32 = 0, TC_OUT_F32_ADD = 1, TC_OUT_SPLIT = 2 };
+// TC_OUT_SWIGLU: the B rows are [gate_0, up_0, gate_1, up_1, ...]; output column i of the hi/lo result
+// [M][N/2] is silu(alpha * gate_i) * (alpha * up_i) (the feed-forward block's non-linearity).
+enum : int { TC_OUT_F32 = 0, TC_OUT_F32_ADD = 1, TC_OUT_SPLIT = 2, TC_OUT_SWIGLU = 3 };
 
 struct TcArgs {
   int M, N, K;              // A rows, B rows (= output columns), inner dimension
@@ -187,7 +189,37 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
         // a thread owns 32 consecutive columns of its row: 16-byte stores where the row start
         // and the width allow it (ldo and out_batch multiples of 8, all 32 columns present)
         const bool vec = nv == 32 && (a.ldo & 7) == 0 && (a.out_batch & 7) == 0;
-        if (a.mode == TC_OUT_SPLIT) {
+        if (a.mode == TC_OUT_SWIGLU) {
+          // this thread's 32 columns are 16 (gate, up) pairs -> 16 output columns from col0 / 2 on
+          const long long off2 = (long long)z * a.out_batch + (long long)row * a.ldo + (col0 >> 1);
+          const int np = nv >> 1;
+          if (np == 16 && (a.ldo & 7) == 0 && (a.out_batch & 7) == 0) {
+#pragma unroll
+            for (int j = 0; j < 16; j += 8) {
+              uint32_t hw[4], lw[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const float g0 = __uint_as_float(v[2 * (j + 2 * q)]) * a.alpha, u0 = __uint_as_float(v[2 * (j + 2 * q) + 1]) * a.alpha;
+                const float g1 = __uint_as_float(v[2 * (j + 2 * q) + 2]) * a.alpha, u1 = __uint_as_float(v[2 * (j + 2 * q) + 3]) * a.alpha;
+                const float x0 = (g0 / (1.0f + expf(-g0))) * u0, x1 = (g1 / (1.0f + expf(-g1))) * u1;
+                const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+                const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - __low2float(h), x1 - __high2float(h));
+                hw[q] = *reinterpret_cast<const uint32_t*>(&h);
+                lw[q] = *reinterpret_cast<const uint32_t*>(&l);
+              }
+              *reinterpret_cast<uint4*>(a.out_hi + off2 + j) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+              *reinterpret_cast<uint4*>(a.out_lo + off2 + j) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+            }
+          } else {
+            for (int j = 0; j < np; ++j) {
+              const float g0 = __uint_as_float(v[2 * j]) * a.alpha, u0 = __uint_as_float(v[2 * j + 1]) * a.alpha;
+              const float x0 = (g0 / (1.0f + expf(-g0))) * u0;
+              const __nv_bfloat16 h0 = __float2bfloat16_rn(x0);
+              a.out_hi[off2 + j] = h0;
+              a.out_lo[off2 + j] = __float2bfloat16_rn(x0 - __bfloat162float(h0));
+            }
+          }
+        } else if (a.mode == TC_OUT_SPLIT) {
           if (vec) {
 #pragma unroll
             for (int j = 0; j < 32; j += 8) {
@@ -408,11 +440,12 @@ __global__ void __launch_bounds__(256) softmax_causal_split_kernel(const float* 
     store_split(hi, lo, base + k, k < n ? expf(row[k] - mx) / tot : 0.f);
 }
 
-// gu fp32 [R][2f] = [gate | up] -> silu(gate) * up, split into hi/lo [R][f]
+// gu fp32 [R][2f] = [gate_0, up_0, gate_1, up_1, ...] -> silu(gate) * up, split into hi/lo [R][f]
+// (used where the gate/up projection was cut into K slices and could not apply it in its epilogue)
 __global__ void swiglu_split_kernel(const float* gu, int R, int f, __nv_bfloat16* hi, __nv_bfloat16* lo) {
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < (size_t)R * f; i += (size_t)gridDim.x * blockDim.x) {
     const size_t r = i / f, c = i - r * f;
-    const float g = gu[r * 2 * f + c], u = gu[r * 2 * f + f + c];
+    const float g = gu[r * 2 * f + 2 * c], u = gu[r * 2 * f + 2 * c + 1];
     store_split(hi, lo, i, (g / (1.0f + expf(-g))) * u);
   }
 }
