@@ -1009,6 +1009,15 @@ __device__ __forceinline__ void split_frag(float2 xa, float2 xb, uint32_t& h0, u
   l1 = pack_bf16(xb.x - bf16lo(h1), xb.y - bf16hi(h1));
 }
 
+// Piece i of a K/V tile -> (row, 16-byte piece of the row).  The long units of the batched kernel
+// (SHIFT) use the fact that a row has a power-of-two number of pieces; the decode kernel keeps
+// the division (its instruction stream is left exactly as it was measured).
+template <bool SHIFT>
+__device__ __forceinline__ void piece_of(int i, int cpr, int csh, int& r, int& cc) {
+  if constexpr (SHIFT) { r = i >> csh; cc = i & (cpr - 1); }
+  else { r = i / cpr; cc = i - r * cpr; }
+}
+
 // bf16 KV cache: the same unit / split / merge scheme as attn_phase, with both products on
 // the tensor cores.  Scores: D[16 positions x 8 queries] = K tile (A, ldmatrix) x q^T (B,
 // fp32 q split into bf16 hi + lo).  Output: D[16 dims x 8 queries] = V^T (A, transposing
@@ -1046,8 +1055,10 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int ns
     char* Kt = Kt0 + (size_t)buf * 2 * tileb;
     char* Vt = Kt + tileb;
     const int n16 = (n + 15) & ~15;
+    const int csh = 31 - __clz(cpr);     // 16-byte pieces per row: a power of two
     for (int i = tid; i < n16 * cpr; i += CONSUMER_THREADS) {
-      const int r = i / cpr, cc = i - r * cpr;
+      int r, cc;
+      piece_of<PIPE>(i, cpr, csh, r, cc);
       const int dst = r * rowb + ((cc ^ (r & 7)) << 4);
       if (r < n) {
         const size_t g = (((size_t)h * md.max_seq + c0 + r) * dh) * 2 + (size_t)cc * 16;
