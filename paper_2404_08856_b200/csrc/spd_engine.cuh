@@ -1039,17 +1039,26 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int ns
   const char* Kl = static_cast<const char*>(md.kcache) + (size_t)layer * md.max_seq * d * 2;
   const char* Vl = static_cast<const char*>(md.vcache) + (size_t)layer * md.max_seq * d * 2;
   // scratch: q [M][dh+8] fp32 | NB x (K tile [SC][rowb] | V tile [SC][rowb]) | S [M][SC+8] fp32
+  // PIPE also keeps q and the probabilities as packed bf16 (hi, lo) pairs -- the B fragments of the
+  // MMAs as they are -- so that the fp32 -> hi/lo split is done once per unit / per probability
+  // instead of once per use: + Qh | Ql [M][dh/2+4] words behind q, + Ph | Pl [M][SC/2+4] words behind S
   constexpr int NB = PIPE ? 2 : 1;
-  int SC = ((xbytes - M * qst * 4 - M * 8 * 4) / (2 * NB * rowb + M * 4)) & ~15;
+  const int qw = (dh >> 1) + 4;                              // words per packed q row
+  const int qpk = PIPE ? 2 * M * qw * 4 : 0;
+  int SC = ((xbytes - M * qst * 4 - qpk - M * 8 * 4 - (PIPE ? M * 8 * 4 : 0)) / (2 * NB * rowb + M * (PIPE ? 8 : 4))) & ~15;
   {  // equal sub-chunks instead of full ones plus a sliver
     const int nsub = (Lc + SC - 1) / SC;
     SC = min(SC, (((Lc + nsub - 1) / nsub) + 15) & ~15);
   }
-  const int sst = SC + 8;
+  const int sst = SC + 8, pw = (SC >> 1) + 4;                // fp32 row of S, words per packed probability row
   float* qs = reinterpret_cast<float*>(xs);
-  char* const Kt0 = xs + M * qst * 4;
+  uint32_t* Qh = reinterpret_cast<uint32_t*>(xs + M * qst * 4);
+  uint32_t* Ql = Qh + M * qw;
+  char* const Kt0 = xs + M * qst * 4 + qpk;
   const size_t tileb = (size_t)SC * rowb;
   float* S = reinterpret_cast<float*>(Kt0 + 2 * NB * tileb);
+  uint32_t* Ph = reinterpret_cast<uint32_t*>(S + M * sst);
+  uint32_t* Pl = Ph + M * pw;
   // request rows [c0, c0 + n) of the head's K and V into tile buffer `buf`
   auto request = [&](int h, int c0, int n, int buf) {
     char* Kt = Kt0 + (size_t)buf * 2 * tileb;
@@ -1101,18 +1110,37 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int ns
       char* Kt = Kt0 + (size_t)buf * 2 * tileb;
       char* Vt = Kt + tileb;
       named_sync(1, CONSUMER_THREADS);
+      if constexpr (PIPE) {
+        if (c0 == p0) {   // q has arrived with the first sub-chunk: split it once for the whole unit
+          for (int i = tid; i < M * (dh >> 1); i += CONSUMER_THREADS) {
+            const int m = i / (dh >> 1), j = i - m * (dh >> 1);
+            const float2 x = *reinterpret_cast<const float2*>(qs + m * qst + 2 * j);
+            const uint32_t hq = pack_bf16(x.x, x.y);
+            Qh[m * qw + j] = hq;
+            Ql[m * qw + j] = pack_bf16(x.x - bf16lo(hq), x.y - bf16hi(hq));
+          }
+          named_sync(1, CONSUMER_THREADS);
+        }
+      }
       // ---- scores: warp takes 16-position groups
       for (int gp = warp; gp * 16 < n; gp += 8) {
         float dsc[4] = {0.f, 0.f, 0.f, 0.f};
         for (int kd = 0; kd < nkd; ++kd) {
-          float2 xa = make_float2(0.f, 0.f), xb = make_float2(0.f, 0.f);
-          if (gq < M) {
-            const float* qr = qs + gq * qst + kd * 16 + 2 * tq;
-            xa = *reinterpret_cast<const float2*>(qr);
-            xb = *reinterpret_cast<const float2*>(qr + 8);
+          uint32_t b0 = 0, b1 = 0, b2 = 0, b3 = 0;
+          if constexpr (PIPE) {
+            if (gq < M) {
+              const int w = gq * qw + kd * 8 + tq;
+              b0 = Qh[w]; b1 = Qh[w + 4]; b2 = Ql[w]; b3 = Ql[w + 4];
+            }
+          } else {
+            float2 xa = make_float2(0.f, 0.f), xb = make_float2(0.f, 0.f);
+            if (gq < M) {
+              const float* qr = qs + gq * qst + kd * 16 + 2 * tq;
+              xa = *reinterpret_cast<const float2*>(qr);
+              xb = *reinterpret_cast<const float2*>(qr + 8);
+            }
+            split_frag(xa, xb, b0, b1, b2, b3);
           }
-          uint32_t b0, b1, b2, b3;
-          split_frag(xa, xb, b0, b1, b2, b3);
           const int r = gp * 16 + (mat & 1) * 8 + rr;
           const int ch = (kd * 2 + (mat >> 1)) ^ (r & 7);
           uint32_t a0, a1, a2, a3;
@@ -1142,10 +1170,21 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int ns
         const float old = ctl->rowmax[warp];
         const float nm = fmaxf(old, mx);
         float sum = 0.f;
-        for (int i = lane; i < n16; i += 32) {
-          const float ex = (nm == -INFINITY) ? 0.f : expf(row[i] - nm);
-          row[i] = ex;
-          sum += ex;
+        if constexpr (PIPE) {   // probabilities leave as packed (hi, lo) pairs of two positions
+          for (int i = 2 * lane; i < n16; i += 64) {
+            const float2 sv = *reinterpret_cast<const float2*>(row + i);
+            const float e0 = (nm == -INFINITY) ? 0.f : expf(sv.x - nm), e1 = (nm == -INFINITY) ? 0.f : expf(sv.y - nm);
+            const uint32_t hp = pack_bf16(e0, e1);
+            Ph[warp * pw + (i >> 1)] = hp;
+            Pl[warp * pw + (i >> 1)] = pack_bf16(e0 - bf16lo(hp), e1 - bf16hi(hp));
+            sum += e0 + e1;
+          }
+        } else {
+          for (int i = lane; i < n16; i += 32) {
+            const float ex = (nm == -INFINITY) ? 0.f : expf(row[i] - nm);
+            row[i] = ex;
+            sum += ex;
+          }
         }
 #pragma unroll
         for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
@@ -1162,14 +1201,21 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int ns
         const float r0s = 2 * tq < M ? ctl->red[0][2 * tq] : 0.f, r1s = 2 * tq + 1 < M ? ctl->red[0][2 * tq + 1] : 0.f;
         oacc[0] *= r0s; oacc[1] *= r1s; oacc[2] *= r0s; oacc[3] *= r1s;
         for (int kp = 0; kp * 16 < n; ++kp) {
-          float2 xa = make_float2(0.f, 0.f), xb = make_float2(0.f, 0.f);
-          if (gq < M) {
-            const float* pr = S + gq * sst + kp * 16 + 2 * tq;
-            xa = *reinterpret_cast<const float2*>(pr);
-            xb = *reinterpret_cast<const float2*>(pr + 8);
+          uint32_t b0 = 0, b1 = 0, b2 = 0, b3 = 0;
+          if constexpr (PIPE) {
+            if (gq < M) {
+              const int w = gq * pw + kp * 8 + tq;
+              b0 = Ph[w]; b1 = Ph[w + 4]; b2 = Pl[w]; b3 = Pl[w + 4];
+            }
+          } else {
+            float2 xa = make_float2(0.f, 0.f), xb = make_float2(0.f, 0.f);
+            if (gq < M) {
+              const float* pr = S + gq * sst + kp * 16 + 2 * tq;
+              xa = *reinterpret_cast<const float2*>(pr);
+              xb = *reinterpret_cast<const float2*>(pr + 8);
+            }
+            split_frag(xa, xb, b0, b1, b2, b3);
           }
-          uint32_t b0, b1, b2, b3;
-          split_frag(xa, xb, b0, b1, b2, b3);
           // A = V^T: matrices {pos 0-7 x dims 0-7, pos 0-7 x dims 8-15, pos 8-15 x dims 0-7, pos 8-15 x dims 8-15}
           const int r = kp * 16 + (mat >> 1) * 8 + rr;
           const int ch = (warp * 2 + (mat & 1)) ^ (r & 7);
