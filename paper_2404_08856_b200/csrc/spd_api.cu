@@ -645,16 +645,17 @@ struct Operand { const void* ptr; int inner, rows, batch; size_t row_stride, bat
 // stream_ksplit = 0: the prefill form (3 stages, two CTAs per SM).  > 0: few rows against a large
 // weight matrix -- 6 stages, one CTA per SM, and the K loop cut into that many slices so that
 // enough CTAs stream; the slices' partial products go to `ws` and are summed in slice order.
-// `wide`: the streaming form with 256-row weight tiles (one activation tile per two weight tiles).
+// `wide`: weight-tile rows of the streaming form (0 or 128, 160, 256): the wider, the fewer activation bytes
+// re-read per weight byte.
 spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const Operand& b, TcArgs args,
-                   bool gelu = false, int stream_ksplit = 0, float* ws = nullptr, bool wide = false,
+                   bool gelu = false, int stream_ksplit = 0, float* ws = nullptr, int wide = 0,
                    bool leave_slices = false) {
   CUtensorMap ma, ml, mb;
   spd_status s;
   if ((s = make_map(ctx, &ma, a_hi.ptr, a_hi.inner, a_hi.rows, a_hi.batch, a_hi.row_stride, a_hi.batch_stride))) return s;
   if ((s = make_map(ctx, &ml, a_lo.ptr, a_lo.inner, a_lo.rows, a_lo.batch, a_lo.row_stride, a_lo.batch_stride))) return s;
   if ((s = make_map(ctx, &mb, b.ptr, b.inner, b.rows, b.batch, b.row_stride, b.batch_stride,
-                    wide && stream_ksplit > 0 ? TC_BN_WIDE : TC_BN))) return s;
+                    stream_ksplit > 0 && wide > 0 ? wide : TC_BN))) return s;
   static bool attr_set[MAX_DEV];
   if (ctx->device < 0 || ctx->device >= MAX_DEV) return fail(ctx, SPD_ECUDA, "device index out of range");
   if (!attr_set[ctx->device]) {
@@ -664,6 +665,8 @@ spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const
                             tc_smem_bytes(TC_STAGES_STREAM)));
     CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel<false, TC_STAGES_WIDE, TC_BN_WIDE>,
                             cudaFuncAttributeMaxDynamicSharedMemorySize, tc_smem_bytes(TC_STAGES_WIDE, TC_BN_WIDE)));
+    CU(cudaFuncSetAttribute((const void*)tc_gemm_kernel<false, TC_STAGES_MID, TC_BN_MID>,
+                            cudaFuncAttributeMaxDynamicSharedMemorySize, tc_smem_bytes(TC_STAGES_MID, TC_BN_MID)));
     attr_set[ctx->device] = true;
   }
   args.split = 1;
@@ -679,10 +682,13 @@ spd_status tc_gemm(spd_ctx* ctx, const Operand& a_hi, const Operand& a_lo, const
       if (!ws || ldo != args.N) return fail(ctx, SPD_EINVAL, "split GEMM needs a workspace and a dense output");
       args.ksplit = stream_ksplit; args.out_f32 = ws; args.mode = TC_OUT_F32;
     }
-    const int bn = wide ? TC_BN_WIDE : TC_BN;
+    if (wide != 0 && wide != TC_BN && wide != TC_BN_MID && wide != TC_BN_WIDE) return fail(ctx, SPD_EINVAL, "streaming GEMM: tile width");
+    const int bn = wide > 0 ? wide : TC_BN;
     dim3 grid((args.N + bn - 1) / bn, (args.M + TC_BM - 1) / TC_BM, stream_ksplit);
-    if (wide)
+    if (bn == TC_BN_WIDE)
       tc_gemm_kernel<false, TC_STAGES_WIDE, TC_BN_WIDE><<<grid, 128, tc_smem_bytes(TC_STAGES_WIDE, TC_BN_WIDE), ctx->stream>>>(ma, ml, mb, args);
+    else if (bn == TC_BN_MID)
+      tc_gemm_kernel<false, TC_STAGES_MID, TC_BN_MID><<<grid, 128, tc_smem_bytes(TC_STAGES_MID, TC_BN_MID), ctx->stream>>>(ma, ml, mb, args);
     else
       tc_gemm_kernel<false, TC_STAGES_STREAM><<<grid, 128, tc_smem_bytes(TC_STAGES_STREAM), ctx->stream>>>(ma, ml, mb, args);
     if (stream_ksplit > 1 && !leave_slices)   // (leave_slices: the caller's next kernel adds them up)
@@ -1494,8 +1500,11 @@ spd_status batch_forward(spd_batch* bt, bool draft, int M, int j) {
   if (attn_split > mh.md.nsplit) attn_split = mh.md.nsplit;
   if (attn_split < 1) attn_split = 1;
   // every GEMM here is a few rows against a large weight matrix: cut K so that about one CTA per SM streams
-  // K slices: up to one CTA per SM, never a second wave, at least 8 K blocks per slice.  256-row weight
-  // tiles (half the activation re-reads of 128-row ones) wherever they still give half the SMs a CTA.
+  // K slices: up to one CTA per SM, never a second wave, at least 8 K blocks per slice.  Weight-tile
+  // width (256, 160 or 128 rows): a CTA moves (width + 2 x 128) x K / slices bytes per 64 columns of K
+  // -- its weight rows plus the hi and lo activation tiles -- so the pair (width, slices) that fits
+  // one wave with the fewest bytes per CTA streams fastest; widths whose grid would leave more than
+  // half the SMs without a CTA are not considered.
   auto slices = [&](int N, int K, int bn) {
     const int tiles = (N + bn - 1) / bn, kb = (K + TC_BK - 1) / TC_BK;
     int sp = ctx->n_sm / tiles;
@@ -1504,9 +1513,18 @@ spd_status batch_forward(spd_batch* bt, bool draft, int M, int j) {
     return sp < 1 ? 1 : sp;
   };
   auto wide = [&](int N, int K) {
-    return ((N + TC_BN_WIDE - 1) / TC_BN_WIDE) * slices(N, K, TC_BN_WIDE) * 2 >= ctx->n_sm;
+    int best = TC_BN;
+    double best_cost = 0.0;
+    for (int bn : {TC_BN_WIDE, TC_BN_MID, TC_BN}) {
+      const int tiles = (N + bn - 1) / bn, sp = slices(N, K, bn);
+      if (bn != TC_BN && (tiles * sp * 2 < ctx->n_sm || tiles > ctx->n_sm)) continue;
+      const double waves = (double)((tiles * sp + ctx->n_sm - 1) / ctx->n_sm);
+      const double cost = waves * (double)(bn + 2 * TC_BM) * K / sp;
+      if (best_cost == 0.0 || cost < best_cost) { best_cost = cost; best = bn; }
+    }
+    return best;
   };
-  auto ksplit = [&](int N, int K) { return slices(N, K, wide(N, K) ? TC_BN_WIDE : TC_BN); };
+  auto ksplit = [&](int N, int K) { return slices(N, K, wide(N, K)); };
   // Where a projection is cut into K slices, the kernel that reads its result adds the slices up
   // (in slice order): the rotary / cache-append kernel for QKV, the fused residual + RMSNorm + split
   // kernel for the output and down projections.

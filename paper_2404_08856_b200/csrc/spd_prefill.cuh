@@ -26,6 +26,9 @@ __host__ __device__ constexpr int tc_stage_bytes(int bn) { return 2 * TC_A_BYTES
 __host__ __device__ constexpr int tc_smem_bytes(int stages, int bn = TC_BN) { return stages * tc_stage_bytes(bn) + 1024 + 256; }   // + alignment slack + barriers
 constexpr int TC_BN_WIDE = 256;       // streaming form: two weight tiles per activation tile (half the activation re-reads)
 constexpr int TC_STAGES_WIDE = 3;     // 3 x 64 KB
+constexpr int TC_BN_MID = 160;        // ... or 160 weight rows, where 256-row tiles would leave too many SMs without a CTA
+constexpr int TC_STAGES_MID = 4;      // 4 x 52 KB
+__host__ __device__ constexpr int tc_tmem_cols(int bn) { return bn <= 128 ? 128 : 256; }   // allocations are powers of two
 constexpr int TC_SMEM_BYTES = tc_smem_bytes(TC_STAGES);
 
 // TC_OUT_SWIGLU: the B rows are [gate_0, up_0, gate_1, up_1, ...]; output column i of the hi/lo result
@@ -119,7 +122,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(BN)
+                 "r"(tc_tmem_cols(BN))
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -280,7 +283,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
   __syncthreads();
   if (warp == 0) {
     if (!done) for (int i = 0; i < 200; ++i) __nanosleep(1000);   // let copies in flight land
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tc_tmem_cols(BN)) : "memory");
   }
 }
 
