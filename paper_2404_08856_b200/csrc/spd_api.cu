@@ -1449,7 +1449,7 @@ constexpr int BATCH_KSPLIT_MAX = 8;
 
 template <int M>
 spd_status launch_batch_attn(spd_ctx* ctx, const ModelDev* mds, const int* origins, int B, int layer, int chain0,
-                             int max_split) {
+                             int max_split, __nv_bfloat16* o_hi, __nv_bfloat16* o_lo) {
   static bool attr[MAX_DEV];
   const size_t smem = CTRL_BYTES + BATCH_ATTN_SCRATCH;
   if (!attr[ctx->device]) {
@@ -1457,22 +1457,22 @@ spd_status launch_batch_attn(spd_ctx* ctx, const ModelDev* mds, const int* origi
     attr[ctx->device] = true;
   }
   batch_attn_kernel<M><<<2 * ctx->n_sm, CONSUMER_THREADS, smem, ctx->stream>>>(mds, origins, B, layer, chain0,
-                                                                          BATCH_ATTN_SCRATCH, max_split);
+                                                                          BATCH_ATTN_SCRATCH, max_split, o_hi, o_lo);
   CU(cudaGetLastError());
   return SPD_OK;
 }
 
 spd_status batch_attn(spd_ctx* ctx, int M, const ModelDev* mds, const int* origins, int B, int layer, int chain0,
-                      int max_split) {
+                      int max_split, __nv_bfloat16* o_hi, __nv_bfloat16* o_lo) {
   switch (M) {
-    case 1: return launch_batch_attn<1>(ctx, mds, origins, B, layer, chain0, max_split);
-    case 2: return launch_batch_attn<2>(ctx, mds, origins, B, layer, chain0, max_split);
-    case 3: return launch_batch_attn<3>(ctx, mds, origins, B, layer, chain0, max_split);
-    case 4: return launch_batch_attn<4>(ctx, mds, origins, B, layer, chain0, max_split);
-    case 5: return launch_batch_attn<5>(ctx, mds, origins, B, layer, chain0, max_split);
-    case 6: return launch_batch_attn<6>(ctx, mds, origins, B, layer, chain0, max_split);
-    case 7: return launch_batch_attn<7>(ctx, mds, origins, B, layer, chain0, max_split);
-    default: return launch_batch_attn<8>(ctx, mds, origins, B, layer, chain0, max_split);
+    case 1: return launch_batch_attn<1>(ctx, mds, origins, B, layer, chain0, max_split, o_hi, o_lo);
+    case 2: return launch_batch_attn<2>(ctx, mds, origins, B, layer, chain0, max_split, o_hi, o_lo);
+    case 3: return launch_batch_attn<3>(ctx, mds, origins, B, layer, chain0, max_split, o_hi, o_lo);
+    case 4: return launch_batch_attn<4>(ctx, mds, origins, B, layer, chain0, max_split, o_hi, o_lo);
+    case 5: return launch_batch_attn<5>(ctx, mds, origins, B, layer, chain0, max_split, o_hi, o_lo);
+    case 6: return launch_batch_attn<6>(ctx, mds, origins, B, layer, chain0, max_split, o_hi, o_lo);
+    case 7: return launch_batch_attn<7>(ctx, mds, origins, B, layer, chain0, max_split, o_hi, o_lo);
+    default: return launch_batch_attn<8>(ctx, mds, origins, B, layer, chain0, max_split, o_hi, o_lo);
   }
 }
 
@@ -1539,8 +1539,8 @@ spd_status batch_forward(spd_batch* bt, bool draft, int M, int j) {
                      wide(3 * d, d), true))) return s;
     batch_rope_append_kernel<<<1184, 256, 0, cs>>>(sq > 1 ? bt->gemm_ws : pf.wide, sq, R, M, d, dh, bt->rowslot,
                                                  mh.md.rope_cos, mh.md.rope_sin, mds, l);
-    if ((s = batch_attn(ctx, M, mds, bt->origins, B, l, draft ? j - 1 : 0, attn_split))) return s;
-    batch_gather_split_kernel<<<296, 256, 0, cs>>>(mds, R, M, d, pf.h_hi, pf.h_lo);
+    // (the attention kernel leaves its rows as the hi/lo operand of the output projection)
+    if ((s = batch_attn(ctx, M, mds, bt->origins, B, l, draft ? j - 1 : 0, attn_split, pf.h_hi, pf.h_lo))) return s;
     a = TcArgs{}; a.M = R; a.N = d; a.K = d; a.mode = TC_OUT_F32_ADD; a.alpha = 1.f; a.out_f32 = X; a.ldo = d;
     const int so = ksplit(d, d);
     if ((s = tc_gemm(ctx, h_hi, h_lo, {w.wo, d, d, 1, (size_t)d * 2, (size_t)d * d * 2}, a, false, so, bt->gemm_ws, wide(d, d),

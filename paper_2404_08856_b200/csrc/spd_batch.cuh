@@ -91,9 +91,12 @@ __global__ void batch_rope_append_kernel(const float* qkv, int slices, int R, in
 // attends the rows from the origin up to its own.
 // `max_split`: KV splits per head at most -- with B sequences there are enough (sequence, head) pairs
 // to fill the grid, so heads are cut no further than needed (fewer partial results to merge).
+// o_hi / o_lo: every sequence's output rows as one matrix [B * M][d] split into bf16 hi + lo (the
+// operand of the output projection).
 template <int M>
 __global__ void __launch_bounds__(CONSUMER_THREADS, 2) batch_attn_kernel(const ModelDev* mds, const int* origins, int B,
-                                                                      int layer, int chain0, int xbytes, int max_split) {
+                                                                      int layer, int chain0, int xbytes, int max_split,
+                                                                      __nv_bfloat16* o_hi, __nv_bfloat16* o_lo) {
   extern __shared__ __align__(1024) char bsm[];
   Ctrl* ctl = reinterpret_cast<Ctrl*>(bsm);
   char* xs = bsm + CTRL_BYTES;
@@ -110,21 +113,9 @@ __global__ void __launch_bounds__(CONSUMER_THREADS, 2) batch_attn_kernel(const M
     const int units = md.H * eff_nsplit(md, origins[b] + chain0 + M);
     if (u >= units) continue;
     // one unit: the phase's own loop runs once for "CTA u of a grid of `units`"
-    attn_phase_mma<M, true>(md, layer, origins[b], chain0 + M, u, units, xs, xbytes, ctl);
+    const size_t row0 = (size_t)b * M * md.d;
+    attn_phase_mma<M, true>(md, layer, origins[b], chain0 + M, u, units, xs, xbytes, ctl, o_hi + row0, o_lo + row0);
     named_sync(1, CONSUMER_THREADS);
-  }
-}
-
-// Each sequence's attention rows [M][d] (fp32) -> one matrix [R][d] split into bf16 hi + lo.
-__global__ void batch_gather_split_kernel(const ModelDev* mds, int R, int M, int d, __nv_bfloat16* hi,
-                                          __nv_bfloat16* lo) {
-  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < (size_t)R * d; i += (size_t)gridDim.x * blockDim.x) {
-    const int r = (int)(i / d), c = (int)(i - (size_t)r * d);
-    const int b = r / M, m = r - b * M;
-    const float x = __ldcg(mds[b].attn + (size_t)m * d + c);
-    const __nv_bfloat16 h = __float2bfloat16_rn(x);
-    hi[i] = h;
-    lo[i] = __float2bfloat16_rn(x - __bfloat162float(h));
   }
 }
 

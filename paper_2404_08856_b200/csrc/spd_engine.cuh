@@ -1024,10 +1024,11 @@ __device__ __forceinline__ void piece_of(int i, int cpr, int csh, int& r, int& c
 // ldmatrix) x P^T (B, fp32 probabilities split the same way); warp w owns dims 16w..16w+15,
 // so no cross-warp reduction is needed.  Tile rows are 16-byte-chunk swizzled by position.
 // PIPE (the batched kernel, where a unit spans several sub-chunks): two K/V tile buffers, the
-// next sub-chunk's rows are requested before the current one is computed.
+// next sub-chunk's rows are requested before the current one is computed; with o_hi / o_lo the
+// head's output rows [M][d] also leave as bf16 hi + lo (the next GEMM's operand).
 template <int M, bool PIPE = false>
 __device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int nslots, int cta, int G, char* xs,
-                               int xbytes, Ctrl* ctl) {
+                               int xbytes, Ctrl* ctl, __nv_bfloat16* o_hi = nullptr, __nv_bfloat16* o_lo = nullptr) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int H = md.H, dh = md.dh, d = md.d;
   const int len = origin + nslots;
@@ -1234,7 +1235,20 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int ns
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int q = 2 * tq + (j & 1), c = warp * 16 + gq + (j >> 1) * 8;
-          if (q < M) stcg(md.attn + (size_t)q * d + h * dh + c, oacc[j] / ctl->rowsum[q]);
+          if (q < M) {
+            const float v = oacc[j] / ctl->rowsum[q];
+            if constexpr (PIPE) {
+              if (o_hi) {
+                const __nv_bfloat16 hv = __float2bfloat16_rn(v);
+                o_hi[(size_t)q * d + h * dh + c] = hv;
+                o_lo[(size_t)q * d + h * dh + c] = __float2bfloat16_rn(v - __bfloat162float(hv));
+              } else {
+                stcg(md.attn + (size_t)q * d + h * dh + c, v);
+              }
+            } else {
+              stcg(md.attn + (size_t)q * d + h * dh + c, v);
+            }
+          }
         }
       }
       named_sync(1, CONSUMER_THREADS);
@@ -1263,6 +1277,18 @@ __device__ void attn_phase_mma(const ModelDev& md, int layer, int origin, int ns
     named_sync(1, CONSUMER_THREADS);
     if (ctl->flag) merge_head<M>(md, h, nsplit, reinterpret_cast<float*>(Kt0));
     named_sync(1, CONSUMER_THREADS);
+    if constexpr (PIPE) {
+      if (ctl->flag && o_hi) {   // the merged rows of this head, once more as bf16 hi + lo
+        for (int i = tid; i < M * dh; i += CONSUMER_THREADS) {
+          const int m = i / dh, c = i - m * dh;
+          const float v = ldcg(md.attn + (size_t)m * d + h * dh + c);
+          const __nv_bfloat16 hv = __float2bfloat16_rn(v);
+          o_hi[(size_t)m * d + h * dh + c] = hv;
+          o_lo[(size_t)m * d + h * dh + c] = __float2bfloat16_rn(v - __bfloat162float(hv));
+        }
+        named_sync(1, CONSUMER_THREADS);
+      }
+    }
   }
 }
 
